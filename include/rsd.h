@@ -1,0 +1,171 @@
+/*
+ * librsd: the data-parallel hot path of Recursive Speculative Decoding (RSD) on one GPU.
+ *
+ *   drafting      rsd_gumbel_topk_draft   per-node Gumbel-Top-k (sampling without replacement)
+ *                 rsd_sbs_step            one level of Stochastic Beam Search
+ *   verification  rsd_verify_tree         recursive rejection sampling along the draft tree
+ *                 rsd_resample_residual   draw from a residual distribution on its own
+ *
+ * The draft and target language models are outside this library: their logits come in as rows of V values.
+ *
+ * Conventions that hold for every entry point
+ *   - Plain C ABI.  Unless an argument says "host", pointers are DEVICE pointers owned by the caller; the library
+ *     never allocates or frees device memory.  The small structs (rsd_rows, rsd_tree) live in host memory and are
+ *     read before the call returns.
+ *   - Work is enqueued on `stream` (a cudaStream_t) and the call returns without waiting for it.
+ *   - The return value reports argument and launch errors only (RSD_OK = 0); rsd_last_error() gives a message for
+ *     the calling thread.  Data-dependent trouble (NaN logits, rows with fewer than k finite entries, an empty
+ *     residual) never traps: it sets bits in the per-sequence `status` output and follows the documented fallback.
+ *     Each call overwrites status[0..B).
+ *   - Rows: element (b, r, x) of a batch of rows sits at data + b*seq_stride + r*row_stride + x (strides in
+ *     elements).  fp32 or bf16 storage; all arithmetic is fp32 or wider.  The vectorised path needs the base
+ *     pointer and both strides to be multiples of 16 bytes; anything else takes a slower scalar path with the same
+ *     results.
+ *   - Tree layout: flat node index, root = 0, then level by level in stored order.  parent[n] is the flat index of
+ *     n's parent (root: -1).  Siblings are ordered by increasing flat index, which is the order the drafting calls
+ *     produce (decreasing perturbed value).  A node with token[n] < 0 is absent.
+ *   - Randomness is a pure function of (seed, step, global sequence index, flat node id, stream tag, index), drawn
+ *     from Philox4x32-10 (Salmon et al., SC'11): key = (seed low word, seed high word), counter = (index,
+ *     node | tag << 28, sequence, step).  Global sequence index = seq_base + b, so a batch may be split over
+ *     several GPUs without changing any result.  Streams (rsd_rng_layout() == 1):
+ *       tag 0  Gumbel, coarse : index = x >> 4; output byte x & 15 (little-endian over the 4 words) is the top
+ *                               byte of element x's 32 random bits
+ *       tag 1  Gumbel, fine   : index = x >> 2; the upper 24 bits of output word x & 3 are the low 24 bits
+ *              U = (bits + 1/2) / 2^32,  G = -ln(-ln U)
+ *       tag 2  acceptance     : index = rank of the child among its siblings; U = (word0 >> 8) / 2^24
+ *       tag 3  final token    : index = 0; u = (word0 + 1/2) / 2^32
+ *     The same (seed, step, inputs) give bit-identical outputs whatever the launch shape.
+ */
+#ifndef RSD_H_
+#define RSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void* rsd_stream_t; /* a cudaStream_t */
+
+enum { RSD_OK = 0, RSD_ERR_INVALID_ARG = 1, RSD_ERR_UNSUPPORTED = 2, RSD_ERR_WORKSPACE = 3, RSD_ERR_CUDA = 4 };
+enum { RSD_F32 = 0, RSD_BF16 = 1 };
+
+/* bits of status[b] */
+enum {
+    RSD_ST_NAN_INPUT = 1,       /* a NaN logit was read; it was treated as -inf */
+    RSD_ST_FEWER_THAN_K = 2,    /* a row had fewer finite entries than picks asked for; outputs padded with -1 */
+    RSD_ST_ZERO_RESIDUAL = 4,   /* sum of [q - p]+ was not positive; the previous residual was kept */
+    RSD_ST_ZERO_DRAFT_PROB = 8, /* a child token had draft probability 0; accepted iff its residual mass is > 0 */
+    RSD_ST_DRAFT_EXHAUSTED = 16 /* the draft had no mass left after a removal; later siblings were ignored */
+};
+
+/* stop_reason[b] of the verification walk */
+enum { RSD_STOP_ALL_REJECTED = 0, RSD_STOP_NO_CHILDREN = 1, RSD_STOP_LEAF = 2 };
+
+enum {
+    RSD_MAX_K = 32,              /* largest number of picks per row / beam width */
+    RSD_MAX_ROWS_PER_SEQ = 256,  /* largest R of rsd_gumbel_topk_draft and n_par of rsd_sbs_step */
+    RSD_MAX_VOCAB = 262144,
+    RSD_MAX_TREE_NODES = 4096    /* largest N + 1 */
+};
+
+typedef struct rsd_rows {
+    const void* data;   /* device */
+    int32_t dtype;      /* RSD_F32 or RSD_BF16 */
+    int32_t is_logprob; /* 1: rows are log-probabilities already (drafting uses them as given) */
+    int64_t seq_stride; /* elements between sequences */
+    int64_t row_stride; /* elements between rows of one sequence, >= V */
+} rsd_rows;
+
+typedef struct rsd_tree {
+    int32_t num_levels;         /* L */
+    int32_t num_nodes;          /* N + 1, root included */
+    const int32_t* parent;      /* device, [num_nodes] if topology_is_shared else [B][num_nodes] */
+    const int32_t* token;       /* device, [B][num_nodes]; root entry unused */
+    int32_t topology_is_shared; /* 1: one parent[] for all sequences (constant branching factors) */
+} rsd_tree;
+
+int rsd_version(void);
+int rsd_rng_layout(void);
+/* Message of the last error on the calling thread ("" if none).  Host pointer, valid until the next call. */
+const char* rsd_last_error(void);
+
+/*
+ * Gumbel-Top-k drafting for RSD with constant branching factors (Section 3.2.1, Eqs. 5-8; Algorithm 4).
+ * For each of the B*R rows: phi = log-softmax(row) (Eq. 5), phi~ = phi + G (Eq. 6), and the k_per_row[r] tokens
+ * with the largest phi~ in decreasing order (Eq. 7); equal values go to the smaller token.  The noise of row r is
+ * the Gumbel stream of node rng_node[r] of the sequence.  The arg-top-k does not depend on the row's normaliser,
+ * so the log-sum-exp is computed only when out_perturbed or out_logprob is asked for.
+ *   draft        rows [B][R][V]
+ *   k_per_row    host [R], 1 <= k <= max_k <= RSD_MAX_K
+ *   rng_node     host [R], flat node id of each row (< 2^28)
+ *   out_token    [B][R][max_k] int32; entries beyond k_per_row[r], or beyond the finite entries of the row, are -1
+ *   out_perturbed, out_logprob  optional (NULL to skip) [B][R][max_k] fp32: phi~ and phi of each pick
+ *   status       [B]
+ */
+int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int32_t* k_per_row,
+                          const int32_t* rng_node, int max_k, uint64_t seed, uint32_t step, uint32_t seq_base,
+                          int32_t* out_token, float* out_perturbed, float* out_logprob, int32_t* status,
+                          rsd_stream_t stream);
+
+/*
+ * One level of Stochastic Beam Search for RSD-S (Section 3.2.1, Eqs. 10-12; Algorithm 9).
+ * Parent slot k of a sequence (flat node first_parent_node + k) has the sequence log-probability
+ * sum_logprob_in[b][k] and the truncated Gumbel trunc_gumbel_in[b][k] (both NULL at the root: zeros).
+ *   phi_k(x)  = sum_logprob_in[k] + log p_k(x)            phi~_k(x) = phi_k(x) + G_k(x)
+ *   psi_k(x)  = T(trunc_gumbel_in[k], phi~_k(x)),  T(u, f) = -log(exp(-u) - exp(-max f) + exp(-f))   (Eq. 11)
+ * and the W pairs (x, k) with the largest psi are returned in decreasing order (Eq. 12); equal values go to the
+ * smaller parent, then the smaller token.  Entries whose log-probability is -inf are dropped.
+ *   draft_level       rows [B][n_par][V], n_par <= RSD_MAX_ROWS_PER_SEQ, W <= RSD_MAX_K
+ *   out_token, out_parent   [B][W] int32 (parent = slot index within the level); -1 beyond out_count[b]
+ *   sum_logprob_out, trunc_gumbel_out  [B][W] fp32: phi and psi of each pick, the next level's inputs
+ *   out_count         [B]
+ *   ws                scratch of at least rsd_sbs_workspace_bytes(B, n_par, W) bytes, 256-byte aligned; contents
+ *                     are undefined afterwards; calls that overlap on the GPU need separate scratch
+ */
+size_t rsd_sbs_workspace_bytes(int B, int n_par, int W);
+int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, int32_t first_parent_node,
+                 const float* sum_logprob_in, const float* trunc_gumbel_in, uint64_t seed, uint32_t step,
+                 uint32_t seq_base, int32_t* out_token, int32_t* out_parent, float* sum_logprob_out,
+                 float* trunc_gumbel_out, int32_t* out_count, int32_t* status, void* ws, size_t ws_bytes,
+                 rsd_stream_t stream);
+
+/*
+ * Draft-tree verification by recursive rejection sampling (Section 3.1, Eqs. 1-4, Algorithm 1; Section 3.2.2,
+ * Algorithm 6).  Per sequence, starting at the root: the children of the current node are tested in stored order
+ * with p = softmax(draft row of the node), q = softmax(target row of the node):
+ *   accept child j with probability min(1, q_j(x_j) / p_j(x_j))                                      (Eq. 3)
+ *   on rejection  q_{j+1} = Norm[(q_j - p_j)+],  p_{j+1} = p_j without x_j, renormalised           (Eqs. 1-2)
+ * The first accepted child becomes the current node.  The walk ends with one more token drawn by inverse CDF:
+ * from the last residual if every child was rejected, from the node's target row if it has no children
+ * (RSD_STOP_NO_CHILDREN) or is at depth L (RSD_STOP_LEAF).  Only the rows of visited nodes are read.
+ *   draft   rows of nodes that can have children (flat ids 0 .. P-1);  target  rows of all nodes (0 .. N)
+ *   accepted_len [B]; accepted_node, accepted_token [B][L] (-1 padded); last_token [B]; stop_reason [B]
+ *   dbg_theta    optional [B][num_nodes] fp32: the acceptance threshold of every child that was tested, NaN elsewhere
+ * draft and target must have the same dtype.  Rows given as log-probabilities are renormalised like logits.
+ */
+int rsd_verify_tree(const rsd_rows* draft, const rsd_rows* target, const rsd_tree* tree, int B, int V,
+                    uint64_t seed, uint32_t step, uint32_t seq_base, int32_t* accepted_len, int32_t* accepted_node,
+                    int32_t* accepted_token, int32_t* last_token, int32_t* stop_reason, float* dbg_theta,
+                    int32_t* status, rsd_stream_t stream);
+
+/*
+ * One draw from a residual distribution (Eq. 2 applied along a list of rejected drafts; Section 2's
+ * Norm[(q - p)+] is the one-token case).  Per sequence: p = softmax(draft row), q = softmax(target row); for each
+ * token of rejected[b][0..max_k) in order (-1 = none) the chain step of Eqs. 1-2 is applied; then one token is
+ * drawn by inverse CDF with the final-token stream of node rng_node[b].  With no rejected token this is a plain
+ * draw from the target row and `draft` may be NULL.
+ *   draft_row, target_row   rows [B][1][V] (row_stride unused)
+ *   rejected     [B][max_k] int32 or NULL;  rng_node [B] int32 (device)
+ *   out_token    [B];  out_residual  optional [B][V] fp32, the normalised distribution drawn from
+ */
+int rsd_resample_residual(const rsd_rows* draft_row, const rsd_rows* target_row, int B, int V,
+                          const int32_t* rejected, int max_k, const int32_t* rng_node, uint64_t seed, uint32_t step,
+                          uint32_t seq_base, int32_t* out_token, float* out_residual, int32_t* status,
+                          rsd_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RSD_H_ */

@@ -1,0 +1,9 @@
+"""B200-native hot path of Recursive Speculative Decoding: Gumbel-Top-k / Stochastic Beam Search drafting and
+recursive rejection sampling over the draft tree, as CUDA kernels (sm_100a) behind a C ABI (include/rsd.h).
+
+The functions below are argument-marshalling wrappers with the names of the C entry points.
+"""
+from .api import (LIB_PATH, MAX_K, RsdError, lib, rows_of, rsd_gumbel_topk_draft, rsd_resample_residual,  # noqa: F401
+                  rsd_sbs_step, rsd_sbs_workspace_bytes, rsd_verify_tree)
+from .api import (ST_DRAFT_EXHAUSTED, ST_FEWER_THAN_K, ST_NAN_INPUT, ST_ZERO_DRAFT_PROB, ST_ZERO_RESIDUAL,  # noqa: F401
+                  STOP_ALL_REJECTED, STOP_LEAF, STOP_NO_CHILDREN)

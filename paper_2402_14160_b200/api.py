@@ -1,0 +1,200 @@
+"""Thin binding over librsd's C ABI (include/rsd.h): argument marshalling only.
+
+Every function takes torch CUDA tensors, passes their device pointers and the current CUDA stream to the entry
+point of the same name, and returns freshly allocated output tensors.  Nothing is computed here.  The library is
+loaded on first use and a missing or unbuilt library raises: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librsd.so")
+
+RSD_F32, RSD_BF16 = 0, 1
+ST_NAN_INPUT, ST_FEWER_THAN_K, ST_ZERO_RESIDUAL, ST_ZERO_DRAFT_PROB, ST_DRAFT_EXHAUSTED = 1, 2, 4, 8, 16
+STOP_ALL_REJECTED, STOP_NO_CHILDREN, STOP_LEAF = 0, 1, 2
+MAX_K = 32
+
+EXPORTS = ["rsd_version", "rsd_rng_layout", "rsd_last_error", "rsd_gumbel_topk_draft", "rsd_sbs_workspace_bytes",
+           "rsd_sbs_step", "rsd_verify_tree", "rsd_resample_residual"]
+
+
+class RsdRows(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("dtype", C.c_int32), ("is_logprob", C.c_int32),
+                ("seq_stride", C.c_int64), ("row_stride", C.c_int64)]
+
+
+class RsdTree(C.Structure):
+    _fields_ = [("num_levels", C.c_int32), ("num_nodes", C.c_int32), ("parent", C.c_void_p),
+                ("token", C.c_void_p), ("topology_is_shared", C.c_int32)]
+
+
+class RsdError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def lib():
+    """The loaded library.  Raises if it has not been built (python -m paper_2402_14160_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RsdError("librsd.so is missing at %s: build it with `python -m paper_2402_14160_b200.build` "
+                           "(there is no fallback path)" % LIB_PATH)
+        l = C.CDLL(LIB_PATH)
+        l.rsd_last_error.restype = C.c_char_p
+        l.rsd_sbs_workspace_bytes.restype = C.c_size_t
+        l.rsd_sbs_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
+        l.rsd_gumbel_topk_draft.argtypes = [C.POINTER(RsdRows), C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                            C.c_int, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_void_p]
+        l.rsd_sbs_step.argtypes = [C.POINTER(RsdRows), C.c_int, C.c_int, C.c_int, C.c_int, C.c_int32, C.c_void_p,
+                                   C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
+                                   C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                   C.c_void_p]
+        l.rsd_verify_tree.argtypes = [C.POINTER(RsdRows), C.POINTER(RsdRows), C.POINTER(RsdTree), C.c_int, C.c_int,
+                                      C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        l.rsd_resample_residual.argtypes = [C.POINTER(RsdRows), C.POINTER(RsdRows), C.c_int, C.c_int, C.c_void_p,
+                                            C.c_int, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_void_p]
+        _lib = l
+    return _lib
+
+
+def _check(code: int):
+    if code != 0:
+        raise RsdError("librsd error %d: %s" % (code, lib().rsd_last_error().decode()))
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def rows_of(t: torch.Tensor, is_logprob: bool = False) -> RsdRows:
+    """Describe a [B, R, V] (or [B, V]) CUDA tensor of fp32 or bf16 rows; the last dimension must be dense."""
+    if not t.is_cuda:
+        raise RsdError("rows must live on a CUDA device")
+    if t.dtype == torch.float32:
+        dt = RSD_F32
+    elif t.dtype == torch.bfloat16:
+        dt = RSD_BF16
+    else:
+        raise RsdError("rows must be float32 or bfloat16")
+    if t.stride(-1) != 1:
+        raise RsdError("rows must be dense along the vocabulary")
+    if t.dim() == 3:
+        return RsdRows(t.data_ptr(), dt, int(is_logprob), t.stride(0), t.stride(1))
+    if t.dim() == 2:
+        return RsdRows(t.data_ptr(), dt, int(is_logprob), t.stride(0), t.shape[1])
+    raise RsdError("rows must be [B, R, V] or [B, V]")
+
+
+def _host_i32(values: Sequence[int]):
+    arr = (C.c_int32 * len(values))(*[int(v) for v in values])
+    return arr
+
+
+def rsd_gumbel_topk_draft(draft: torch.Tensor, k_per_row: Sequence[int], rng_node: Sequence[int], seed: int,
+                          step: int, *, is_logprob: bool = False, seq_base: int = 0, max_k: Optional[int] = None,
+                          want_values: bool = False):
+    """draft [B, R, V] -> dict(token [B, R, max_k], status [B], and perturbed/logprob when want_values)."""
+    B, R, V = draft.shape
+    max_k = int(max_k or max(k_per_row))
+    dev = draft.device
+    token = torch.empty((B, R, max_k), dtype=torch.int32, device=dev)
+    status = torch.empty((B,), dtype=torch.int32, device=dev)
+    pert = torch.empty((B, R, max_k), dtype=torch.float32, device=dev) if want_values else None
+    logp = torch.empty((B, R, max_k), dtype=torch.float32, device=dev) if want_values else None
+    rows = rows_of(draft, is_logprob)
+    _check(lib().rsd_gumbel_topk_draft(C.byref(rows), B, R, V, _host_i32(k_per_row), _host_i32(rng_node), max_k,
+                                       seed, step, seq_base, _ptr(token), _ptr(pert), _ptr(logp), _ptr(status),
+                                       _stream()))
+    return dict(token=token, perturbed=pert, logprob=logp, status=status)
+
+
+def rsd_sbs_workspace_bytes(B: int, n_par: int, W: int) -> int:
+    return int(lib().rsd_sbs_workspace_bytes(B, n_par, W))
+
+
+def rsd_sbs_step(draft_level: torch.Tensor, W: int, first_parent_node: int, sum_logprob_in: Optional[torch.Tensor],
+                 trunc_gumbel_in: Optional[torch.Tensor], seed: int, step: int, *, is_logprob: bool = False,
+                 seq_base: int = 0, workspace: Optional[torch.Tensor] = None, out: Optional[dict] = None):
+    """draft_level [B, n_par, V] -> dict(token, parent, sum_logprob, trunc_gumbel [B, W], count [B], status [B])."""
+    B, n_par, V = draft_level.shape
+    dev = draft_level.device
+    need = rsd_sbs_workspace_bytes(B, n_par, W)
+    if workspace is None:
+        workspace = torch.empty((need,), dtype=torch.uint8, device=dev)
+    if out is None:
+        out = dict(token=torch.empty((B, W), dtype=torch.int32, device=dev),
+                   parent=torch.empty((B, W), dtype=torch.int32, device=dev),
+                   sum_logprob=torch.empty((B, W), dtype=torch.float32, device=dev),
+                   trunc_gumbel=torch.empty((B, W), dtype=torch.float32, device=dev),
+                   count=torch.empty((B,), dtype=torch.int32, device=dev),
+                   status=torch.empty((B,), dtype=torch.int32, device=dev))
+    rows = rows_of(draft_level, is_logprob)
+    _check(lib().rsd_sbs_step(C.byref(rows), B, n_par, V, W, first_parent_node, _ptr(sum_logprob_in),
+                              _ptr(trunc_gumbel_in), seed, step, seq_base, _ptr(out["token"]), _ptr(out["parent"]),
+                              _ptr(out["sum_logprob"]), _ptr(out["trunc_gumbel"]), _ptr(out["count"]),
+                              _ptr(out["status"]), _ptr(workspace), workspace.numel(), _stream()))
+    return out
+
+
+def rsd_verify_tree(draft: torch.Tensor, target: torch.Tensor, parent: torch.Tensor, token: torch.Tensor,
+                    num_levels: int, seed: int, step: int, *, seq_base: int = 0, want_theta: bool = False,
+                    out: Optional[dict] = None):
+    """draft [B, P, V], target [B, N+1, V], parent [N+1] or [B, N+1] int32, token [B, N+1] int32."""
+    B, _, V = target.shape
+    dev = target.device
+    n_nodes = token.shape[1]
+    L = int(num_levels)
+    if parent.dtype != torch.int32 or token.dtype != torch.int32:
+        raise RsdError("parent and token must be int32")
+    if not (parent.is_contiguous() and token.is_contiguous()):
+        raise RsdError("parent and token must be contiguous")
+    if out is None:
+        out = dict(accepted_len=torch.empty((B,), dtype=torch.int32, device=dev),
+                   accepted_node=torch.empty((B, max(L, 1)), dtype=torch.int32, device=dev)[:, :L],
+                   accepted_token=torch.empty((B, max(L, 1)), dtype=torch.int32, device=dev)[:, :L],
+                   last_token=torch.empty((B,), dtype=torch.int32, device=dev),
+                   stop_reason=torch.empty((B,), dtype=torch.int32, device=dev),
+                   status=torch.empty((B,), dtype=torch.int32, device=dev))
+        out["theta"] = torch.empty((B, n_nodes), dtype=torch.float32, device=dev) if want_theta else None
+    tree = RsdTree(L, n_nodes, parent.data_ptr(), token.data_ptr(), 1 if parent.dim() == 1 else 0)
+    d, t = rows_of(draft), rows_of(target)
+    _check(lib().rsd_verify_tree(C.byref(d), C.byref(t), C.byref(tree), B, V, seed, step, seq_base,
+                                 _ptr(out["accepted_len"]), _ptr(out["accepted_node"]), _ptr(out["accepted_token"]),
+                                 _ptr(out["last_token"]), _ptr(out["stop_reason"]), _ptr(out.get("theta")),
+                                 _ptr(out["status"]), _stream()))
+    return out
+
+
+def rsd_resample_residual(draft_row: Optional[torch.Tensor], target_row: torch.Tensor,
+                          rejected: Optional[torch.Tensor], rng_node: torch.Tensor, seed: int, step: int, *,
+                          seq_base: int = 0, want_residual: bool = False):
+    """draft_row/target_row [B, V]; rejected [B, max_k] int32 (-1 padded) or None; rng_node [B] int32."""
+    B, V = target_row.shape
+    dev = target_row.device
+    token = torch.empty((B,), dtype=torch.int32, device=dev)
+    status = torch.empty((B,), dtype=torch.int32, device=dev)
+    residual = torch.empty((B, V), dtype=torch.float32, device=dev) if want_residual else None
+    t = rows_of(target_row)
+    d = rows_of(draft_row) if draft_row is not None else t
+    max_k = 0 if rejected is None else rejected.shape[1]
+    if rejected is not None and (rejected.dtype != torch.int32 or not rejected.is_contiguous()):
+        raise RsdError("rejected must be contiguous int32")
+    _check(lib().rsd_resample_residual(C.byref(d), C.byref(t), B, V, _ptr(rejected), max_k, _ptr(rng_node), seed,
+                                       step, seq_base, _ptr(token), _ptr(residual), _ptr(status), _stream()))
+    return dict(token=token, residual=residual, status=status)

@@ -1,0 +1,234 @@
+// C ABI of librsd (declared in include/rsd.h): argument checks and kernel launches, nothing else.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+
+#include "../../include/rsd.h"
+#include "rsd_scan.cuh"
+#include "rsd_verify.cuh"
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+int fail(int code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int check_launch(const char* what) {
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(RSD_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+    return RSD_OK;
+}
+
+int check_rows(const char* name, const rsd_rows* r, int V, bool need_row_stride) {
+    if (!r || !r->data) return fail(RSD_ERR_INVALID_ARG, "%s: null rows", name);
+    if (r->dtype != RSD_F32 && r->dtype != RSD_BF16) return fail(RSD_ERR_UNSUPPORTED, "%s: unknown dtype %d", name, r->dtype);
+    if (need_row_stride && r->row_stride < V) return fail(RSD_ERR_INVALID_ARG, "%s: row_stride %lld < V %d", name, (long long)r->row_stride, V);
+    if (r->seq_stride < 0 || r->row_stride < 0) return fail(RSD_ERR_INVALID_ARG, "%s: negative stride", name);
+    return RSD_OK;
+}
+
+bool rows_aligned(const rsd_rows* r) {
+    const int64_t eb = r->dtype == RSD_F32 ? 4 : 2;
+    return ((uintptr_t)r->data % 16 == 0) && ((r->seq_stride * eb) % 16 == 0) && ((r->row_stride * eb) % 16 == 0);
+}
+
+int check_vocab(int V) {
+    if (V < 1 || V > RSD_MAX_VOCAB) return fail(RSD_ERR_UNSUPPORTED, "V = %d outside [1, %d]", V, (int)RSD_MAX_VOCAB);
+    return RSD_OK;
+}
+
+template <bool NEED_LSE>
+void launch_scan_lse(const rsd_rows* rows, bool aligned, int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
+    using namespace rsd;
+    if (rows->dtype == RSD_F32) {
+        if (aligned) scan_topk_kernel<float, true, NEED_LSE><<<blocks, kScanThreads, 0, s>>>(a);
+        else scan_topk_kernel<float, false, NEED_LSE><<<blocks, kScanThreads, 0, s>>>(a);
+    } else {
+        if (aligned) scan_topk_kernel<__nv_bfloat16, true, NEED_LSE><<<blocks, kScanThreads, 0, s>>>(a);
+        else scan_topk_kernel<__nv_bfloat16, false, NEED_LSE><<<blocks, kScanThreads, 0, s>>>(a);
+    }
+}
+
+void launch_scan(const rsd_rows* rows, bool need_lse, int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
+    const bool aligned = rows_aligned(rows);
+    if (need_lse) launch_scan_lse<true>(rows, aligned, blocks, a, s);
+    else launch_scan_lse<false>(rows, aligned, blocks, a, s);
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" {
+
+int rsd_version(void) { return 100; }
+int rsd_rng_layout(void) { return 1; }
+const char* rsd_last_error(void) { return g_err; }
+
+int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int32_t* k_per_row, const int32_t* rng_node,
+                          int max_k, uint64_t seed, uint32_t step, uint32_t seq_base, int32_t* out_token,
+                          float* out_perturbed, float* out_logprob, int32_t* status, rsd_stream_t stream) {
+    g_err[0] = 0;
+    if (int e = check_vocab(V)) return e;
+    if (int e = check_rows("draft", draft, V, R > 1)) return e;
+    if (B < 0 || R < 1) return fail(RSD_ERR_INVALID_ARG, "B = %d, R = %d", B, R);
+    if (R > RSD_MAX_ROWS_PER_SEQ) return fail(RSD_ERR_UNSUPPORTED, "R = %d > %d", R, (int)RSD_MAX_ROWS_PER_SEQ);
+    if (max_k < 1 || max_k > RSD_MAX_K) return fail(RSD_ERR_UNSUPPORTED, "max_k = %d outside [1, %d]", max_k, (int)RSD_MAX_K);
+    if (!k_per_row || !rng_node || !out_token || !status) return fail(RSD_ERR_INVALID_ARG, "null argument");
+    if ((int64_t)B * R > 0x7FFFFFFF) return fail(RSD_ERR_UNSUPPORTED, "B * R too large");
+    rsd::ScanArgs a;
+    memset(&a, 0, sizeof(a));
+    for (int r = 0; r < R; ++r) {
+        if (k_per_row[r] < 1 || k_per_row[r] > max_k) return fail(RSD_ERR_INVALID_ARG, "k_per_row[%d] = %d outside [1, max_k]", r, k_per_row[r]);
+        if (rng_node[r] < 0 || rng_node[r] >= (1 << 28)) return fail(RSD_ERR_INVALID_ARG, "rng_node[%d] = %d outside [0, 2^28)", r, rng_node[r]);
+        a.k_row[r] = (uint8_t)k_per_row[r];
+        a.node_row[r] = rng_node[r];
+    }
+    if (B == 0) return RSD_OK;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(status, 0, sizeof(int32_t) * (size_t)B, s) != cudaSuccess) return check_launch("memset(status)");
+    a.data = draft->data; a.seq_stride = draft->seq_stride; a.row_stride = draft->row_stride;
+    a.R = R; a.V = V; a.max_k = max_k;
+    a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
+    a.subtract_lse = 1;
+    a.out_token = out_token; a.out_perturbed = out_perturbed; a.out_value = out_logprob; a.out_lse = nullptr;
+    a.status = status;
+    const bool need_lse = !draft->is_logprob && (out_perturbed || out_logprob);
+    launch_scan(draft, need_lse, B * R, a, s);
+    return check_launch("rsd_gumbel_topk_draft");
+}
+
+size_t rsd_sbs_workspace_bytes(int B, int n_par, int W) {
+    if (B < 0 || n_par < 1 || W < 1) return 0;
+    const size_t f = (size_t)B * n_par * W;
+    return align_up(f * 4, 256) * 2 + align_up((size_t)B * n_par * 4, 256);
+}
+
+int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, int32_t first_parent_node,
+                 const float* sum_logprob_in, const float* trunc_gumbel_in, uint64_t seed, uint32_t step,
+                 uint32_t seq_base, int32_t* out_token, int32_t* out_parent, float* sum_logprob_out,
+                 float* trunc_gumbel_out, int32_t* out_count, int32_t* status, void* ws, size_t ws_bytes,
+                 rsd_stream_t stream) {
+    g_err[0] = 0;
+    if (int e = check_vocab(V)) return e;
+    if (int e = check_rows("draft_level", draft_level, V, n_par > 1)) return e;
+    if (B < 0 || n_par < 1) return fail(RSD_ERR_INVALID_ARG, "B = %d, n_par = %d", B, n_par);
+    if (n_par > RSD_MAX_ROWS_PER_SEQ) return fail(RSD_ERR_UNSUPPORTED, "n_par = %d > %d", n_par, (int)RSD_MAX_ROWS_PER_SEQ);
+    if (W < 1 || W > RSD_MAX_K) return fail(RSD_ERR_UNSUPPORTED, "W = %d outside [1, %d]", W, (int)RSD_MAX_K);
+    if (n_par * W > 1024) return fail(RSD_ERR_UNSUPPORTED, "n_par * W = %d > 1024", n_par * W);
+    if (first_parent_node < 0 || (int64_t)first_parent_node + n_par > (1 << 28)) return fail(RSD_ERR_INVALID_ARG, "first_parent_node out of range");
+    if (!out_token || !out_parent || !sum_logprob_out || !trunc_gumbel_out || !out_count || !status) return fail(RSD_ERR_INVALID_ARG, "null output");
+    if ((int64_t)B * n_par > 0x7FFFFFFF) return fail(RSD_ERR_UNSUPPORTED, "B * n_par too large");
+    if (B == 0) return RSD_OK;
+    const size_t need = rsd_sbs_workspace_bytes(B, n_par, W);
+    if (!ws || ws_bytes < need) return fail(RSD_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
+    if ((uintptr_t)ws % 256 != 0) return fail(RSD_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(status, 0, sizeof(int32_t) * (size_t)B, s) != cudaSuccess) return check_launch("memset(status)");
+
+    const size_t f = (size_t)B * n_par * W;
+    char* w = (char*)ws;
+    int32_t* fin_token = (int32_t*)w;
+    float* fin_value = (float*)(w + align_up(f * 4, 256));
+    float* fin_lse = (float*)(w + 2 * align_up(f * 4, 256));
+
+    rsd::ScanArgs a;
+    memset(&a, 0, sizeof(a));
+    for (int r = 0; r < n_par; ++r) { a.k_row[r] = (uint8_t)W; a.node_row[r] = first_parent_node + r; }
+    a.data = draft_level->data; a.seq_stride = draft_level->seq_stride; a.row_stride = draft_level->row_stride;
+    a.R = n_par; a.V = V; a.max_k = W;
+    a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
+    a.subtract_lse = 0;
+    a.out_token = fin_token; a.out_perturbed = nullptr; a.out_value = fin_value; a.out_lse = fin_lse;
+    a.status = status;
+    launch_scan(draft_level, !draft_level->is_logprob, B * n_par, a, s);
+    if (int e = check_launch("rsd_sbs_step(scan)")) return e;
+
+    rsd::SbsEpilogueArgs e;
+    e.n_par = n_par; e.W = W; e.is_logprob = draft_level->is_logprob; e.first_parent_node = first_parent_node;
+    e.seed_lo = (uint32_t)seed; e.seed_hi = (uint32_t)(seed >> 32); e.step = step; e.seq_base = seq_base;
+    e.fin_token = fin_token; e.fin_value = fin_value; e.fin_lse = fin_lse;
+    e.sum_in = sum_logprob_in; e.gamma_in = trunc_gumbel_in;
+    e.out_token = out_token; e.out_parent = out_parent; e.sum_out = sum_logprob_out; e.gamma_out = trunc_gumbel_out;
+    e.out_count = out_count; e.status = status;
+    const size_t smem = (size_t)n_par * W * (8 + 8 + 4);
+    rsd::sbs_epilogue_kernel<<<B, rsd::kEpilogueThreads, smem, s>>>(e);
+    return check_launch("rsd_sbs_step(epilogue)");
+}
+
+int rsd_verify_tree(const rsd_rows* draft, const rsd_rows* target, const rsd_tree* tree, int B, int V, uint64_t seed,
+                    uint32_t step, uint32_t seq_base, int32_t* accepted_len, int32_t* accepted_node,
+                    int32_t* accepted_token, int32_t* last_token, int32_t* stop_reason, float* dbg_theta,
+                    int32_t* status, rsd_stream_t stream) {
+    g_err[0] = 0;
+    if (int e = check_vocab(V)) return e;
+    if (int e = check_rows("draft", draft, V, true)) return e;
+    if (int e = check_rows("target", target, V, true)) return e;
+    if (draft->dtype != target->dtype) return fail(RSD_ERR_UNSUPPORTED, "draft and target rows must have the same dtype");
+    if (!tree || !tree->parent || !tree->token) return fail(RSD_ERR_INVALID_ARG, "null tree");
+    if (tree->num_levels < 0 || tree->num_nodes < 1 || tree->num_nodes > RSD_MAX_TREE_NODES)
+        return fail(RSD_ERR_UNSUPPORTED, "num_levels = %d, num_nodes = %d", tree->num_levels, tree->num_nodes);
+    if (B < 0) return fail(RSD_ERR_INVALID_ARG, "B = %d", B);
+    if (!accepted_len || !accepted_node || !accepted_token || !last_token || !stop_reason || !status) return fail(RSD_ERR_INVALID_ARG, "null output");
+    if (B == 0) return RSD_OK;
+    rsd::VerifyArgs a;
+    a.draft = {draft->data, draft->seq_stride, draft->row_stride};
+    a.target = {target->data, target->seq_stride, target->row_stride};
+    a.V = V; a.L = tree->num_levels; a.num_nodes = tree->num_nodes; a.shared_topology = tree->topology_is_shared;
+    a.parent = tree->parent; a.token = tree->token;
+    a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
+    a.accepted_len = accepted_len; a.accepted_node = accepted_node; a.accepted_token = accepted_token;
+    a.last_token = last_token; a.stop_reason = stop_reason; a.dbg_theta = dbg_theta; a.status = status;
+    cudaStream_t s = (cudaStream_t)stream;
+    const bool aligned = rows_aligned(draft) && rows_aligned(target);
+    using namespace rsd;
+    if (draft->dtype == RSD_F32) {
+        if (aligned) verify_tree_kernel<float, true><<<B, kVerifyThreads, 0, s>>>(a);
+        else verify_tree_kernel<float, false><<<B, kVerifyThreads, 0, s>>>(a);
+    } else {
+        if (aligned) verify_tree_kernel<__nv_bfloat16, true><<<B, kVerifyThreads, 0, s>>>(a);
+        else verify_tree_kernel<__nv_bfloat16, false><<<B, kVerifyThreads, 0, s>>>(a);
+    }
+    return check_launch("rsd_verify_tree");
+}
+
+int rsd_resample_residual(const rsd_rows* draft_row, const rsd_rows* target_row, int B, int V, const int32_t* rejected,
+                          int max_k, const int32_t* rng_node, uint64_t seed, uint32_t step, uint32_t seq_base,
+                          int32_t* out_token, float* out_residual, int32_t* status, rsd_stream_t stream) {
+    g_err[0] = 0;
+    if (int e = check_vocab(V)) return e;
+    if (int e = check_rows("target_row", target_row, V, false)) return e;
+    if (rejected) {
+        if (int e = check_rows("draft_row", draft_row, V, false)) return e;
+        if (draft_row->dtype != target_row->dtype) return fail(RSD_ERR_UNSUPPORTED, "draft and target rows must have the same dtype");
+        if (max_k < 1 || max_k > RSD_MAX_K) return fail(RSD_ERR_UNSUPPORTED, "max_k = %d outside [1, %d]", max_k, (int)RSD_MAX_K);
+    }
+    if (B < 0) return fail(RSD_ERR_INVALID_ARG, "B = %d", B);
+    if (!rng_node || !out_token || !status) return fail(RSD_ERR_INVALID_ARG, "null argument");
+    if (B == 0) return RSD_OK;
+    rsd::ResampleArgs a;
+    a.target = {target_row->data, target_row->seq_stride, 0};
+    a.draft = rejected ? rsd::RowsDev{draft_row->data, draft_row->seq_stride, 0} : a.target;
+    a.V = V; a.max_k = rejected ? max_k : 0; a.rejected = rejected; a.rng_node = rng_node;
+    a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
+    a.out_token = out_token; a.out_residual = out_residual; a.status = status;
+    cudaStream_t s = (cudaStream_t)stream;
+    const bool aligned = rows_aligned(target_row) && (!rejected || rows_aligned(draft_row));
+    using namespace rsd;
+    if (target_row->dtype == RSD_F32) {
+        if (aligned) resample_residual_kernel<float, true><<<B, kVerifyThreads, 0, s>>>(a);
+        else resample_residual_kernel<float, false><<<B, kVerifyThreads, 0, s>>>(a);
+    } else {
+        if (aligned) resample_residual_kernel<__nv_bfloat16, true><<<B, kVerifyThreads, 0, s>>>(a);
+        else resample_residual_kernel<__nv_bfloat16, false><<<B, kVerifyThreads, 0, s>>>(a);
+    }
+    return check_launch("rsd_resample_residual");
+}
+
+}  // extern "C"

@@ -1,0 +1,272 @@
+"""GPU-vs-oracle parity through the C ABI (needs a CUDA device)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+from tests.parity import Tally, close, compare_sbs_level, compare_topk, compare_verify
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rsd():
+    import paper_2402_14160_b200 as m
+    m.lib()
+    return m
+
+
+def _np(d):
+    return {k: (v.cpu().numpy() if isinstance(v, torch.Tensor) else v) for k, v in d.items()}
+
+
+def _rows(shape, dtype, sigma, seed, device="cuda"):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    t = torch.randn(shape, generator=g, dtype=torch.float32) * sigma
+    return t.to(torch.bfloat16 if dtype == "bf16" else torch.float32).to(device)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Gumbel-Top-k drafting
+# ---------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("V", [1, 5, 16, 17, 70, 1000, 4099, 32000, 50272])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_gumbel_topk_matches_oracle(rsd, V, dtype):
+    B, R = 3, 4
+    rows = _rows((B, R, V), dtype, 2.0, 100 + V)
+    k = [min(V, kk) for kk in (1, 2, 4, 32)]
+    nodes = [0, 3, 7, 1000]
+    g = _np(rsd.rsd_gumbel_topk_draft(rows, k, nodes, seed=11, step=5, seq_base=9, max_k=max(k), want_values=True))
+    o = oracle.gumbel_topk(workloads.as_oracle_rows(rows), k, nodes, 11, 5, seq_base=9, max_k=max(k))
+    t = Tally()
+    compare_topk(t, g["token"], o, k, g["perturbed"], g["logprob"])
+    t.check()
+    assert np.array_equal(g["status"], o["status"])
+    # production form: no values asked, no normaliser computed, same picks
+    g2 = _np(rsd.rsd_gumbel_topk_draft(rows, k, nodes, seed=11, step=5, seq_base=9, max_k=max(k)))
+    assert np.array_equal(g2["token"], g["token"])
+
+
+def test_gumbel_topk_unaligned_rows_and_logprob_input(rsd):
+    B, R, V = 2, 3, 1003
+    base = _rows((B, R, V + 5), "f32", 2.0, 7)
+    rows = torch.log_softmax(base, -1)[:, :, 3:3 + V]            # odd offset, odd stride: scalar path
+    k, nodes = [3, 3, 3], [1, 2, 3]
+    g = _np(rsd.rsd_gumbel_topk_draft(rows, k, nodes, seed=1, step=0, is_logprob=True, want_values=True))
+    o = oracle.gumbel_topk(workloads.as_oracle_rows(rows.contiguous()), k, nodes, 1, 0, is_logprob=True)
+    t = Tally()
+    compare_topk(t, g["token"], o, k, g["perturbed"], g["logprob"])
+    t.check()
+    bf = _rows((B, R, V + 8), "bf16", 2.0, 8)[:, :, 1:1 + V]
+    g = _np(rsd.rsd_gumbel_topk_draft(bf, k, nodes, seed=1, step=0))
+    o = oracle.gumbel_topk(workloads.as_oracle_rows(bf.contiguous()), k, nodes, 1, 0)
+    t = Tally()
+    compare_topk(t, g["token"], o, k)
+    t.check()
+
+
+def test_gumbel_topk_degenerate_rows(rsd):
+    V = 300
+    rows = torch.full((2, 2, V), float("-inf"), device="cuda")
+    rows[0, 0, [5, 77]] = torch.tensor([0.5, 1.0], device="cuda")
+    rows[0, 1, :] = 0.0                                           # all equal: noise alone decides
+    rows[1, 0, 10:20] = 1.0
+    rows[1, 0, 15] = float("nan")
+    rows[1, 1, :] = torch.arange(V, device="cuda") * 0.1          # increasing: every element beats the running bound
+    k, nodes = [4, 4], [0, 1]
+    g = _np(rsd.rsd_gumbel_topk_draft(rows, k, nodes, seed=3, step=0, want_values=True))
+    o = oracle.gumbel_topk(workloads.as_oracle_rows(rows), k, nodes, 3, 0)
+    t = Tally()
+    compare_topk(t, g["token"], o, k, g["perturbed"], g["logprob"])
+    t.check()
+    assert np.array_equal(g["status"], o["status"])
+    assert g["status"][0] & rsd.ST_FEWER_THAN_K and g["status"][1] & rsd.ST_NAN_INPUT
+    assert g["token"][0, 0, 2] == -1 and 15 not in g["token"][1, 0]
+
+
+def test_gumbel_topk_is_deterministic_and_shardable(rsd):
+    rows = _rows((8, 3, 5000), "bf16", 2.0, 21)
+    k, nodes = [4, 2, 8], [0, 1, 2]
+    a = _np(rsd.rsd_gumbel_topk_draft(rows, k, nodes, seed=5, step=1, want_values=True))
+    b = _np(rsd.rsd_gumbel_topk_draft(rows, k, nodes, seed=5, step=1, want_values=True))
+    assert all(np.array_equal(a[x], b[x]) for x in ("token", "perturbed", "logprob"))
+    lo = _np(rsd.rsd_gumbel_topk_draft(rows[:3], k, nodes, seed=5, step=1, seq_base=0))
+    hi = _np(rsd.rsd_gumbel_topk_draft(rows[3:], k, nodes, seed=5, step=1, seq_base=3))
+    assert np.array_equal(np.concatenate([lo["token"], hi["token"]]), a["token"])
+
+
+def test_argument_errors_are_reported_not_trapped(rsd):
+    rows = _rows((1, 1, 64), "f32", 1.0, 1)
+    with pytest.raises(rsd.RsdError, match="max_k"):
+        rsd.rsd_gumbel_topk_draft(rows, [40], [0], seed=0, step=0)
+    with pytest.raises(rsd.RsdError, match="workspace"):
+        rsd.rsd_sbs_step(rows, 2, 0, None, None, 0, 0, workspace=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(rsd.RsdError):
+        rsd.rsd_gumbel_topk_draft(rows.double(), [1], [0], seed=0, step=0)
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Stochastic Beam Search
+# ---------------------------------------------------------------------------------------------------------
+def _sbs_chain(rsd, draft, W, L, seed, step, is_logprob, seq_base=0):
+    """Run L levels on both sides, each from its own previous level; returns (tally, gpu levels, oracle levels)."""
+    B = draft.shape[0]
+    host = workloads.as_oracle_rows(draft)
+    t = Tally()
+    skip = set()
+    g_prev = o_prev = None
+    g_levels, o_levels = [], []
+    for l in range(L):
+        first = 0 if l == 0 else 1 + (l - 1) * W
+        n_par = 1 if l == 0 else W
+        g = rsd.rsd_sbs_step(draft[:, first:first + n_par], W, first,
+                             None if l == 0 else g_prev["sum_logprob"], None if l == 0 else g_prev["trunc_gumbel"],
+                             seed, step, is_logprob=is_logprob, seq_base=seq_base)
+        o = oracle.sbs_step(host[:, first:first + n_par], W, first,
+                            None if l == 0 else o_prev["sum_logprob"], None if l == 0 else o_prev["trunc_gumbel"],
+                            seed, step, is_logprob=is_logprob, seq_base=seq_base)
+        skip |= compare_sbs_level(t, _np(g), o, W, skip)
+        g_prev, o_prev = g, o
+        g_levels.append(_np(g))
+        o_levels.append(o)
+    return t, g_levels, o_levels, skip
+
+
+def _sbs_tree(levels, W):
+    """parent [B, N+1] (flat) and token [B, N+1] from per-level (token, parent) outputs."""
+    B = levels[0]["token"].shape[0]
+    L = len(levels)
+    parent = np.full((B, 1 + L * W), -1, np.int32)
+    token = np.full((B, 1 + L * W), -1, np.int32)
+    for l, lv in enumerate(levels):
+        off_prev = 0 if l == 0 else 1 + (l - 1) * W
+        sl = slice(1 + l * W, 1 + (l + 1) * W)
+        token[:, sl] = lv["token"]
+        parent[:, sl] = np.where(lv["parent"] >= 0, off_prev + lv["parent"], -1)
+    return parent, token
+
+
+@pytest.mark.parametrize("dtype,V,W,L,is_logprob", [("f32", 1000, 3, 3, False), ("bf16", 4099, 8, 4, False),
+                                                    ("f32", 515, 4, 3, True), ("bf16", 32000, 6, 3, False)])
+def test_sbs_levels_match_oracle(rsd, dtype, V, W, L, is_logprob):
+    B = 6
+    P = 1 + (L - 1) * W
+    draft = _rows((B, P, V), dtype, 2.0, 300 + V)
+    if is_logprob:
+        draft = torch.log_softmax(draft.float(), -1).to(draft.dtype)
+    t, g_levels, o_levels, _ = _sbs_chain(rsd, draft, W, L, seed=17, step=2, is_logprob=is_logprob, seq_base=4)
+    t.check()
+    assert all(np.all(g["count"] == W) for g in g_levels)
+
+
+def test_sbs_drops_minus_infinity_candidates(rsd):
+    rows = torch.full((1, 2, 64), float("-inf"), device="cuda")
+    rows[0, 0, [2, 9]] = torch.tensor([0.0, 1.0], device="cuda")
+    rows[0, 1, 5] = 0.3
+    sig = torch.zeros((1, 2), device="cuda")
+    gam = torch.tensor([[0.0, -0.5]], device="cuda")
+    g = _np(rsd.rsd_sbs_step(rows, 4, 1, sig, gam, 3, 0))
+    o = oracle.sbs_step(workloads.as_oracle_rows(rows), 4, 1, sig.cpu().numpy(), gam.cpu().numpy(), 3, 0)
+    assert np.array_equal(g["token"], o["token"]) and np.array_equal(g["parent"], o["parent"])
+    assert g["count"][0] == 3 and g["status"][0] & rsd.ST_FEWER_THAN_K
+    assert close(g["trunc_gumbel"][0, :3], o["trunc_gumbel"][0, :3]).all()
+
+
+# ---------------------------------------------------------------------------------------------------------
+# verification
+# ---------------------------------------------------------------------------------------------------------
+def _verify_both(rsd, draft, target, parent, token, L, seed, step, seq_base=0):
+    par_t = torch.from_numpy(parent).cuda()
+    tok_t = torch.from_numpy(token).cuda()
+    g = _np(rsd.rsd_verify_tree(draft, target, par_t, tok_t, L, seed, step, seq_base=seq_base, want_theta=True))
+    o = oracle.verify_tree(workloads.as_oracle_rows(draft), workloads.as_oracle_rows(target), parent, token, L,
+                           seed, step, seq_base=seq_base)
+    return g, o
+
+
+@pytest.mark.parametrize("dtype,V,branching,noise", [("f32", 64, (3, 2, 2), 1.0), ("bf16", 515, (4, 2, 1), 1.5),
+                                                      ("f32", 4099, (3, 3), 2.0), ("bf16", 32000, (3, 2, 2, 1), 1.0),
+                                                      ("f32", 32000, (2, 2, 2), 0.5), ("bf16", 50272, (4, 2), 1.0)])
+def test_verify_tree_matches_oracle_constant_branching(rsd, dtype, V, branching, noise):
+    B = 48 if V <= 5000 else 12
+    L = len(branching)
+    parent = workloads.rsdc_parent_array(branching)
+    n_nodes = len(parent)
+    k, nodes = workloads.rsdc_rows(branching)
+    P = len(k)
+    base = _rows((B, n_nodes, V), "f32", 2.0, 500 + V)
+    draft = base[:, :P].to(torch.bfloat16 if dtype == "bf16" else torch.float32).contiguous()
+    target = (base + _rows((B, n_nodes, V), "f32", noise, 501 + V)).to(draft.dtype).contiguous()
+    o_draft = oracle.gumbel_topk(workloads.as_oracle_rows(draft), k, nodes, 23, 1, seq_base=2)
+    token = workloads.rsdc_tokens_from_rows(branching, o_draft["token"])
+    g, o = _verify_both(rsd, draft, target, parent, token, L, 23, 1, seq_base=2)
+    t = Tally()
+    compare_verify(t, g, o, parent)
+    t.check()
+    assert t.final_mismatch <= max(1, 0.02 * B)
+    assert np.array_equal(g["status"], o["status"])
+    assert len(set(o["accepted_len"].tolist())) > 1 or B < 20     # the cases exercise several path lengths
+
+
+def test_verify_tree_special_trees(rsd):
+    rng = np.random.default_rng(3)
+    V = 200
+    parent = np.array([[-1, 0, 0, 1, 1, 2]] * 4, np.int32)       # per-sequence topology
+    token = np.array([[-1, 4, 7, 1, -1, 3]] * 4, np.int32)
+    token[1, 1:] = -1                                             # sequence 1: the root has no children
+    token[2, 2] = 250                                             # sequence 2: a token outside the vocabulary is absent
+    draft = torch.from_numpy(rng.normal(0, 1, (4, 3, V)).astype(np.float32)).cuda()
+    target = torch.from_numpy(rng.normal(0, 1, (4, 6, V)).astype(np.float32)).cuda()
+    target[3] = torch.cat([draft[3], draft[3]], 0)                # sequence 3: target == draft on the visited rows
+    tok_o = token.copy()
+    tok_o[2, 2] = -1
+    par_t, tok_t = torch.from_numpy(parent).cuda(), torch.from_numpy(token).cuda()
+    g = _np(rsd.rsd_verify_tree(draft, target, par_t, tok_t, 2, 9, 0, want_theta=True))
+    o = oracle.verify_tree(workloads.as_oracle_rows(draft), workloads.as_oracle_rows(target), parent, tok_o, 2, 9, 0)
+    t = Tally()
+    compare_verify(t, g, o, parent)
+    t.check()
+    assert g["stop_reason"][1] == rsd.STOP_NO_CHILDREN and g["accepted_len"][1] == 0
+    assert g["accepted_len"][3] == 2 and g["stop_reason"][3] == rsd.STOP_LEAF
+    assert np.array_equal(g["last_token"], o["last_token"])
+
+
+def test_verify_tree_on_stochastic_beam_trees(rsd):
+    w = workloads.scaled(workloads.WORKLOADS[3], batch=8, vocab=4000)
+    draft, target = workloads.make_logits(w, step=0, device="cuda")
+    W, L = w.beam_width, w.depth
+    _, g_levels, o_levels, skip = _sbs_chain(rsd, draft, W, L, seed=5, step=0, is_logprob=True)
+    parent, token = _sbs_tree(o_levels, W)
+    g, o = _verify_both(rsd, draft, target, parent, token, L, 5, 0)
+    t = Tally()
+    compare_verify(t, g, o, parent)
+    t.check()
+
+
+# ---------------------------------------------------------------------------------------------------------
+# residual draw
+# ---------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,V", [("f32", 70), ("bf16", 4099), ("f32", 32000)])
+def test_resample_residual_matches_oracle(rsd, dtype, V):
+    B = 16
+    d = _rows((B, V), dtype, 2.0, 900 + V)
+    tg = (d.float() + _rows((B, V), "f32", 1.0, 901 + V)).to(d.dtype)
+    nodes = torch.arange(B, dtype=torch.int32, device="cuda") + 3
+    rng = np.random.default_rng(V)
+    rej = np.full((B, 4), -1, np.int32)
+    for b in range(B):
+        n = b % 4
+        rej[b, :n] = rng.choice(V, n, replace=False)
+    rej[:, 0][rej[:, 0] < 0] = -1
+    g = _np(rsd.rsd_resample_residual(d, tg, torch.from_numpy(rej).cuda(), nodes, 13, 2, seq_base=1, want_residual=True))
+    o = oracle.resample_residual(workloads.as_oracle_rows(d), workloads.as_oracle_rows(tg), rej, nodes.cpu().numpy(),
+                                 13, 2, seq_base=1)
+    peak = o["residual"].max(axis=1, keepdims=True)
+    assert np.all(np.abs(g["residual"] - o["residual"]) <= 1e-5 * peak)
+    mism = g["token"] != o["token"]
+    assert np.all(o["margin"][mism] <= 1e-5) and mism.sum() <= 1
+    plain = _np(rsd.rsd_resample_residual(None, tg, None, nodes, 13, 2, seq_base=1, want_residual=True))
+    o2 = oracle.resample_residual(None, workloads.as_oracle_rows(tg), None, nodes.cpu().numpy(), 13, 2, seq_base=1)
+    assert np.all(np.abs(plain["residual"] - o2["residual"]) <= 1e-5 * o2["residual"].max(axis=1, keepdims=True))
+    assert (plain["token"] != o2["token"]).sum() <= 1
