@@ -92,6 +92,13 @@ int rsd_rng_layout(void);
 const char* rsd_last_error(void);
 
 /*
+ * Timing aid (the paper has no counterpart).  The next rsd_gumbel_topk_draft or rsd_sbs_step call made by this host
+ * thread records the CUDA event `before` right before and `after` right after its row-scan kernel, on that call's
+ * stream; the request is then cleared.  Either may be NULL.  Host handles (cudaEvent_t) owned by the caller.
+ */
+int rsd_profile_next_scan(void* before, void* after);
+
+/*
  * Gumbel-Top-k drafting for RSD with constant branching factors (Section 3.2.1, Eqs. 5-8; Algorithm 4).
  * For each of the B*R rows: phi = log-softmax(row) (Eq. 5), phi~ = phi + G (Eq. 6), and the k_per_row[r] tokens
  * with the largest phi~ in decreasing order (Eq. 7); equal values go to the smaller token.  The noise of row r is
@@ -102,12 +109,15 @@ const char* rsd_last_error(void);
  *   rng_node     host [R], flat node id of each row (< 2^28)
  *   out_token    [B][R][max_k] int32; entries beyond k_per_row[r], or beyond the finite entries of the row, are -1
  *   out_perturbed, out_logprob  optional (NULL to skip) [B][R][max_k] fp32: phi~ and phi of each pick
+ *   child_base   optional host [R], node_token optional [B][node_stride] int32: when both are given, pick j of row r
+ *                is also stored as the token of tree node child_base[r] + j (Eq. 8's (token, parent) pairs in the
+ *                flat layout rsd_verify_tree reads); other entries of node_token are left alone
  *   status       [B]
  */
 int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int32_t* k_per_row,
                           const int32_t* rng_node, int max_k, uint64_t seed, uint32_t step, uint32_t seq_base,
-                          int32_t* out_token, float* out_perturbed, float* out_logprob, int32_t* status,
-                          rsd_stream_t stream);
+                          int32_t* out_token, float* out_perturbed, float* out_logprob, const int32_t* child_base,
+                          int32_t* node_token, int node_stride, int32_t* status, rsd_stream_t stream);
 
 /*
  * One level of Stochastic Beam Search for RSD-S (Section 3.2.1, Eqs. 10-12; Algorithm 9).
@@ -118,7 +128,10 @@ int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int3
  * and the W pairs (x, k) with the largest psi are returned in decreasing order (Eq. 12); equal values go to the
  * smaller parent, then the smaller token.  Entries whose log-probability is -inf are dropped.
  *   draft_level       rows [B][n_par][V], n_par <= RSD_MAX_ROWS_PER_SEQ, W <= RSD_MAX_K
- *   out_token, out_parent   [B][W] int32 (parent = slot index within the level); -1 beyond out_count[b]
+ *   out_token, out_parent   int32, pick i of sequence b at [b * out_stride + i], out_stride >= W; the parent is
+ *                     parent_base + slot index within the level, so with out_token/out_parent pointing at a level's
+ *                     first node inside [B][N+1] tree arrays and parent_base = first_parent_node the tree arrays
+ *                     of rsd_verify_tree are filled in place; entries beyond out_count[b] are -1
  *   sum_logprob_out, trunc_gumbel_out  [B][W] fp32: phi and psi of each pick, the next level's inputs
  *   out_count         [B]
  *   ws                scratch of at least rsd_sbs_workspace_bytes(B, n_par, W) bytes, 256-byte aligned; contents
@@ -127,9 +140,9 @@ int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int3
 size_t rsd_sbs_workspace_bytes(int B, int n_par, int W);
 int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, int32_t first_parent_node,
                  const float* sum_logprob_in, const float* trunc_gumbel_in, uint64_t seed, uint32_t step,
-                 uint32_t seq_base, int32_t* out_token, int32_t* out_parent, float* sum_logprob_out,
-                 float* trunc_gumbel_out, int32_t* out_count, int32_t* status, void* ws, size_t ws_bytes,
-                 rsd_stream_t stream);
+                 uint32_t seq_base, int32_t* out_token, int32_t* out_parent, int64_t out_stride, int32_t parent_base,
+                 float* sum_logprob_out, float* trunc_gumbel_out, int32_t* out_count, int32_t* status, void* ws,
+                 size_t ws_bytes, rsd_stream_t stream);
 
 /*
  * Draft-tree verification by recursive rejection sampling (Section 3.1, Eqs. 1-4, Algorithm 1; Section 3.2.2,

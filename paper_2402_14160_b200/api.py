@@ -20,7 +20,7 @@ ST_NAN_INPUT, ST_FEWER_THAN_K, ST_ZERO_RESIDUAL, ST_ZERO_DRAFT_PROB, ST_DRAFT_EX
 STOP_ALL_REJECTED, STOP_NO_CHILDREN, STOP_LEAF = 0, 1, 2
 MAX_K = 32
 
-EXPORTS = ["rsd_version", "rsd_rng_layout", "rsd_last_error", "rsd_gumbel_topk_draft", "rsd_sbs_workspace_bytes",
+EXPORTS = ["rsd_version", "rsd_rng_layout", "rsd_last_error", "rsd_profile_next_scan", "rsd_gumbel_topk_draft", "rsd_sbs_workspace_bytes",
            "rsd_sbs_step", "rsd_verify_tree", "rsd_resample_residual"]
 
 
@@ -50,15 +50,16 @@ def lib():
                            "(there is no fallback path)" % LIB_PATH)
         l = C.CDLL(LIB_PATH)
         l.rsd_last_error.restype = C.c_char_p
+        l.rsd_profile_next_scan.argtypes = [C.c_void_p, C.c_void_p]
         l.rsd_sbs_workspace_bytes.restype = C.c_size_t
         l.rsd_sbs_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         l.rsd_gumbel_topk_draft.argtypes = [C.POINTER(RsdRows), C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                             C.c_int, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
-                                            C.c_void_p, C.c_void_p, C.c_void_p]
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         l.rsd_sbs_step.argtypes = [C.POINTER(RsdRows), C.c_int, C.c_int, C.c_int, C.c_int, C.c_int32, C.c_void_p,
                                    C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
-                                   C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
-                                   C.c_void_p]
+                                   C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                   C.c_void_p, C.c_size_t, C.c_void_p]
         l.rsd_verify_tree.argtypes = [C.POINTER(RsdRows), C.POINTER(RsdRows), C.POINTER(RsdTree), C.c_int, C.c_int,
                                       C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -108,20 +109,35 @@ def _host_i32(values: Sequence[int]):
 
 def rsd_gumbel_topk_draft(draft: torch.Tensor, k_per_row: Sequence[int], rng_node: Sequence[int], seed: int,
                           step: int, *, is_logprob: bool = False, seq_base: int = 0, max_k: Optional[int] = None,
-                          want_values: bool = False):
-    """draft [B, R, V] -> dict(token [B, R, max_k], status [B], and perturbed/logprob when want_values)."""
+                          want_values: bool = False, child_base: Optional[Sequence[int]] = None,
+                          node_token: Optional[torch.Tensor] = None, out: Optional[dict] = None):
+    """draft [B, R, V] -> dict(token [B, R, max_k], status [B], and perturbed/logprob when want_values).
+
+    With child_base [R] and node_token [B, N+1] (int32) the picks also land in the tree's per-node token array.
+    """
     B, R, V = draft.shape
     max_k = int(max_k or max(k_per_row))
     dev = draft.device
-    token = torch.empty((B, R, max_k), dtype=torch.int32, device=dev)
-    status = torch.empty((B,), dtype=torch.int32, device=dev)
-    pert = torch.empty((B, R, max_k), dtype=torch.float32, device=dev) if want_values else None
-    logp = torch.empty((B, R, max_k), dtype=torch.float32, device=dev) if want_values else None
+    if out is None:
+        out = dict(token=torch.empty((B, R, max_k), dtype=torch.int32, device=dev),
+                   status=torch.empty((B,), dtype=torch.int32, device=dev),
+                   perturbed=torch.empty((B, R, max_k), dtype=torch.float32, device=dev) if want_values else None,
+                   logprob=torch.empty((B, R, max_k), dtype=torch.float32, device=dev) if want_values else None)
     rows = rows_of(draft, is_logprob)
+    if node_token is not None and (node_token.dtype != torch.int32 or not node_token.is_contiguous()):
+        raise RsdError("node_token must be contiguous int32")
     _check(lib().rsd_gumbel_topk_draft(C.byref(rows), B, R, V, _host_i32(k_per_row), _host_i32(rng_node), max_k,
-                                       seed, step, seq_base, _ptr(token), _ptr(pert), _ptr(logp), _ptr(status),
-                                       _stream()))
-    return dict(token=token, perturbed=pert, logprob=logp, status=status)
+                                       seed, step, seq_base, _ptr(out["token"]), _ptr(out.get("perturbed")),
+                                       _ptr(out.get("logprob")), None if child_base is None else _host_i32(child_base),
+                                       _ptr(node_token), 0 if node_token is None else node_token.shape[1],
+                                       _ptr(out["status"]), _stream()))
+    return out
+
+
+def rsd_profile_next_scan(before: Optional[torch.cuda.Event], after: Optional[torch.cuda.Event]):
+    """Have the next drafting call record these (timing-enabled, already created) events around its scan kernel."""
+    _check(lib().rsd_profile_next_scan(None if before is None else before.cuda_event,
+                                       None if after is None else after.cuda_event))
 
 
 def rsd_sbs_workspace_bytes(B: int, n_par: int, W: int) -> int:
@@ -130,8 +146,13 @@ def rsd_sbs_workspace_bytes(B: int, n_par: int, W: int) -> int:
 
 def rsd_sbs_step(draft_level: torch.Tensor, W: int, first_parent_node: int, sum_logprob_in: Optional[torch.Tensor],
                  trunc_gumbel_in: Optional[torch.Tensor], seed: int, step: int, *, is_logprob: bool = False,
-                 seq_base: int = 0, workspace: Optional[torch.Tensor] = None, out: Optional[dict] = None):
-    """draft_level [B, n_par, V] -> dict(token, parent, sum_logprob, trunc_gumbel [B, W], count [B], status [B])."""
+                 seq_base: int = 0, workspace: Optional[torch.Tensor] = None, out: Optional[dict] = None,
+                 parent_base: int = 0):
+    """draft_level [B, n_par, V] -> dict(token, parent, sum_logprob, trunc_gumbel [B, W], count [B], status [B]).
+
+    out["token"] / out["parent"] may be [B, W] views into wider [B, N+1] tree arrays (row stride kept); parent_base
+    is added to every parent index.
+    """
     B, n_par, V = draft_level.shape
     dev = draft_level.device
     need = rsd_sbs_workspace_bytes(B, n_par, W)
@@ -145,9 +166,11 @@ def rsd_sbs_step(draft_level: torch.Tensor, W: int, first_parent_node: int, sum_
                    count=torch.empty((B,), dtype=torch.int32, device=dev),
                    status=torch.empty((B,), dtype=torch.int32, device=dev))
     rows = rows_of(draft_level, is_logprob)
+    if out["token"].stride(0) != out["parent"].stride(0) or out["token"].stride(1) != 1 or out["parent"].stride(1) != 1:
+        raise RsdError("out token/parent must share a row stride and be dense along the picks")
     _check(lib().rsd_sbs_step(C.byref(rows), B, n_par, V, W, first_parent_node, _ptr(sum_logprob_in),
                               _ptr(trunc_gumbel_in), seed, step, seq_base, _ptr(out["token"]), _ptr(out["parent"]),
-                              _ptr(out["sum_logprob"]), _ptr(out["trunc_gumbel"]), _ptr(out["count"]),
+                              out["token"].stride(0), parent_base, _ptr(out["sum_logprob"]), _ptr(out["trunc_gumbel"]), _ptr(out["count"]),
                               _ptr(out["status"]), _ptr(workspace), workspace.numel(), _stream()))
     return out
 

@@ -10,6 +10,7 @@
 namespace {
 
 thread_local char g_err[512] = "";
+thread_local cudaEvent_t g_scan_before = nullptr, g_scan_after = nullptr;  // one-shot, see rsd_profile_next_scan
 
 int fail(int code, const char* fmt, ...) {
     va_list ap;
@@ -57,8 +58,11 @@ void launch_scan_lse(const rsd_rows* rows, bool aligned, int blocks, const rsd::
 
 void launch_scan(const rsd_rows* rows, bool need_lse, int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
     const bool aligned = rows_aligned(rows);
+    if (g_scan_before) cudaEventRecord(g_scan_before, s);
     if (need_lse) launch_scan_lse<true>(rows, aligned, blocks, a, s);
     else launch_scan_lse<false>(rows, aligned, blocks, a, s);
+    if (g_scan_after) cudaEventRecord(g_scan_after, s);
+    g_scan_before = g_scan_after = nullptr;
 }
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -71,9 +75,16 @@ int rsd_version(void) { return 100; }
 int rsd_rng_layout(void) { return 1; }
 const char* rsd_last_error(void) { return g_err; }
 
+int rsd_profile_next_scan(void* before, void* after) {
+    g_scan_before = (cudaEvent_t)before;
+    g_scan_after = (cudaEvent_t)after;
+    return RSD_OK;
+}
+
 int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int32_t* k_per_row, const int32_t* rng_node,
                           int max_k, uint64_t seed, uint32_t step, uint32_t seq_base, int32_t* out_token,
-                          float* out_perturbed, float* out_logprob, int32_t* status, rsd_stream_t stream) {
+                          float* out_perturbed, float* out_logprob, const int32_t* child_base, int32_t* node_token,
+                          int node_stride, int32_t* status, rsd_stream_t stream) {
     g_err[0] = 0;
     if (int e = check_vocab(V)) return e;
     if (int e = check_rows("draft", draft, V, R > 1)) return e;
@@ -89,6 +100,12 @@ int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int3
         if (rng_node[r] < 0 || rng_node[r] >= (1 << 28)) return fail(RSD_ERR_INVALID_ARG, "rng_node[%d] = %d outside [0, 2^28)", r, rng_node[r]);
         a.k_row[r] = (uint8_t)k_per_row[r];
         a.node_row[r] = rng_node[r];
+        if (node_token) {
+            if (!child_base) return fail(RSD_ERR_INVALID_ARG, "node_token needs child_base");
+            if (child_base[r] < 0 || child_base[r] + k_per_row[r] > node_stride)
+                return fail(RSD_ERR_INVALID_ARG, "child_base[%d] = %d: children fall outside [0, node_stride = %d)", r, child_base[r], node_stride);
+            a.child_base[r] = child_base[r];
+        }
     }
     if (B == 0) return RSD_OK;
     cudaStream_t s = (cudaStream_t)stream;
@@ -98,7 +115,7 @@ int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int3
     a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
     a.subtract_lse = 1;
     a.out_token = out_token; a.out_perturbed = out_perturbed; a.out_value = out_logprob; a.out_lse = nullptr;
-    a.status = status;
+    a.status = status; a.node_token = node_token; a.node_stride = node_stride;
     const bool need_lse = !draft->is_logprob && (out_perturbed || out_logprob);
     launch_scan(draft, need_lse, B * R, a, s);
     return check_launch("rsd_gumbel_topk_draft");
@@ -112,9 +129,9 @@ size_t rsd_sbs_workspace_bytes(int B, int n_par, int W) {
 
 int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, int32_t first_parent_node,
                  const float* sum_logprob_in, const float* trunc_gumbel_in, uint64_t seed, uint32_t step,
-                 uint32_t seq_base, int32_t* out_token, int32_t* out_parent, float* sum_logprob_out,
-                 float* trunc_gumbel_out, int32_t* out_count, int32_t* status, void* ws, size_t ws_bytes,
-                 rsd_stream_t stream) {
+                 uint32_t seq_base, int32_t* out_token, int32_t* out_parent, int64_t out_stride, int32_t parent_base,
+                 float* sum_logprob_out, float* trunc_gumbel_out, int32_t* out_count, int32_t* status, void* ws,
+                 size_t ws_bytes, rsd_stream_t stream) {
     g_err[0] = 0;
     if (int e = check_vocab(V)) return e;
     if (int e = check_rows("draft_level", draft_level, V, n_par > 1)) return e;
@@ -124,6 +141,8 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     if (n_par * W > 1024) return fail(RSD_ERR_UNSUPPORTED, "n_par * W = %d > 1024", n_par * W);
     if (first_parent_node < 0 || (int64_t)first_parent_node + n_par > (1 << 28)) return fail(RSD_ERR_INVALID_ARG, "first_parent_node out of range");
     if (!out_token || !out_parent || !sum_logprob_out || !trunc_gumbel_out || !out_count || !status) return fail(RSD_ERR_INVALID_ARG, "null output");
+    if (out_stride < W) return fail(RSD_ERR_INVALID_ARG, "out_stride = %lld < W = %d", (long long)out_stride, W);
+    if (parent_base < 0) return fail(RSD_ERR_INVALID_ARG, "parent_base = %d", parent_base);
     if ((int64_t)B * n_par > 0x7FFFFFFF) return fail(RSD_ERR_UNSUPPORTED, "B * n_par too large");
     if (B == 0) return RSD_OK;
     const size_t need = rsd_sbs_workspace_bytes(B, n_par, W);
@@ -155,7 +174,8 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     e.seed_lo = (uint32_t)seed; e.seed_hi = (uint32_t)(seed >> 32); e.step = step; e.seq_base = seq_base;
     e.fin_token = fin_token; e.fin_value = fin_value; e.fin_lse = fin_lse;
     e.sum_in = sum_logprob_in; e.gamma_in = trunc_gumbel_in;
-    e.out_token = out_token; e.out_parent = out_parent; e.sum_out = sum_logprob_out; e.gamma_out = trunc_gumbel_out;
+    e.out_token = out_token; e.out_parent = out_parent; e.out_stride = out_stride; e.parent_base = parent_base;
+    e.sum_out = sum_logprob_out; e.gamma_out = trunc_gumbel_out;
     e.out_count = out_count; e.status = status;
     const size_t smem = (size_t)n_par * W * (8 + 8 + 4);
     rsd::sbs_epilogue_kernel<<<B, rsd::kEpilogueThreads, smem, s>>>(e);

@@ -28,8 +28,11 @@ struct ScanArgs {
     float* out_value;     // [B][R][max_k] or null: the row's own value at each pick
     float* out_lse;       // [B][R] or null
     int32_t* status;      // [B], OR-ed into
+    int32_t* node_token;  // [B][node_stride] or null: pick j of row r also goes to node child_base[r] + j
+    int node_stride;
     uint8_t k_row[kMaxRows];
     int32_t node_row[kMaxRows];
+    int32_t child_base[kMaxRows];
 };
 
 __device__ __forceinline__ bool better(float v1, int i1, float v2, int i2) {
@@ -233,11 +236,13 @@ __global__ void __launch_bounds__(kScanThreads) scan_topk_kernel(const ScanArgs 
     const float shift = (a.subtract_lse && NEED_LSE) ? lse : 0.0f;
     if (mine && rank < k) {
         a.out_token[o + rank] = top.idx;
+        if (a.node_token) a.node_token[(int64_t)b * a.node_stride + a.child_base[r] + rank] = top.idx;
         if (a.out_perturbed) a.out_perturbed[o + rank] = top.v - shift;
         if (a.out_value) a.out_value[o + rank] = top.raw - shift;
     }
     if (tid >= total && tid < a.max_k) {
         a.out_token[o + tid] = -1;
+        if (a.node_token && tid < k) a.node_token[(int64_t)b * a.node_stride + a.child_base[r] + tid] = -1;
         if (a.out_perturbed) a.out_perturbed[o + tid] = kNegInf;
         if (a.out_value) a.out_value[o + tid] = kNegInf;
     }
@@ -267,8 +272,10 @@ struct SbsEpilogueArgs {
     const float* fin_lse;      // [B][n_par]
     const float* sum_in;       // [B][n_par] or null
     const float* gamma_in;     // [B][n_par] or null
-    int32_t* out_token;
-    int32_t* out_parent;
+    int32_t* out_token;   // [B][out_stride]
+    int32_t* out_parent;  // [B][out_stride], parent_base added
+    int64_t out_stride;
+    int32_t parent_base;
     float* sum_out;
     float* gamma_out;
     int32_t* out_count;
@@ -346,8 +353,8 @@ __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const Sb
         }
         if (rank < a.W) {
             const int64_t o = (int64_t)b * a.W + rank;
-            a.out_token[o] = x;
-            a.out_parent[o] = f / a.W;
+            a.out_token[(int64_t)b * a.out_stride + rank] = x;
+            a.out_parent[(int64_t)b * a.out_stride + rank] = a.parent_base + f / a.W;
             a.sum_out[o] = (float)s_phi[f];
             a.gamma_out[o] = (float)psi;
         }
@@ -360,8 +367,8 @@ __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const Sb
     const int cnt = s_cnt < a.W ? s_cnt : a.W;
     if (tid >= cnt && tid < a.W) {
         const int64_t o = (int64_t)b * a.W + tid;
-        a.out_token[o] = -1;
-        a.out_parent[o] = -1;
+        a.out_token[(int64_t)b * a.out_stride + tid] = -1;
+        a.out_parent[(int64_t)b * a.out_stride + tid] = -1;
         a.sum_out[o] = kNegInf;
         a.gamma_out[o] = kNegInf;
     }

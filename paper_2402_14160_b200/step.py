@@ -1,0 +1,99 @@
+"""One draft + verify step over resident logits, as a fixed sequence of librsd calls.
+
+These classes only own buffers and issue the C-ABI calls in order (Algorithm 2 for constant branching factors,
+Algorithm 7 for Stochastic Beam Search, with the language-model calls replaced by rows that already sit in device
+memory).  The drafting calls write the tree's token/parent arrays in place, so no tensor work happens between the
+library's kernels.
+"""
+from __future__ import annotations
+
+from typing import Sequence
+
+import torch
+
+from . import api
+
+
+class RsdCStep:
+    """RSD with constant branching factors b = (b_0, ..., b_{L-1}) for a batch of B sequences."""
+
+    def __init__(self, B: int, V: int, branching: Sequence[int], device="cuda"):
+        self.B, self.V, self.branching = B, V, tuple(int(b) for b in branching)
+        self.L = len(self.branching)
+        sizes = [1]
+        for b in self.branching:
+            sizes.append(sizes[-1] * b)
+        off = [0]
+        for n in sizes:
+            off.append(off[-1] + n)
+        self.level_offsets = off
+        self.P, self.n_nodes = off[-2], off[-1]
+        k, child_base, parent = [], [], [-1] * self.n_nodes
+        for l, b in enumerate(self.branching):
+            for i in range(sizes[l]):
+                k.append(b)
+                child_base.append(off[l + 1] + i * b)
+                for j in range(b):
+                    parent[off[l + 1] + i * b + j] = off[l] + i
+        self.k_per_row, self.child_base = k, child_base
+        self.rng_node = list(range(self.P))
+        self.max_k = max(k)
+        self.parent = torch.tensor(parent, dtype=torch.int32, device=device)
+        self.token = torch.full((B, self.n_nodes), -1, dtype=torch.int32, device=device)
+        self.draft_out = dict(token=torch.empty((B, self.P, self.max_k), dtype=torch.int32, device=device),
+                              status=torch.empty((B,), dtype=torch.int32, device=device), perturbed=None, logprob=None)
+        self.verify_out = None
+        self.kernel_launches = 2  # one scan, one walk
+
+    def run(self, draft: torch.Tensor, target: torch.Tensor, seed: int, step: int, seq_base: int = 0):
+        api.rsd_gumbel_topk_draft(draft, self.k_per_row, self.rng_node, seed, step, seq_base=seq_base,
+                                  max_k=self.max_k, child_base=self.child_base, node_token=self.token,
+                                  out=self.draft_out)
+        self.verify_out = api.rsd_verify_tree(draft, target, self.parent, self.token, self.L, seed, step,
+                                              seq_base=seq_base, out=self.verify_out)
+        return self.verify_out
+
+
+class RsdSStep:
+    """RSD with Stochastic Beam Search of width W and depth L for a batch of B sequences."""
+
+    def __init__(self, B: int, V: int, W: int, L: int, draft_is_logprob: bool = False, device="cuda"):
+        self.B, self.V, self.W, self.L, self.is_logprob = B, V, W, L, draft_is_logprob
+        self.n_nodes = 1 + W * L
+        self.P = 1 + W * (L - 1)
+        self.parent = torch.full((B, self.n_nodes), -1, dtype=torch.int32, device=device)
+        self.token = torch.full((B, self.n_nodes), -1, dtype=torch.int32, device=device)
+        self.state = [dict(sum_logprob=torch.empty((B, W), dtype=torch.float32, device=device),
+                           trunc_gumbel=torch.empty((B, W), dtype=torch.float32, device=device)) for _ in range(2)]
+        self.count = torch.empty((L, B), dtype=torch.int32, device=device)
+        self.status = torch.empty((L, B), dtype=torch.int32, device=device)
+        self.workspace = torch.empty((api.rsd_sbs_workspace_bytes(B, W, W),), dtype=torch.uint8, device=device)
+        self.verify_out = None
+        self.kernel_launches = 2 * L + 1  # per level one scan and one epilogue, then one walk
+
+    def level_slice(self, l: int):
+        return slice(1 + l * self.W, 1 + (l + 1) * self.W)
+
+    def run(self, draft: torch.Tensor, target: torch.Tensor, seed: int, step: int, seq_base: int = 0):
+        W = self.W
+        for l in range(self.L):
+            first = 0 if l == 0 else 1 + (l - 1) * W
+            n_par = 1 if l == 0 else W
+            prev, cur = self.state[(l + 1) % 2], self.state[l % 2]
+            sl = self.level_slice(l)
+            out = dict(token=self.token[:, sl], parent=self.parent[:, sl], sum_logprob=cur["sum_logprob"],
+                       trunc_gumbel=cur["trunc_gumbel"], count=self.count[l], status=self.status[l])
+            api.rsd_sbs_step(draft[:, first:first + n_par], W, first, None if l == 0 else prev["sum_logprob"],
+                             None if l == 0 else prev["trunc_gumbel"], seed, step, is_logprob=self.is_logprob,
+                             seq_base=seq_base, workspace=self.workspace, out=out, parent_base=first)
+        self.verify_out = api.rsd_verify_tree(draft, target, self.parent, self.token, self.L, seed, step,
+                                              seq_base=seq_base, out=self.verify_out)
+        return self.verify_out
+
+
+def make_step(w, batch=None, device="cuda"):
+    """Step object for a workloads.Workload description."""
+    B = w.batch if batch is None else batch
+    if w.mode == "rsd_c":
+        return RsdCStep(B, w.vocab, w.branching, device=device)
+    return RsdSStep(B, w.vocab, w.beam_width, w.depth, draft_is_logprob=w.draft_is_logprob, device=device)

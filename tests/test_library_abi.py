@@ -27,11 +27,11 @@ def test_argument_validation_needs_no_gpu():
     lib = api.lib()
     rows = api.RsdRows(None, 0, 0, 0, 0)
     k = (ctypes.c_int32 * 1)(1)
-    code = lib.rsd_gumbel_topk_draft(ctypes.byref(rows), 1, 1, 8, k, k, 1, 0, 0, 0, None, None, None, None, None)
+    code = lib.rsd_gumbel_topk_draft(ctypes.byref(rows), 1, 1, 8, k, k, 1, 0, 0, 0, None, None, None, None, None, 0, None, None)
     assert code == 1 and b"null" in lib.rsd_last_error()
     rows = api.RsdRows(16, 7, 0, 8, 8)
-    code = lib.rsd_gumbel_topk_draft(ctypes.byref(rows), 1, 1, 8, k, k, 1, 0, 0, 0, None, None, None, None, None)
+    code = lib.rsd_gumbel_topk_draft(ctypes.byref(rows), 1, 1, 8, k, k, 1, 0, 0, 0, None, None, None, None, None, 0, None, None)
     assert code == 2 and b"dtype" in lib.rsd_last_error()
     rows = api.RsdRows(16, 0, 0, 8, 8)
-    code = lib.rsd_gumbel_topk_draft(ctypes.byref(rows), 1, 1, 0, k, k, 1, 0, 0, 0, None, None, None, None, None)
+    code = lib.rsd_gumbel_topk_draft(ctypes.byref(rows), 1, 1, 0, k, k, 1, 0, 0, 0, None, None, None, None, None, 0, None, None)
     assert code == 2
