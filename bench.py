@@ -165,8 +165,11 @@ def main():
     ap.add_argument("--cpu-baseline-sequences", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sequences", type=int, default=0, help="sequences per GPU (default: the workload's batch)")
     args = ap.parse_args()
     w = workloads.WORKLOADS[args.workload]
+    if args.sequences > 0:
+        w = workloads.scaled(w, batch=args.sequences)
 
     if args.impl == "reference":
         if args.steps > 20:

@@ -56,8 +56,12 @@ void launch_scan_lse(const rsd_rows* rows, bool aligned, int blocks, const rsd::
     }
 }
 
-void launch_scan(const rsd_rows* rows, bool need_lse, int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
+void launch_scan(const rsd_rows* rows, bool need_lse, int blocks, rsd::ScanArgs& a, cudaStream_t s) {
     const bool aligned = rows_aligned(rows);
+    for (int r = 0; r < 10; ++r) {
+        a.rk0[r] = a.seed_lo + (uint32_t)r * 0x9E3779B9u;
+        a.rk1[r] = a.seed_hi + (uint32_t)r * 0xBB67AE85u;
+    }
     if (g_scan_before) cudaEventRecord(g_scan_before, s);
     if (need_lse) launch_scan_lse<true>(rows, aligned, blocks, a, s);
     else launch_scan_lse<false>(rows, aligned, blocks, a, s);
