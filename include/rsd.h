@@ -145,6 +145,29 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
                  size_t ws_bytes, rsd_stream_t stream);
 
 /*
+ * rsd_sbs_step for callers that cannot allocate device memory (the paper has no counterpart).
+ * Some hosts of this library may not call cudaMalloc where they draft: code running inside a serving engine whose
+ * memory pool is fixed at start-up, a plug-in that is handed a stream but no allocator, a latency-critical loop that
+ * must not take the allocator's lock.  This entry point does the same work as rsd_sbs_step, with the same
+ * arguments except the scratch: the scratch is a fixed array of RSD_SBS_STATIC_SCRATCH_BYTES inside the library's
+ * device image, which every GPU that loads the library holds until the process exits.  The call itself allocates
+ * and frees nothing.
+ *   - Sizes: rsd_sbs_workspace_bytes(B, n_par, W) must not exceed RSD_SBS_STATIC_SCRATCH_BYTES (for example
+ *     B = 1024, n_par = 8, W = 8 needs 557,056 bytes); larger calls return RSD_ERR_WORKSPACE with a message.
+ *   - The first call on each device looks up the array's device address (with that device current) and keeps it;
+ *     make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it has to start at zero (every entry is written before
+ *     it is read) and its contents after a call are unspecified.  Two calls that overlap on the same GPU (different
+ *     streams, or different host threads) race on it: order them, or use rsd_sbs_step with separate scratch.
+ */
+enum { RSD_SBS_STATIC_SCRATCH_BYTES = 1 << 20 };
+int rsd_sbs_step_static(const rsd_rows* draft_level, int B, int n_par, int V, int W, int32_t first_parent_node,
+                        const float* sum_logprob_in, const float* trunc_gumbel_in, uint64_t seed, uint32_t step,
+                        uint32_t seq_base, int32_t* out_token, int32_t* out_parent, int64_t out_stride,
+                        int32_t parent_base, float* sum_logprob_out, float* trunc_gumbel_out, int32_t* out_count,
+                        int32_t* status, rsd_stream_t stream);
+
+/*
  * Draft-tree verification by recursive rejection sampling (Section 3.1, Eqs. 1-4, Algorithm 1; Section 3.2.2,
  * Algorithm 6).  Per sequence, starting at the root: the children of the current node are tested in stored order
  * with p = softmax(draft row of the node), q = softmax(target row of the node):

@@ -21,7 +21,7 @@ STOP_ALL_REJECTED, STOP_NO_CHILDREN, STOP_LEAF = 0, 1, 2
 MAX_K = 32
 
 EXPORTS = ["rsd_version", "rsd_rng_layout", "rsd_last_error", "rsd_profile_next_scan", "rsd_gumbel_topk_draft", "rsd_sbs_workspace_bytes",
-           "rsd_sbs_step", "rsd_verify_tree", "rsd_resample_residual"]
+           "rsd_sbs_step", "rsd_sbs_step_static", "rsd_verify_tree", "rsd_resample_residual"]
 
 
 class RsdRows(C.Structure):
@@ -60,6 +60,10 @@ def lib():
                                    C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
                                    C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]
+        l.rsd_sbs_step_static.argtypes = [C.POINTER(RsdRows), C.c_int, C.c_int, C.c_int, C.c_int, C.c_int32,
+                                          C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
+                                          C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p]
         l.rsd_verify_tree.argtypes = [C.POINTER(RsdRows), C.POINTER(RsdRows), C.POINTER(RsdTree), C.c_int, C.c_int,
                                       C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -172,6 +176,30 @@ def rsd_sbs_step(draft_level: torch.Tensor, W: int, first_parent_node: int, sum_
                               _ptr(trunc_gumbel_in), seed, step, seq_base, _ptr(out["token"]), _ptr(out["parent"]),
                               out["token"].stride(0), parent_base, _ptr(out["sum_logprob"]), _ptr(out["trunc_gumbel"]), _ptr(out["count"]),
                               _ptr(out["status"]), _ptr(workspace), workspace.numel(), _stream()))
+    return out
+
+
+SBS_STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def rsd_sbs_step_static(draft_level: torch.Tensor, W: int, first_parent_node: int,
+                        sum_logprob_in: Optional[torch.Tensor], trunc_gumbel_in: Optional[torch.Tensor], seed: int,
+                        step: int, out: dict, *, is_logprob: bool = False, seq_base: int = 0, parent_base: int = 0):
+    """rsd_sbs_step with the library's built-in scratch, for callers that may not allocate device memory.
+
+    `out` must hold the caller's own tensors (token, parent, sum_logprob, trunc_gumbel [B, W]; count, status [B]):
+    this wrapper allocates nothing either.  Raises RsdError when B * n_par * W is too large for the built-in
+    scratch.  Calls that overlap on one GPU share that scratch and race.
+    """
+    B, n_par, V = draft_level.shape
+    rows = rows_of(draft_level, is_logprob)
+    if out["token"].stride(0) != out["parent"].stride(0) or out["token"].stride(1) != 1 or out["parent"].stride(1) != 1:
+        raise RsdError("out token/parent must share a row stride and be dense along the picks")
+    _check(lib().rsd_sbs_step_static(C.byref(rows), B, n_par, V, W, first_parent_node, _ptr(sum_logprob_in),
+                                     _ptr(trunc_gumbel_in), seed, step, seq_base, _ptr(out["token"]),
+                                     _ptr(out["parent"]), out["token"].stride(0), parent_base,
+                                     _ptr(out["sum_logprob"]), _ptr(out["trunc_gumbel"]), _ptr(out["count"]),
+                                     _ptr(out["status"]), _stream()))
     return out
 
 

@@ -2,6 +2,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/rsd.h"
 #include "rsd_scan.cuh"
@@ -256,3 +257,55 @@ int rsd_resample_residual(const rsd_rows* draft_row, const rsd_rows* target_row,
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------------
+// rsd_sbs_step_static: the same level of Stochastic Beam Search with built-in scratch, for callers that must not
+// allocate.  The array below lives in the library's device image on every GPU that loads it.  In host code its
+// name is only a handle: the device address has to be asked for, once per device, with that device current.
+// ---------------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_sbs_static_scratch[RSD_SBS_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_scratch_ptr[kMaxDevices] = {};
+
+// Device address of the built-in scratch on the current device (looked up on the first call per device).
+int static_scratch_address(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(RSD_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= kMaxDevices) return fail(RSD_ERR_UNSUPPORTED, "device index %d outside [0, %d)", dev, kMaxDevices);
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_scratch_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress((void**)&p, g_sbs_static_scratch);
+        if (e != cudaSuccess || !p) return fail(RSD_ERR_CUDA, "cudaGetSymbolAddress(built-in scratch): %s", cudaGetErrorString(e));
+        g_static_scratch_ptr[dev] = p;
+    }
+    *out = g_static_scratch_ptr[dev];
+    return RSD_OK;
+}
+}  // namespace
+
+extern "C" int rsd_sbs_step_static(const rsd_rows* draft_level, int B, int n_par, int V, int W, int32_t first_parent_node,
+                                   const float* sum_logprob_in, const float* trunc_gumbel_in, uint64_t seed,
+                                   uint32_t step, uint32_t seq_base, int32_t* out_token, int32_t* out_parent,
+                                   int64_t out_stride, int32_t parent_base, float* sum_logprob_out,
+                                   float* trunc_gumbel_out, int32_t* out_count, int32_t* status, rsd_stream_t stream) {
+    g_err[0] = 0;
+    if (B < 0 || n_par < 1 || W < 1) return fail(RSD_ERR_INVALID_ARG, "B = %d, n_par = %d, W = %d", B, n_par, W);
+    const size_t need = rsd_sbs_workspace_bytes(B, n_par, W);
+    if (need > (size_t)RSD_SBS_STATIC_SCRATCH_BYTES)
+        return fail(RSD_ERR_WORKSPACE,
+                    "B = %d, n_par = %d, W = %d needs %zu bytes of scratch, the built-in scratch holds %d: "
+                    "split the batch or use rsd_sbs_step with your own scratch",
+                    B, n_par, W, need, (int)RSD_SBS_STATIC_SCRATCH_BYTES);
+    void* scratch = nullptr;
+    if (int e = static_scratch_address(&scratch)) return e;
+    // nothing in the scratch has to be cleared: the scan writes every finalist slot and every row's log-sum-exp
+    // before the epilogue reads them
+    return rsd_sbs_step(draft_level, B, n_par, V, W, first_parent_node, sum_logprob_in, trunc_gumbel_in, seed, step,
+                        seq_base, out_token, out_parent, out_stride, parent_base, sum_logprob_out, trunc_gumbel_out,
+                        out_count, status, scratch, (size_t)RSD_SBS_STATIC_SCRATCH_BYTES, stream);
+}
