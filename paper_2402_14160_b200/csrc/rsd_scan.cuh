@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_topk_kernel(const ScanArgs 
     __shared__ uint32_t cand[kCandCap];       // guessed-threshold pass: queued (index | byte << 24)
     __shared__ float sv_val[kSurvCap], sv_raw[kSurvCap];
     __shared__ int sv_idx[kSurvCap];
-    __shared__ unsigned long long s_fixed;    // running sum of exp(value - ref), fixed point
+    __shared__ uint32_t s_fixed;              // running sum of exp(value - ref), fixed point
     __shared__ int n_cand, n_surv;
     __shared__ float kth_val;
     __shared__ int nan_flag;
@@ -233,7 +233,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_topk_kernel(const ScanArgs 
     const int V = a.V, n_groups = (V + 15) >> 4;
     const int n_iter = (n_groups + kScanThreads - 1) / kScanThreads;
 
-    if (tid == 0) { tau_blk = float_to_ordered(kNegInf); nan_flag = 0; kth_val = kNegInf; s_fixed = 0ull; n_cand = 0; n_surv = 0; }
+    if (tid == 0) { tau_blk = float_to_ordered(kNegInf); nan_flag = 0; kth_val = kNegInf; s_fixed = 0u; n_cand = 0; n_surv = 0; }
 
     WarpTop top;
     top.init();
@@ -356,10 +356,12 @@ __global__ void __launch_bounds__(kScanThreads) scan_topk_kernel(const ScanArgs 
             }
             return pass;
         };
+        // one capped term per group: the 32-bit total cannot overflow
+        const float lane_cap = 2147483648.0f / (float)n_groups;
         auto add_to_sum = [&](float lane_sum) {
-            const uint32_t u = (uint32_t)fminf(lane_sum * kSumScale, 67108864.0f);  // NaN becomes the cap
+            const uint32_t u = (uint32_t)fminf(lane_sum * kSumScale, lane_cap);  // NaN becomes the cap
             const uint32_t wu = __reduce_add_sync(0xFFFFFFFFu, u);
-            if (lane == 0) atomicAdd(&s_fixed, (unsigned long long)wu);
+            if (lane == 0) atomicAdd(&s_fixed, wu);
         };
         auto tree16 = [](const float (&q)[16]) {
             return (((q[0] + q[1]) + (q[2] + q[3])) + ((q[4] + q[5]) + (q[6] + q[7]))) +
@@ -385,7 +387,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_topk_kernel(const ScanArgs 
             lse_acc = lane_sum;
             add_to_sum(lane_sum);
             __syncthreads();
-            float K = __fdividef(256.0f * mu * kSumScale, (float)*(volatile unsigned long long*)&s_fixed);
+            float K = __fdividef(256.0f * mu * kSumScale, (float)*(volatile uint32_t*)&s_fixed);
             if (!(K < 1.0e30f)) K = 1.0e30f;
 #pragma unroll
             for (int j = 0; j < 16; ++j) q[j] *= K;
@@ -403,7 +405,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_topk_kernel(const ScanArgs 
             uint4 cw = make_uint4(0, 0, 0, 0);
             if (valid) cw = philox_row(a, pr, (uint32_t)g);
             // K from the sum so far (any earlier value is valid: the threshold only rises)
-            const float S = (float)*(volatile unsigned long long*)&s_fixed;
+            const float S = (float)*(volatile uint32_t*)&s_fixed;
             float K = __fdividef(256.0f * mu * kSumScale, S);
             if (!(K < 1.0e30f)) K = 1.0e30f;
             const float e_off = __log2f(K) - c_ref;
@@ -440,7 +442,7 @@ __global__ void __launch_bounds__(kScanThreads) scan_topk_kernel(const ScanArgs 
         __syncthreads();
         const int ns = n_surv;
         ok = (n_queued <= kCandCap) && (ns >= k) && (ns <= kSurvCap) && (S_exact > 0.0) && (S_exact < 1.0e300) &&
-             (s_fixed > 0ull);
+             (s_fixed > 0u);
         if (ok) {
             lse = (float)((double)ref + log(S_exact));
             const float shift = (a.subtract_lse && NEED_LSE) ? lse : 0.0f;
