@@ -42,10 +42,9 @@ def lib():
         _lib = C.CDLL(build())
         _lib.rsd_oracle_gumbel.restype = C.c_double
         _lib.rsd_oracle_gumbel.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32]
-        _lib.rsd_oracle_gumbel_bits.restype = C.c_uint32
-        _lib.rsd_oracle_gumbel_bits.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32]
-        _lib.rsd_oracle_gumbel_from_bits.restype = C.c_double
-        _lib.rsd_oracle_gumbel_from_bits.argtypes = [C.c_uint32]
+        _lib.rsd_oracle_gumbel_parts.restype = None
+        _lib.rsd_oracle_gumbel_parts.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32,
+                                                 C.POINTER(C.c_double), C.POINTER(C.c_int32), C.POINTER(C.c_double)]
         _lib.rsd_oracle_accept_uniform.restype = C.c_double
         _lib.rsd_oracle_accept_uniform.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint32]
         _lib.rsd_oracle_resample_uniform.restype = C.c_double
@@ -98,12 +97,11 @@ def gumbel(seed, step, seq, node, e):
     return lib().rsd_oracle_gumbel(seed, step, seq, node, e)
 
 
-def gumbel_bits(seed, step, seq, node, e):
-    return lib().rsd_oracle_gumbel_bits(seed, step, seq, node, e)
-
-
-def gumbel_from_bits(bits):
-    return lib().rsd_oracle_gumbel_from_bits(bits)
+def gumbel_parts(seed, step, seq, node, e):
+    """(t of the group's uniform, position of the group's largest noise, t of the element's uniform)."""
+    tg, a, te = C.c_double(), C.c_int32(), C.c_double()
+    lib().rsd_oracle_gumbel_parts(seed, step, seq, node, e, C.byref(tg), C.byref(a), C.byref(te))
+    return tg.value, a.value, te.value
 
 
 def accept_uniform(seed, step, seq, node, j):

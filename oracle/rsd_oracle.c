@@ -17,7 +17,7 @@
  * Random numbers.  The paper only says "standard Gumbel" and "Uniform[0,1]".
  * Both sides of the parity check draw them from the counter-based generator
  * Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) with the counter layout
- * documented at rsd_oracle_gumbel() below (RNG layout version 1).
+ * documented at rsd_oracle_gumbel() below (RNG layout version 2).
  *
  * Pins (see tests, "-m 'not gpu'"): Philox known answers and bijectivity,
  * Gumbel moments/CDF, Plackett-Luce law of Gumbel-Top-k, exact enumeration of
@@ -92,33 +92,40 @@ static void draw(uint64_t seed, uint32_t step, uint32_t seq, uint32_t node, uint
     rsd_oracle_philox4x32_10(ctr, key, out);
 }
 
-int rsd_oracle_rng_layout(void) { return 1; }
+int rsd_oracle_rng_layout(void) { return 2; }
 
 /*
- * The 32 random bits of vocabulary element e of (sequence, node): the top
- * byte comes from the coarse stream (one Philox call covers 16 consecutive
- * elements, byte e%16 of the 16 output bytes in little-endian word order),
- * the low 24 bits from the fine stream (one call covers 4 consecutive
- * elements, word e%4, its upper 24 bits).
+ * Gumbel noise of (sequence, node), RNG layout 2.  The noise of the V elements must be i.i.d. standard Gumbel
+ * (Eq. 6).  It is drawn group-wise, 16 consecutive elements per group, from the order statistics of 16 i.i.d.
+ * uniforms: the largest of them is V^(1/16) for a uniform V, it sits at a uniformly random position a, and the
+ * other 15 are i.i.d. uniform below it.  With t(U) = -ln U this reads
+ *     coarse stream, index = group: word 0 -> U_M, word 1 (low 4 bits) -> a
+ *     fine stream, index = x >> 2, word x & 3 -> U_x                  (32 bits each, U = (bits + 1/2) / 2^32)
+ *     G_x = -ln( t(U_M) / 16 + [x mod 16 != a] * t(U_x) ).
+ * (max of 16 uniforms M = U_M^(1/16) has -ln M = t(U_M)/16; another element is M * U_x, so -ln of it is
+ * t(U_M)/16 + t(U_x); G = -ln(-ln U).)  The element at position a carries the group's largest noise, which is
+ * known from the coarse stream alone.
  */
-uint32_t rsd_oracle_gumbel_bits(uint64_t seed, uint32_t step, uint32_t seq, uint32_t node, uint32_t e) {
-    uint32_t w[4];
-    draw(seed, step, seq, node, TAG_GUMBEL_COARSE, e >> 4, w);
-    uint32_t pos = e & 15u;
-    uint32_t h = (w[pos >> 2] >> (8u * (pos & 3u))) & 0xFFu;
-    draw(seed, step, seq, node, TAG_GUMBEL_FINE, e >> 2, w);
-    uint32_t f = w[e & 3u] >> 8;
-    return (h << 24) | f;
+static double neg_log_uniform(uint32_t bits) {
+    return -log(((double)bits + 0.5) * (1.0 / 4294967296.0));
 }
 
-/* U = (bits + 1/2) / 2^32 in (0,1);  G = -ln(-ln U)  (Eq. 6's G) */
-double rsd_oracle_gumbel_from_bits(uint32_t bits) {
-    double u = ((double)bits + 0.5) * (1.0 / 4294967296.0);
-    return -log(-log(u));
+/* the three ingredients of G_x: t(U_M) of the group, the position a, t(U_x) */
+void rsd_oracle_gumbel_parts(uint64_t seed, uint32_t step, uint32_t seq, uint32_t node, uint32_t e,
+                             double* t_group, int32_t* argmax_pos, double* t_elem) {
+    uint32_t w[4];
+    draw(seed, step, seq, node, TAG_GUMBEL_COARSE, e >> 4, w);
+    *t_group = neg_log_uniform(w[0]);
+    *argmax_pos = (int32_t)(w[1] & 15u);
+    draw(seed, step, seq, node, TAG_GUMBEL_FINE, e >> 2, w);
+    *t_elem = neg_log_uniform(w[e & 3u]);
 }
 
 double rsd_oracle_gumbel(uint64_t seed, uint32_t step, uint32_t seq, uint32_t node, uint32_t e) {
-    return rsd_oracle_gumbel_from_bits(rsd_oracle_gumbel_bits(seed, step, seq, node, e));
+    double tg, te;
+    int32_t a;
+    rsd_oracle_gumbel_parts(seed, step, seq, node, e, &tg, &a, &te);
+    return -log(tg / 16.0 + ((int32_t)(e & 15u) != a ? te : 0.0));
 }
 
 /* U for the acceptance test of the j-th child (stored order) of `node`: 24 bits, in [0,1) */

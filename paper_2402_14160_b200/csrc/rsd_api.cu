@@ -45,15 +45,26 @@ int check_vocab(int V) {
     return RSD_OK;
 }
 
+template <typename T, bool ALIGNED, bool NEED_LSE>
+void launch_scan_one(int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
+    const size_t smem = sizeof(float) * (size_t)((a.V + 15) / 16);  // one bound per group of 16 elements
+    static bool raised = false;  // per instantiation: allow the largest vocabulary's dynamic shared memory
+    if (!raised) {
+        cudaFuncSetAttribute(rsd::scan_topk_kernel<T, ALIGNED, NEED_LSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)(sizeof(float) * (RSD_MAX_VOCAB / 16)));
+        raised = true;
+    }
+    rsd::scan_topk_kernel<T, ALIGNED, NEED_LSE><<<blocks, rsd::kScanThreads, smem, s>>>(a);
+}
+
 template <bool NEED_LSE>
 void launch_scan_lse(const rsd_rows* rows, bool aligned, int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
-    using namespace rsd;
     if (rows->dtype == RSD_F32) {
-        if (aligned) scan_topk_kernel<float, true, NEED_LSE><<<blocks, kScanThreads, 0, s>>>(a);
-        else scan_topk_kernel<float, false, NEED_LSE><<<blocks, kScanThreads, 0, s>>>(a);
+        if (aligned) launch_scan_one<float, true, NEED_LSE>(blocks, a, s);
+        else launch_scan_one<float, false, NEED_LSE>(blocks, a, s);
     } else {
-        if (aligned) scan_topk_kernel<__nv_bfloat16, true, NEED_LSE><<<blocks, kScanThreads, 0, s>>>(a);
-        else scan_topk_kernel<__nv_bfloat16, false, NEED_LSE><<<blocks, kScanThreads, 0, s>>>(a);
+        if (aligned) launch_scan_one<__nv_bfloat16, true, NEED_LSE>(blocks, a, s);
+        else launch_scan_one<__nv_bfloat16, false, NEED_LSE>(blocks, a, s);
     }
 }
 
@@ -77,7 +88,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 extern "C" {
 
 int rsd_version(void) { return 100; }
-int rsd_rng_layout(void) { return 1; }
+int rsd_rng_layout(void) { return 2; }
 const char* rsd_last_error(void) { return g_err; }
 
 int rsd_profile_next_scan(void* before, void* after) {

@@ -42,46 +42,27 @@ __device__ __forceinline__ uint4 rng_draw(const RngKey& k, uint32_t node, uint32
     return philox4x32_10(index, (node & 0x0FFFFFFFu) | (tag << 28), k.seq, k.step, k.seed_lo, k.seed_hi);
 }
 
-// byte (e & 15) of the 16 coarse bytes of element group e >> 4
-__device__ __forceinline__ uint32_t coarse_byte(const uint4& w, uint32_t pos) {
-    const uint32_t word = pos < 8 ? (pos < 4 ? w.x : w.y) : (pos < 12 ? w.z : w.w);
-    return (word >> (8u * (pos & 3u))) & 0xFFu;
-}
-
-__device__ __forceinline__ uint32_t fine_bits(const RngKey& k, uint32_t node, uint32_t e) {
+// Gumbel noise, RNG layout 2: the 16 noises of a group of consecutive elements are drawn through the order
+// statistics of 16 i.i.d. uniforms.  With t(U) = -ln U,
+//     coarse stream (index = group):  word 0 -> U_M,  word 1 low 4 bits -> position a of the group's largest noise
+//     fine stream (index = x >> 2, word x & 3) -> U_x
+//     G_x = -ln( t(U_M) / 16 + [x mod 16 != a] t(U_x) ),
+// so the element at position a has the largest noise of its group, -ln(t(U_M) / 16), known from the coarse stream.
+__device__ __forceinline__ uint32_t fine_word(const RngKey& k, uint32_t node, uint32_t e) {
     const uint4 w = rng_draw(k, node, kTagGumbelFine, e >> 2);
     const uint32_t sel = e & 3u;
-    const uint32_t word = sel < 2 ? (sel == 0 ? w.x : w.y) : (sel == 2 ? w.z : w.w);
-    return word >> 8;
+    return sel < 2 ? (sel == 0 ? w.x : w.y) : (sel == 2 ? w.z : w.w);
 }
 
-// G = -ln(-ln U), U = (bits + 1/2) / 2^32, in fp32 with ~1e-7 relative error in the inner logarithm.
-// For U >= 1/2 the inner term uses 1 - U, which is exact in fp32 when it is small.
-__device__ __forceinline__ float gumbel_f32(uint32_t bits) {
-    float t;
-    if (bits < 0x80000000u) {
-        const float u = ((float)bits + 0.5f) * 2.3283064365386963e-10f;  // (bits + 1/2) / 2^32
-        t = -logf(u);
-    } else {
-        const float eps = ((float)(~bits) + 0.5f) * 2.3283064365386963e-10f;  // 1 - U = (2^32 - 1 - bits + 1/2) / 2^32
-        t = -log1pf(-eps);
-    }
-    return -logf(t);
+// t = -ln U, U = (bits + 1/2) / 2^32, in fp32 with ~1e-7 relative error (for U >= 1/2 through 1 - U, which is
+// exact in fp32 when it is small).
+__device__ __forceinline__ float neg_log_uniform_f32(uint32_t bits) {
+    if (bits < 0x80000000u) return -logf(((float)bits + 0.5f) * 2.3283064365386963e-10f);
+    return -log1pf(-(((float)(~bits) + 0.5f) * 2.3283064365386963e-10f));  // 1 - U = (2^32 - 1 - bits + 1/2) / 2^32
 }
-
-__device__ __forceinline__ double gumbel_f64(uint32_t bits) {
-    const double u = ((double)bits + 0.5) * (1.0 / 4294967296.0);
-    return -log(-log(u));
+__device__ __forceinline__ double neg_log_uniform_f64(uint32_t bits) {
+    return -log(((double)bits + 0.5) * (1.0 / 4294967296.0));
 }
-
-// Upper bound of G over all elements whose top byte is h (strictly above every attainable value, with slack).
-__device__ __forceinline__ float gumbel_upper_bound(uint32_t h) {
-    if (h >= 255u) return 23.0f;  // bits = 2^32 - 1 gives G = 22.87
-    const float u = (float)(h + 1u) * (1.0f / 256.0f);
-    return -__logf(-__logf(u)) + 2e-3f;
-}
-// Largest upper bound over h <= 254: -ln(-ln(255/256)) = 5.5432.
-constexpr float kGumbelBoundBelow255 = 5.55f;
 
 // ---------------------------------------------------------------------------------------------------------
 // 16 consecutive elements of a row as fp32 registers

@@ -1,11 +1,13 @@
 // Row scan: exact sorted arg-top-k of (row + Gumbel noise) in one pass over the row (Eqs. 6-7, Algorithm 4), and
 // the per-sequence epilogue of a Stochastic Beam Search level (Eqs. 10-12, Algorithm 9).
 //
-// The noise of an element is 32 random bits: a coarse byte (16 elements per Philox call) on top of 24 fine bits
-// (4 elements per call).  G is increasing in those bits, so the byte alone bounds G from above.  Every element is
-// tested against "value + bound >= tau", where tau is a running lower bound of the k-th largest perturbed value;
-// only the few that pass get their fine bits and an exact G.  Nothing that could be among the k largest is ever
-// skipped, so the result equals the plain definition (perturb everything, sort) in fp32.
+// The noise of a group of 16 consecutive elements is drawn through its order statistics (see rsd_device.cuh): one
+// Philox call per group gives the group's largest noise and the element that carries it.  The streaming loop
+// therefore needs, per group, only the largest value of the group: value_max + noise_max bounds every perturbed
+// value of the group from above, and value(a) + noise_max is the exact perturbed value of one element, i.e. a
+// sample from below.  The k-th largest of those samples is a true lower bound tau of the k-th largest perturbed
+// value; after the loop only the groups whose upper bound reaches tau are looked at element by element, with
+// exact noise.  Nothing that could rank is skipped, so the result equals "perturb everything and sort" in fp32.
 #pragma once
 #include <cuda_fp16.h>
 
@@ -13,14 +15,13 @@
 
 namespace rsd {
 
-constexpr int kScanThreads = 256;
+constexpr int kScanThreads = 128;
 constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kQueueCap = 64;  // per-warp candidate queue (a push adds at most 32 to at most 31 pending)
 constexpr int kMaxRows = 256;
 constexpr int kIdxNone = 0x7FFFFFFF;
-constexpr int kCandCap = 2048;          // block-level candidate queue of the guessed-threshold pass
-constexpr int kSurvCap = 128;           // candidates whose exact value reaches the guessed threshold
-constexpr float kSumScale = 4096.0f;    // fixed-point scale of the running sum behind the guess
+constexpr int kCandCap = 1024;          // candidate groups queued per row (more are handled in place)
+constexpr int kSurvCap = 512;           // elements whose exact perturbed value reaches the bound
 
 struct ScanArgs {
     const void* data;
@@ -96,23 +97,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return r;
 }
 
-// Sorted list of the 32 best (value, index) pairs seen by a warp: lane i holds the i-th best.
-struct WarpTop {
-    float v;
-    int idx;
-    float raw;
-    __device__ __forceinline__ void init() { v = kNegInf; idx = kIdxNone; raw = kNegInf; }
-    // all lanes call with the same candidate
-    __device__ __forceinline__ void insert(float cv, int ci, float craw, int lane) {
-        const int pos = __popc(__ballot_sync(0xFFFFFFFFu, better(v, idx, cv, ci)));
-        const float uv = __shfl_up_sync(0xFFFFFFFFu, v, 1);
-        const int ui = __shfl_up_sync(0xFFFFFFFFu, idx, 1);
-        const float ur = __shfl_up_sync(0xFFFFFFFFu, raw, 1);
-        if (lane > pos) { v = uv; idx = ui; raw = ur; }
-        else if (lane == pos) { v = cv; idx = ci; raw = craw; }
-    }
-};
-
 // The 16 elements of a group as loaded (fp32: four 16-byte words, bf16: two), kept packed while they wait.
 template <typename T>
 struct Packed;
@@ -186,43 +170,67 @@ struct Packed<__nv_bfloat16> {
     }
 };
 
-__device__ __forceinline__ float warp_sum_f32(float v) {
+// largest of the 16 values, NaN if any is NaN
+__device__ __forceinline__ float group_max_nan(const Packed<float>& p) {
+    float m = max_nan(max_nan(__uint_as_float(p.w[0].x), __uint_as_float(p.w[0].y)),
+                      max_nan(__uint_as_float(p.w[0].z), __uint_as_float(p.w[0].w)));
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-    return v;
+    for (int i = 1; i < 4; ++i)
+        m = max_nan(m, max_nan(max_nan(__uint_as_float(p.w[i].x), __uint_as_float(p.w[i].y)),
+                               max_nan(__uint_as_float(p.w[i].z), __uint_as_float(p.w[i].w))));
+    return m;
+}
+__device__ __forceinline__ uint32_t bf162_max_nan(uint32_t a, uint32_t b) {
+    uint32_t r;
+    asm("max.NaN.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+    return r;
+}
+__device__ __forceinline__ float group_max_nan(const Packed<__nv_bfloat16>& p) {
+    const uint32_t a = bf162_max_nan(bf162_max_nan(p.w[0].x, p.w[0].y), bf162_max_nan(p.w[0].z, p.w[0].w));
+    const uint32_t b = bf162_max_nan(bf162_max_nan(p.w[1].x, p.w[1].y), bf162_max_nan(p.w[1].z, p.w[1].w));
+    const uint32_t m = bf162_max_nan(a, b);
+    return max_nan(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+}
+// element `pos` (0..15) of the group, by a select tree (no dynamic register indexing)
+__device__ __forceinline__ uint32_t pick_word(const uint4& q, int i) {
+    const uint32_t lo = (i & 1) ? q.y : q.x, hi = (i & 1) ? q.w : q.z;
+    return (i & 2) ? hi : lo;
+}
+__device__ __forceinline__ float group_element(const Packed<float>& p, int pos) {
+    const uint32_t a = pick_word(p.w[0], pos), b = pick_word(p.w[1], pos), c = pick_word(p.w[2], pos),
+                   d = pick_word(p.w[3], pos);
+    const uint32_t lo = (pos & 4) ? b : a, hi = (pos & 4) ? d : c;
+    return __uint_as_float((pos & 8) ? hi : lo);
+}
+__device__ __forceinline__ float group_element(const Packed<__nv_bfloat16>& p, int pos) {
+    const int wi = pos >> 1;
+    const uint32_t a = pick_word(p.w[0], wi), b = pick_word(p.w[1], wi);
+    const uint32_t w = (wi & 4) ? b : a;
+    return __uint_as_float((pos & 1) ? (w & 0xFFFF0000u) : (w << 16));
 }
 
-// Expected number of elements above the guessed threshold, chosen so that fewer than k is a 1e-5 event.
-__device__ __forceinline__ float guess_mean_count(int k) { return (float)k + 4.0f * sqrtf((float)k) + 8.0f; }
+// Bounds of the group's largest noise G_max = -ln(t / 16), t = -ln((bits + 1/2) / 2^32), from fast logarithms:
+// lo <= G_max <= hi.  (|t_hat - t| <= 2.5e-7 + 1e-6 t covers the conversion and lg2.approx; the outer logarithm
+// adds at most 2e-6; hi is +huge when t_hat is too small to bound.)
+__device__ __forceinline__ void group_noise_bounds(uint32_t bits, float& lo, float& hi) {
+    const float u = fmaf((float)bits, 2.3283064365386963e-10f, 1.1641532182693481e-10f);
+    const float t_hat = -__logf(u);
+    const float dt = fmaf(t_hat, 1e-6f, 2.5e-7f);
+    hi = -__logf(fmaxf(t_hat - dt, 1e-37f) * 0.0625f) + 2e-4f;
+    lo = -__logf((t_hat + dt) * 0.0625f) - 2e-4f;
+}
 
-// One block per row.  Two ways through the row, with the same result:
-//
-//  guessed threshold (tried first).  With q(x) = exp(value(x) - ref) and S the sum of q over the elements read so
-//    far, tau = ref + ln(S / mu) is exceeded by about mu of those elements' perturbed values (a Poisson count), so
-//    it is very likely at most the k-th largest.  An element can reach tau only if its uniform U exceeds
-//    exp(-q mu / S) >= 1 - q mu / S; with h the top byte of U that needs 255 - h <= 256 mu q / S, an integer
-//    compare per element.  Elements that pass are queued, get their exact noise, and enter the warp's sorted
-//    list.  At the end the guess is CHECKED: if the k-th value found is at least the largest tau used, nothing
-//    that was skipped could have ranked, and the result is exact.  Otherwise the row is redone the other way.
-//
-//  running bound.  tau is the k-th largest perturbed value found so far (a true lower bound from the start, so
-//    there is nothing to check); the test per element uses the bound of G given its byte.  Slower at the start of
-//    a row, used only when the check above fails (fewer than k finite entries, overflow of q, bad luck).
+// One block per row.
 template <typename T, bool ALIGNED, bool NEED_LSE>
-__global__ void __launch_bounds__(kScanThreads) scan_topk_kernel(const ScanArgs a) {
-    __shared__ uint32_t q_idxh[kScanWarps][kQueueCap];
-    __shared__ uint32_t tau_blk;  // order-preserving encoding of the block's best lower bound (running-bound mode)
-    __shared__ float m_v[kScanWarps * 32], m_raw[kScanWarps * 32];
-    __shared__ int m_idx[kScanWarps * 32];
-    __shared__ float red_f[kScanWarps];
-    __shared__ double red_d[kScanWarps];
-    __shared__ uint32_t cand[kCandCap];       // guessed-threshold pass: queued (index | byte << 24)
+__global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanArgs a) {
+    extern __shared__ float ub[];                    // [n_groups] upper bound of each group's perturbed values
+    __shared__ int cand[kCandCap];                   // groups whose bound reaches tau
     __shared__ float sv_val[kSurvCap], sv_raw[kSurvCap];
     __shared__ int sv_idx[kSurvCap];
-    __shared__ uint32_t s_fixed;              // running sum of exp(value - ref), fixed point
-    __shared__ int n_cand, n_surv;
-    __shared__ float kth_val;
-    __shared__ int nan_flag;
+    __shared__ uint32_t bin_max[32];                 // per lane index: largest sample over the warps (ordered encoding)
+    __shared__ float red_f[kScanWarps];
+    __shared__ double red_d[kScanWarps];
+    __shared__ int n_cand, n_surv, nan_flag;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / a.R, r = blockIdx.x % a.R;
@@ -232,279 +240,48 @@ __global__ void __launch_bounds__(kScanThreads) scan_topk_kernel(const ScanArgs 
     const char* row = (const char*)a.data + ((int64_t)b * a.seq_stride + (int64_t)r * a.row_stride) * RowIO<T>::kBytes;
     const int V = a.V, n_groups = (V + 15) >> 4;
     const int n_iter = (n_groups + kScanThreads - 1) / kScanThreads;
+    const PhiloxRow pr = philox_row_setup(a, (node & 0x0FFFFFFFu) | (kTagGumbelCoarse << 28), key.seq, key.step);
 
-    if (tid == 0) { tau_blk = float_to_ordered(kNegInf); nan_flag = 0; kth_val = kNegInf; s_fixed = 0u; n_cand = 0; n_surv = 0; }
+    if (tid == 0) { n_cand = 0; n_surv = 0; nan_flag = 0; }
+    if (tid < 32) bin_max[tid] = float_to_ordered(kNegInf);
+    __syncthreads();
 
-    WarpTop top;
-    top.init();
-    int q_head = 0, q_count = 0;  // warp-uniform
+    // ---- streaming loop: one group per thread per sweep ------------------------------------------------------------
+    float best = kNegInf;                  // largest exact sample of this thread (value(a) + lower bound of G_max)
+    float lse_m = kNegInf, lse_s = 0.0f;   // running log-sum-exp of this thread's elements
     bool saw_nan = false;
-
-    // Take up to 32 queued candidates: (bound test with the exact byte,) exact noise, insertion.
-    auto drain = [&](int n, bool use_bound) {
-        const bool have = lane < n;
-        uint32_t idxh = 0;
-        if (have) idxh = q_idxh[warp][(q_head + lane) & (kQueueCap - 1)];
-        const int idx = (int)(idxh & 0x00FFFFFFu);
-        const uint32_t h = idxh >> 24;
-        float raw = kNegInf;
-        if (have && idx < V) {  // padding of the last group is never read
-            raw = RowIO<T>::scalar(row, idx);
-            if (raw != raw) { saw_nan = true; raw = kNegInf; }
+    Packed<T> nxt;
+    if (tid < n_groups) nxt.load(row, tid, V, ALIGNED && (tid + 1) * 16 <= V);
+    else nxt.fill_neg_inf();
+    for (int it = 0; it < n_iter; ++it) {
+        const int g = it * kScanThreads + tid;
+        const Packed<T> cur = nxt;
+        if (it + 1 < n_iter) {
+            const int g2 = g + kScanThreads;
+            if (g2 < n_groups) nxt.load(row, g2, V, ALIGNED && (g2 + 1) * 16 <= V);
+            else nxt.fill_neg_inf();
         }
-        bool pass = have && raw > kNegInf;
-        if (use_bound) {
-            const float tau = fmaxf(__shfl_sync(0xFFFFFFFFu, top.v, k - 1), ordered_to_float(*(volatile uint32_t*)&tau_blk));
-            pass = pass && (raw + gumbel_upper_bound(h) >= tau);
-        }
-        float pert = kNegInf;
-        if (pass) pert = raw + gumbel_f32((h << 24) | fine_bits(key, node, (uint32_t)idx));
-        unsigned m = __ballot_sync(0xFFFFFFFFu, pass);
-        while (m) {
-            const int src = __ffs(m) - 1;
-            m &= m - 1;
-            const float cv = __shfl_sync(0xFFFFFFFFu, pert, src);
-            const int ci = __shfl_sync(0xFFFFFFFFu, idx, src);
-            const float cr = __shfl_sync(0xFFFFFFFFu, raw, src);
-            const float kv = __shfl_sync(0xFFFFFFFFu, top.v, k - 1);
-            const int ki = __shfl_sync(0xFFFFFFFFu, top.idx, k - 1);
-            if (better(cv, ci, kv, ki)) top.insert(cv, ci, cr, lane);
-        }
-        q_head = (q_head + n) & (kQueueCap - 1);
-        q_count -= n;
-        if (use_bound) {
-            const float tw = __shfl_sync(0xFFFFFFFFu, top.v, k - 1);
-            if (lane == 0 && tw > kNegInf) atomicMax(&tau_blk, float_to_ordered(tw));
-        }
-        __syncwarp();
-    };
-
-    // Merge the warps' lists: every entry learns its rank among all entries; returns the number of picks found.
-    int rank = 0;
-    bool mine = false;
-    auto merge_lists = [&]() -> int {
-        __syncthreads();
-        m_v[tid] = top.v;
-        m_idx[tid] = top.idx;
-        m_raw[tid] = top.raw;
-        if (tid == 0) kth_val = kNegInf;
-        __syncthreads();
-        mine = lane < k && top.idx != kIdxNone;
-        rank = 0;
-        if (mine) {
-            for (int w = 0; w < kScanWarps; ++w)
-                for (int i = 0; i < k; ++i) {
-                    const int e = w * 32 + i;
-                    rank += (m_idx[e] != kIdxNone && better(m_v[e], m_idx[e], top.v, top.idx)) ? 1 : 0;
-                }
-            if (rank == k - 1) kth_val = top.v;
-        }
-        const int cnt = __syncthreads_count(mine);
-        return cnt < k ? cnt : k;
-    };
-
-    // ---- reference for the exponentials: the largest value of the first sweep -------------------------------
-    Packed<T> first;
-    if (tid < n_groups) first.load(row, tid, V, ALIGNED && (tid + 1) * 16 <= V);
-    else first.fill_neg_inf();
-    float ref;
-    {
-        float v[16];
-        first.unpack(v);
-        float vm = kNegInf;
-#pragma unroll
-        for (int j = 0; j < 16; ++j) vm = fmaxf(vm, v[j]);  // ignores NaN
-        ref = block_max<kScanThreads>(vm, red_f);
-        if (!(ref > kNegInf) || !(ref < -kNegInf)) ref = 0.0f;
-    }
-
-    // ---- attempt 1: guessed threshold ---------------------------------------------------------------------------
-    float lse = 0.0f;
-    int total = 0;
-    bool ok;
-    {
-        const float mu = guess_mean_count(k);
-        const float c_ref = ref * kLog2e;
-        const PhiloxRow pr = philox_row_setup(a, (node & 0x0FFFFFFFu) | (kTagGumbelCoarse << 28), key.seq, key.step);
-        float lse_acc = 0.0f;  // this lane's share of sum_x exp(value - ref)
-
-        // candidates of one group: bit (j >> 1) + 16 (j & 1) of `pass` <-> element j
-        auto push = [&](uint32_t pass, const uint4& cw, int g) {
-            while (pass) {
-                const int bit = __ffs(pass) - 1;
-                pass &= pass - 1;
-                const int j = ((bit & 15) << 1) | (bit >> 4);
-                const uint32_t word = j < 8 ? (j < 4 ? cw.x : cw.y) : (j < 12 ? cw.z : cw.w);
-                const uint32_t h = (word >> (8 * (j & 3))) & 0xFFu;
-                const int slot = atomicAdd(&n_cand, 1);
-                if (slot < kCandCap) cand[slot] = (uint32_t)(g * 16 + j) | (h << 24);
-            }
-        };
-        // 255 - h_j <= round(x_j) for the 16 scaled values x = K q of a group, two at a time in half precision:
-        // (1024 + x_j) >= (1024 + 255 - h_j), where 1024 + c has the bit pattern 0x6400 | c.
-        auto byte_test = [&](const float (&x)[16], const uint4& cw) -> uint32_t {
-            const uint32_t inv[4] = {~cw.x, ~cw.y, ~cw.z, ~cw.w};
-            const __half2 bias = __floats2half2_rn(1024.0f, 1024.0f);
-            uint32_t pass = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const __half2 y = __hadd2(__floats2half2_rn(x[2 * i], x[2 * i + 1]), bias);
-                const uint32_t b0 = (uint32_t)((2 * i) & 3);
-                const uint32_t cbits = __byte_perm(inv[i >> 1], 0x64646464u, 0x4040u | ((b0 + 1u) << 8) | b0);
-                const uint32_t m = __hgeu2_mask(y, *reinterpret_cast<const __half2*>(&cbits));
-                pass |= m & ((1u << i) | (1u << (16 + i)));
-            }
-            return pass;
-        };
-        // one capped term per group: the 32-bit total cannot overflow
-        const float lane_cap = 2147483648.0f / (float)n_groups;
-        auto add_to_sum = [&](float lane_sum) {
-            const uint32_t u = (uint32_t)fminf(lane_sum * kSumScale, lane_cap);  // NaN becomes the cap
-            const uint32_t wu = __reduce_add_sync(0xFFFFFFFFu, u);
-            if (lane == 0) atomicAdd(&s_fixed, wu);
-        };
-        auto tree16 = [](const float (&q)[16]) {
-            return (((q[0] + q[1]) + (q[2] + q[3])) + ((q[4] + q[5]) + (q[6] + q[7]))) +
-                   (((q[8] + q[9]) + (q[10] + q[11])) + ((q[12] + q[13]) + (q[14] + q[15])));
-        };
-
-        // first sweep: block-wide sum, then the byte test with K from it
-        Packed<T> nxt;
-        {
-            if (n_iter > 1) {
-                const int g2 = tid + kScanThreads;
-                if (g2 < n_groups) nxt.load(row, g2, V, ALIGNED && (g2 + 1) * 16 <= V);
-                else nxt.fill_neg_inf();
-            }
-            const bool valid = tid < n_groups;
-            uint4 cw = make_uint4(0, 0, 0, 0);
-            if (valid) cw = philox_row(a, pr, (uint32_t)tid);
-            float q[16];
-            first.unpack(q);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) q[j] = ex2_approx(fmaf(q[j], kLog2e, -c_ref));
-            const float lane_sum = tree16(q);
-            lse_acc = lane_sum;
-            add_to_sum(lane_sum);
-            __syncthreads();
-            float K = __fdividef(256.0f * mu * kSumScale, (float)*(volatile uint32_t*)&s_fixed);
-            if (!(K < 1.0e30f)) K = 1.0e30f;
-#pragma unroll
-            for (int j = 0; j < 16; ++j) q[j] *= K;
-            if (valid) push(byte_test(q, cw), cw, tid);
-        }
-        for (int it = 1; it < n_iter; ++it) {
-            const int g = it * kScanThreads + tid;
-            const bool valid = g < n_groups;
-            const Packed<T> cur = nxt;
-            if (it + 1 < n_iter) {
-                const int g2 = g + kScanThreads;
-                if (g2 < n_groups) nxt.load(row, g2, V, ALIGNED && (g2 + 1) * 16 <= V);
-                else nxt.fill_neg_inf();
-            }
-            uint4 cw = make_uint4(0, 0, 0, 0);
-            if (valid) cw = philox_row(a, pr, (uint32_t)g);
-            // K from the sum so far (any earlier value is valid: the threshold only rises)
-            const float S = (float)*(volatile uint32_t*)&s_fixed;
-            float K = __fdividef(256.0f * mu * kSumScale, S);
-            if (!(K < 1.0e30f)) K = 1.0e30f;
-            const float e_off = __log2f(K) - c_ref;
-            const float inv_K = __fdividef(1.0f, K);
-            float q[16];
-            cur.unpack(q);
-#pragma unroll
-            for (int j = 0; j < 16; ++j) q[j] = ex2_approx(fmaf(q[j], kLog2e, e_off));  // K exp(value - ref)
-            const float lane_sum = tree16(q) * inv_K;
-            lse_acc += lane_sum;
-            add_to_sum(lane_sum);
-            if (valid) push(byte_test(q, cw), cw, g);
-        }
-
-        // end of row: exact values of the queued candidates, keep those that reach the final threshold
-        const double S_exact = block_sum<kScanThreads>((double)lse_acc, red_d);  // also a barrier after the pushes
-        const int n_queued = n_cand;
-        const float S_fixed = (float)s_fixed * (1.0f / kSumScale);
-        const float tau_keep = ref + logf(S_fixed / mu) + 1e-4f;  // every threshold used is below this
-        const int n_eval = n_queued < kCandCap ? n_queued : kCandCap;
-        for (int i = tid; i < n_eval; i += kScanThreads) {
-            const uint32_t idxh = cand[i];
-            const int idx = (int)(idxh & 0x00FFFFFFu);
-            if (idx >= V) continue;  // padding of the last group
-            float raw = RowIO<T>::scalar(row, idx);
-            if (raw != raw) { saw_nan = true; continue; }
-            if (!(raw > kNegInf)) continue;
-            const float pert = raw + gumbel_f32((idxh & 0xFF000000u) | fine_bits(key, node, (uint32_t)idx));
-            if (pert >= tau_keep) {
-                const int sidx = atomicAdd(&n_surv, 1);
-                if (sidx < kSurvCap) { sv_val[sidx] = pert; sv_idx[sidx] = idx; sv_raw[sidx] = raw; }
-            }
-        }
-        __syncthreads();
-        const int ns = n_surv;
-        ok = (n_queued <= kCandCap) && (ns >= k) && (ns <= kSurvCap) && (S_exact > 0.0) && (S_exact < 1.0e300) &&
-             (s_fixed > 0u);
-        if (ok) {
-            lse = (float)((double)ref + log(S_exact));
-            const float shift = (a.subtract_lse && NEED_LSE) ? lse : 0.0f;
-            const int64_t o = ((int64_t)b * a.R + r) * a.max_k;
-            if (tid < ns) {
-                const float mv = sv_val[tid];
-                const int mi = sv_idx[tid];
-                int rnk = 0;
-                for (int e = 0; e < ns; ++e) rnk += better(sv_val[e], sv_idx[e], mv, mi) ? 1 : 0;
-                if (rnk < k) {
-                    a.out_token[o + rnk] = mi;
-                    if (a.node_token) a.node_token[(int64_t)b * a.node_stride + a.child_base[r] + rnk] = mi;
-                    if (a.out_perturbed) a.out_perturbed[o + rnk] = mv - shift;
-                    if (a.out_value) a.out_value[o + rnk] = sv_raw[tid] - shift;
-                }
-            }
-            if (tid >= k && tid < a.max_k) {
-                a.out_token[o + tid] = -1;
-                if (a.out_perturbed) a.out_perturbed[o + tid] = kNegInf;
-                if (a.out_value) a.out_value[o + tid] = kNegInf;
-            }
-            if (tid == 0 && a.out_lse) a.out_lse[(int64_t)b * a.R + r] = NEED_LSE ? lse : 0.0f;
-            // a NaN makes S_exact NaN, so this path never ends with one: no status bit to set
-            return;
-        }
-    }
-
-    // ---- attempt 2: running bound (only when the check failed) ----------------------------------------------------
-    {
-        __syncthreads();
-        top.init();
-        q_head = 0;
-        q_count = 0;
-        float lse_m = kNegInf, lse_s = 0.0f;
-        for (int it = 0; it < n_iter; ++it) {
-            const int g = it * kScanThreads + tid;
-            const bool valid = g < n_groups;
-            float v[16];
-            uint4 cw = make_uint4(0, 0, 0, 0);
-            float vmax = kNegInf;
-            if (valid) {
-                load_group<T, ALIGNED>(row, g, V, v);
-                cw = rng_draw(key, node, kTagGumbelCoarse, (uint32_t)g);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) vmax = max_nan(vmax, v[j]);
-                if (vmax != vmax) {  // a NaN in this group: treat as -inf
-                    saw_nan = true;
-                    vmax = kNegInf;
+        if (g < n_groups) {
+            const uint4 cw = philox_row(a, pr, (uint32_t)g);
+            float g_lo, g_hi;
+            group_noise_bounds(cw.x, g_lo, g_hi);
+            float gmax = group_max_nan(cur);
+            ub[g] = gmax + g_hi;                                   // NaN if the group holds a NaN: looked at later
+            best = fmaxf(best, group_element(cur, (int)(cw.y & 15u)) + g_lo);  // fmaxf drops NaN
+            if (NEED_LSE) {
+                float v[16];
+                cur.unpack(v);
+                if (gmax != gmax) {  // NaN counts as -inf
+                    gmax = kNegInf;
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         if (v[j] != v[j]) v[j] = kNegInf;
-                        vmax = fmaxf(vmax, v[j]);
+                        gmax = fmaxf(gmax, v[j]);
                     }
                 }
-            } else {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) v[j] = kNegInf;
-            }
-            if (NEED_LSE) {
-                if (vmax > lse_m) {  // rescale the running sum to the new reference
-                    lse_s *= ex2_approx((lse_m - vmax) * kLog2e);  // lse_m = -inf gives 0
-                    lse_m = vmax;
+                if (gmax > lse_m) {  // rescale the running sum to the new reference
+                    lse_s *= ex2_approx((lse_m - gmax) * kLog2e);  // lse_m = -inf gives 0
+                    lse_m = gmax;
                 }
                 if (lse_m > kNegInf) {
                     const float c = lse_m * kLog2e;
@@ -517,55 +294,143 @@ __global__ void __launch_bounds__(kScanThreads) scan_topk_kernel(const ScanArgs 
                     lse_s += s0 + s1;
                 }
             }
-            // bytes below 255 bound G by kGumbelBoundBelow255; byte 255 always goes on
-            float thr = fmaxf(__shfl_sync(0xFFFFFFFFu, top.v, k - 1), ordered_to_float(*(volatile uint32_t*)&tau_blk)) -
-                        kGumbelBoundBelow255;
-            const uint32_t inv0 = ~cw.x, inv1 = ~cw.y, inv2 = ~cw.z, inv3 = ~cw.w;  // a 0xFF byte is a zero byte here
-            const uint32_t any255 = ((inv0 - 0x01010101u) & ~inv0 & 0x80808080u) | ((inv1 - 0x01010101u) & ~inv1 & 0x80808080u) |
-                                    ((inv2 - 0x01010101u) & ~inv2 & 0x80808080u) | ((inv3 - 0x01010101u) & ~inv3 & 0x80808080u);
-            const bool cand = valid && vmax > kNegInf && (vmax >= thr || any255 != 0u);
-            if (__any_sync(0xFFFFFFFFu, cand)) {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const uint32_t word = j < 8 ? (j < 4 ? cw.x : cw.y) : (j < 12 ? cw.z : cw.w);
-                    const uint32_t h = (word >> (8 * (j & 3))) & 0xFFu;
-                    const bool p = cand && v[j] > kNegInf && (v[j] >= thr || h == 255u);
-                    const unsigned bal = __ballot_sync(0xFFFFFFFFu, p);
-                    if (bal) {
-                        if (p) {
-                            const int slot = (q_head + q_count + __popc(bal & ((1u << lane) - 1u))) & (kQueueCap - 1);
-                            q_idxh[warp][slot] = (uint32_t)(g * 16 + j) | (h << 24);
-                        }
-                        q_count += __popc(bal);
-                        __syncwarp();
-                        if (q_count >= 32) {
-                            drain(32, true);
-                            thr = fmaxf(__shfl_sync(0xFFFFFFFFu, top.v, k - 1),
-                                        ordered_to_float(*(volatile uint32_t*)&tau_blk)) - kGumbelBoundBelow255;
-                        }
-                    }
-                }
-            }
-        }
-        while (q_count > 0) drain(q_count < 32 ? q_count : 32, true);
-        total = merge_lists();
-        if (NEED_LSE) {
-            const float M = block_max<kScanThreads>(lse_m, red_f);
-            const float scaled = (lse_m > kNegInf) ? lse_s * ex2_approx((lse_m - M) * kLog2e) : 0.0f;
-            const double S = block_sum<kScanThreads>((double)scaled, red_d);
-            lse = (M > kNegInf && S > 0.0) ? (float)((double)M + log(S)) : kNegInf;
         }
     }
 
+    // ---- tau: a lower bound of the k-th largest perturbed value from the threads' samples -------------------------
+    // The samples belong to distinct elements.  They are folded into 32 bins (one per lane index, maximum over the
+    // warps); the k-th largest bin maximum is at most the k-th largest sample, hence at most the k-th largest
+    // perturbed value of the row.  Every warp sorts the 32 bin maxima itself, so one barrier is enough.
+    if (best > kNegInf) atomicMax(&bin_max[lane], float_to_ordered(best));
+    if (NEED_LSE) {
+        const float wm = warp_max(lse_m);
+        if (lane == 0) red_f[warp] = wm;
+    }
+    __syncthreads();
+    float tau;
+    {
+        float v = ordered_to_float(bin_max[lane]);  // bitonic sort across the warp, ascending
+#pragma unroll
+        for (int k2 = 2; k2 <= 32; k2 <<= 1) {
+#pragma unroll
+            for (int j = k2 >> 1; j > 0; j >>= 1) {
+                const float other = __shfl_xor_sync(0xFFFFFFFFu, v, j);
+                const bool up = (lane & k2) == 0, lower = (lane & j) == 0;
+                v = (lower == up) ? fminf(v, other) : fmaxf(v, other);
+            }
+        }
+        tau = __shfl_sync(0xFFFFFFFFu, v, 32 - k);  // k-th largest (k <= 32)
+    }
+
+    // ---- candidate groups ---------------------------------------------------------------------------------------------
+    for (int it = 0; it < n_iter; ++it) {
+        const int g = it * kScanThreads + tid;
+        if (g < n_groups) {
+            const float u = ub[g];
+            if (u >= tau || u != u) {
+                const int slot = atomicAdd(&n_cand, 1);
+                if (slot < kCandCap) cand[slot] = g;
+            }
+        }
+    }
+    __syncthreads();
+    const int n_queued = n_cand;
+
+    // exact perturbed values of the elements of group g that can reach tau
+    auto process_group = [&](int g) {
+        Packed<T> grp;
+        grp.load(row, g, V, ALIGNED && (g + 1) * 16 <= V);
+        const uint4 cw = philox_row(a, pr, (uint32_t)g);
+        const float base = neg_log_uniform_f32(cw.x) * 0.0625f;   // t(U_M) / 16
+        const float g_max = -logf(base);
+        const int apos = (int)(cw.y & 15u);
+        // elements whose value plus the group's largest noise reaches tau (NaN compares false both ways: flagged)
+        uint32_t todo = 0;
+        {
+            float v[16];
+            grp.unpack(v);
+            const float need = tau - g_max - 1e-5f;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                if (v[j] != v[j]) saw_nan = true;
+                else if (v[j] > kNegInf && v[j] >= need) todo |= 1u << j;
+            }
+        }
+        while (todo) {
+            const int j = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const int x = g * 16 + j;
+            const float raw = group_element(grp, j);
+            float pert = raw + g_max;
+            if (j != apos) pert = raw - logf(base + neg_log_uniform_f32(fine_word(key, node, (uint32_t)x)));
+            if (pert >= tau) {
+                const int sidx = atomicAdd(&n_surv, 1);
+                if (sidx < kSurvCap) { sv_val[sidx] = pert; sv_idx[sidx] = x; sv_raw[sidx] = raw; }
+            }
+        }
+    };
+
+    int ns = 0;
+    for (int attempt = 0; attempt < 16; ++attempt) {
+        if (n_queued <= kCandCap) {
+            for (int i = tid; i < n_queued; i += kScanThreads) process_group(cand[i]);
+        } else {  // too many candidate groups for the queue: each thread handles its own
+            for (int it = 0; it < n_iter; ++it) {
+                const int g = it * kScanThreads + tid;
+                if (g < n_groups) {
+                    const float u = ub[g];
+                    if (u >= tau || u != u) process_group(g);
+                }
+            }
+        }
+        __syncthreads();
+        ns = n_surv;
+        if (ns <= kSurvCap) break;
+        // more elements reach tau than fit: raise tau to the k-th largest of those kept (still a lower bound)
+        float my = kNegInf;
+        for (int e = tid; e < kSurvCap; e += kScanThreads) {
+            const float mv = sv_val[e];
+            const int mi = sv_idx[e];
+            int rnk = 0;
+            for (int f = 0; f < kSurvCap; ++f) rnk += better(sv_val[f], sv_idx[f], mv, mi) ? 1 : 0;
+            if (rnk == k - 1) my = mv;
+        }
+        const float raised = block_max<kScanThreads>(my, red_f);
+        __syncthreads();
+        tau = fmaxf(tau, raised);
+        if (tid == 0) n_surv = 0;
+        __syncthreads();
+        ns = 0;
+    }
+    if (ns > kSurvCap) ns = kSurvCap;
+
+    float lse = 0.0f;
+    if (NEED_LSE) {  // the warps' maxima were published before the first barrier
+        float M = red_f[0];
+#pragma unroll
+        for (int w = 1; w < kScanWarps; ++w) M = fmaxf(M, red_f[w]);
+        const float scaled = (lse_m > kNegInf) ? lse_s * ex2_approx((lse_m - M) * kLog2e) : 0.0f;
+        const double S = block_sum<kScanThreads>((double)scaled, red_d);
+        lse = (M > kNegInf && S > 0.0) ? (float)((double)M + log(S)) : kNegInf;
+    }
     if (saw_nan) nan_flag = 1;
     __syncthreads();
+
+    // ---- rank the survivors, write the picks ----------------------------------------------------------------------------
+    const int total = ns < k ? ns : k;
     const int64_t o = ((int64_t)b * a.R + r) * a.max_k;
     const float shift = (a.subtract_lse && NEED_LSE) ? lse : 0.0f;
-    if (mine && rank < k) {
-        a.out_token[o + rank] = top.idx;
-        if (a.node_token) a.node_token[(int64_t)b * a.node_stride + a.child_base[r] + rank] = top.idx;
-        if (a.out_perturbed) a.out_perturbed[o + rank] = top.v - shift;
-        if (a.out_value) a.out_value[o + rank] = top.raw - shift;
+    for (int e = tid; e < ns; e += kScanThreads) {
+        const float mv = sv_val[e];
+        const int mi = sv_idx[e];
+        int rnk = 0;
+        for (int f = 0; f < ns; ++f) rnk += better(sv_val[f], sv_idx[f], mv, mi) ? 1 : 0;
+        if (rnk < k) {
+            a.out_token[o + rnk] = mi;
+            if (a.node_token) a.node_token[(int64_t)b * a.node_stride + a.child_base[r] + rnk] = mi;
+            if (a.out_perturbed) a.out_perturbed[o + rnk] = mv - shift;
+            if (a.out_value) a.out_value[o + rnk] = sv_raw[e] - shift;
+        }
     }
     if (tid >= total && tid < a.max_k) {
         a.out_token[o + tid] = -1;
@@ -630,9 +495,10 @@ __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const Sb
             const double lse = a.is_logprob ? 0.0 : (double)a.fin_lse[(int64_t)b * a.n_par + kpar];
             const uint32_t node = (uint32_t)(a.first_parent_node + kpar);
             const uint4 cw = rng_draw(key, node, kTagGumbelCoarse, (uint32_t)x >> 4);
-            const uint32_t bits = (coarse_byte(cw, (uint32_t)x & 15u) << 24) | fine_bits(key, node, (uint32_t)x);
+            const double t_elem = (((uint32_t)x & 15u) != (cw.y & 15u))
+                                      ? neg_log_uniform_f64(fine_word(key, node, (uint32_t)x)) : 0.0;
             phi = sigma + ((double)a.fin_value[(int64_t)b * F + f] - lse);
-            pert = phi + gumbel_f64(bits);
+            pert = phi - log(neg_log_uniform_f64(cw.x) * 0.0625 + t_elem);
         }
         s_tok[f] = x;
         s_phi[f] = phi;

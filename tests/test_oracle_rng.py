@@ -60,39 +60,54 @@ def test_philox_avalanche():
     assert abs(np.mean(flips) - 64.0) < 1.5
 
 
-def test_gumbel_bit_layout():
-    """Top byte from the coarse stream (16 elements per call), low 24 bits from the fine stream (4 per call)."""
+def test_gumbel_stream_layout():
+    """Group uniform and position from the coarse stream (16 elements per call), element uniform from the fine one."""
     seed, step, seq, node = 0x1234567811223344, 5, 17, 9
     key = [seed & MASK, seed >> 32]
     for e in [0, 1, 3, 4, 15, 16, 17, 31999, 50271]:
         coarse = oracle.philox4x32_10([e >> 4, node | (0 << 28), seq, step], key)
         fine = oracle.philox4x32_10([e >> 2, node | (1 << 28), seq, step], key)
-        pos = e & 15
-        h = (int(coarse[pos >> 2]) >> (8 * (pos & 3))) & 0xFF
-        f = int(fine[e & 3]) >> 8
-        assert oracle.gumbel_bits(seed, step, seq, node, e) == (h << 24) | f
+        tg, a, te = oracle.gumbel_parts(seed, step, seq, node, e)
+        assert math.isclose(tg, -math.log((int(coarse[0]) + 0.5) / 2.0 ** 32), rel_tol=1e-14)
+        assert a == int(coarse[1]) & 15
+        assert math.isclose(te, -math.log((int(fine[e & 3]) + 0.5) / 2.0 ** 32), rel_tol=1e-14)
+        g = oracle.gumbel(seed, step, seq, node, e)
+        assert math.isclose(g, -math.log(tg / 16 + (te if (e & 15) != a else 0.0)), rel_tol=1e-13)
 
 
 def test_streams_are_keyed_by_every_coordinate():
-    base = oracle.gumbel_bits(1, 2, 3, 4, 5)
-    assert base != oracle.gumbel_bits(2, 2, 3, 4, 5)
-    assert base != oracle.gumbel_bits(1 + (1 << 32), 2, 3, 4, 5)
-    assert base != oracle.gumbel_bits(1, 3, 3, 4, 5)
-    assert base != oracle.gumbel_bits(1, 2, 4, 4, 5)
-    assert base != oracle.gumbel_bits(1, 2, 3, 5, 5)
-    assert base != oracle.gumbel_bits(1, 2, 3, 4, 6)
+    base = oracle.gumbel(1, 2, 3, 4, 5)
+    assert base != oracle.gumbel(2, 2, 3, 4, 5)
+    assert base != oracle.gumbel(1 + (1 << 32), 2, 3, 4, 5)
+    assert base != oracle.gumbel(1, 3, 3, 4, 5)
+    assert base != oracle.gumbel(1, 2, 4, 4, 5)
+    assert base != oracle.gumbel(1, 2, 3, 5, 5)
+    assert base != oracle.gumbel(1, 2, 3, 4, 6)
     assert oracle.accept_uniform(1, 2, 3, 4, 0) != oracle.accept_uniform(1, 2, 3, 4, 1)
-    assert oracle.accept_uniform(1, 2, 3, 4, 0) != oracle.accept_uniform(1, 2, 3, 5, 0)
+    assert oracle.accept_uniform(1, 2, 3, 4, 0) != oracle.accept_uniform(1, 2, 3, 4, 5)
 
 
-def test_gumbel_transform_closed_form():
-    # U = (bits + 1/2) / 2^32, G = -ln(-ln U): checked at values with simple logarithms
-    for bits in [0, 1, 1 << 31, (1 << 32) - 1, 123456789]:
-        u = (bits + 0.5) / 2.0 ** 32
-        assert math.isclose(oracle.gumbel_from_bits(bits), -math.log(-math.log(u)), rel_tol=1e-14)
-    # the median of a standard Gumbel is -ln ln 2
-    assert abs(oracle.gumbel_from_bits(1 << 31) - (-math.log(math.log(2.0)))) < 1e-9
-    assert oracle.gumbel_from_bits(0) < -3.0 and oracle.gumbel_from_bits((1 << 32) - 1) > 22.0
+def test_group_construction_gives_iid_gumbels():
+    # The 16 noises of a group are built from their order statistics (largest first); they must come out i.i.d.
+    # standard Gumbel: right marginal at every position, the group maximum distributed as Gumbel + ln 16, the
+    # largest at a uniform position, no correlation between positions, and each pair ordered either way equally often.
+    n = 20000
+    G = np.array([[oracle.gumbel(77, 1, s, 3, 32 + j) for j in range(16)] for s in range(n)])
+    cdf = lambda x: np.exp(-np.exp(-x))
+    for j in (0, 5, 15):
+        assert stats.kstest(G[:, j], cdf).pvalue > 1e-3
+    assert stats.kstest(G.max(axis=1) - math.log(16.0), cdf).pvalue > 1e-3
+    assert stats.kstest(np.sort(G, axis=1)[:, -2], lambda x: cdf(x) ** 15 * (16 - 15 * cdf(x))).pvalue > 1e-3
+    pos = np.bincount(G.argmax(axis=1), minlength=16)
+    assert stats.chisquare(pos).pvalue > 1e-3
+    c = np.corrcoef(G.T)
+    assert np.abs(c - np.eye(16)).max() < 0.04
+    wins = (G[:, 2] > G[:, 9]).mean()
+    assert abs(wins - 0.5) < 4 * 0.5 / math.sqrt(n)
+    # the position named by the coarse stream really holds the largest noise
+    for s in range(50):
+        _, a, _ = oracle.gumbel_parts(77, 1, s, 3, 32)
+        assert int(G[s].argmax()) == a
 
 
 def test_gumbel_law():
@@ -114,4 +129,4 @@ def test_uniform_streams():
     assert stats.kstest(ua, "uniform").pvalue > 1e-3
     assert stats.kstest(ur, "uniform").pvalue > 1e-3
     assert abs(np.corrcoef(ua, ur)[0, 1]) < 0.02
-    assert oracle.lib().rsd_oracle_rng_layout() == 1
+    assert oracle.lib().rsd_oracle_rng_layout() == 2
