@@ -20,8 +20,10 @@ constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kQueueCap = 64;  // per-warp candidate queue (a push adds at most 32 to at most 31 pending)
 constexpr int kMaxRows = 256;
 constexpr int kIdxNone = 0x7FFFFFFF;
-constexpr int kCandCap = 1024;          // candidate groups queued per row (more are handled in place)
-constexpr int kSurvCap = 512;           // elements whose exact perturbed value reaches the bound
+constexpr int kCandCap = 512;           // candidate groups queued per row (more are handled in place)
+constexpr int kTaskCap = 512;           // elements of candidate groups that may reach the bound
+constexpr int kFinCap = 256;            // elements that pass the cheap noise test
+constexpr int kSurvCap = 256;           // elements whose exact perturbed value reaches the bound
 
 struct ScanArgs {
     const void* data;
@@ -225,6 +227,10 @@ template <typename T, bool ALIGNED, bool NEED_LSE>
 __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanArgs a) {
     extern __shared__ float ub[];                    // [n_groups] upper bound of each group's perturbed values
     __shared__ int cand[kCandCap];                   // groups whose bound reaches tau
+    __shared__ uint32_t tk_x[kTaskCap];              // element index | (it carries the group's largest noise) << 31
+    __shared__ float tk_base[kTaskCap];              // lower bound of t(U_M) / 16 of the element's group
+    __shared__ uint32_t fin_x[kFinCap], fin_w[kFinCap];  // element (same encoding) and its fine-stream word
+    __shared__ int n_task, n_fin;
     __shared__ float sv_val[kSurvCap], sv_raw[kSurvCap];
     __shared__ int sv_idx[kSurvCap];
     __shared__ uint32_t bin_max[32];                 // per lane index: largest sample over the warps (ordered encoding)
@@ -242,7 +248,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     const int n_iter = (n_groups + kScanThreads - 1) / kScanThreads;
     const PhiloxRow pr = philox_row_setup(a, (node & 0x0FFFFFFFu) | (kTagGumbelCoarse << 28), key.seq, key.step);
 
-    if (tid == 0) { n_cand = 0; n_surv = 0; nan_flag = 0; }
+    if (tid == 0) { n_cand = 0; n_surv = 0; nan_flag = 0; n_task = 0; n_fin = 0; }
     if (tid < 32) bin_max[tid] = float_to_ordered(kNegInf);
     __syncthreads();
 
@@ -307,6 +313,11 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
         if (lane == 0) red_f[warp] = wm;
     }
     __syncthreads();
+    float lse_M = kNegInf;
+    if (NEED_LSE) {
+#pragma unroll
+        for (int w = 0; w < kScanWarps; ++w) lse_M = fmaxf(lse_M, red_f[w]);
+    }
     float tau;
     {
         float v = ordered_to_float(bin_max[lane]);  // bitonic sort across the warp, ascending
@@ -370,8 +381,93 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
         }
     };
 
-    int ns = 0;
-    for (int attempt = 0; attempt < 16; ++attempt) {
+    // ---- short path: three stages of independent items, one item per thread ------------------------------------------
+    // A: per candidate group, the elements whose value plus the group's largest noise can reach tau;
+    // B: per such element, its fine-stream word and a cheap test of  t(U_M)/16 + t(U_x) <= exp(value - tau);
+    // C: exact perturbed value of what is left.  Any overflow falls through to the general path below.
+    bool general = n_queued > kCandCap;
+    if (!general) {
+        for (int i = tid; i < n_queued; i += kScanThreads) {
+            const int g = cand[i];
+            Packed<T> grp;
+            grp.load(row, g, V, ALIGNED && (g + 1) * 16 <= V);
+            const uint4 cw = philox_row(a, pr, (uint32_t)g);
+            const float u = fmaf((float)cw.x, 2.3283064365386963e-10f, 1.1641532182693481e-10f);
+            const float t_hat = -__logf(u);
+            const float base_lo = fmaxf(t_hat - fmaf(t_hat, 1e-6f, 2.5e-7f), 0.0f) * 0.0625f;
+            const float need = tau + __logf(fmaxf(base_lo, 1e-37f)) - 2e-4f;   // tau - (upper bound of G_max)
+            const uint32_t apos = cw.y & 15u;
+            float v[16];
+            grp.unpack(v);
+            uint32_t todo = 0;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                if (v[j] != v[j]) saw_nan = true;
+                else if (v[j] > kNegInf && v[j] >= need) todo |= 1u << j;
+            }
+            while (todo) {
+                const uint32_t j = (uint32_t)__ffs(todo) - 1u;
+                todo &= todo - 1;
+                const int slot = atomicAdd(&n_task, 1);
+                if (slot < kTaskCap) {
+                    tk_x[slot] = (uint32_t)(g * 16) + j + (j == apos ? 0x80000000u : 0u);
+                    tk_base[slot] = base_lo;
+                }
+            }
+        }
+        __syncthreads();
+        const int nt = n_task;
+        general = nt > kTaskCap;
+        if (!general) {
+            for (int i = tid; i < nt; i += kScanThreads) {
+                const uint32_t xe = tk_x[i];
+                const uint32_t x = xe & 0x7FFFFFFFu;
+                uint32_t w = 0;
+                bool keep = true;
+                if (!(xe & 0x80000000u)) {
+                    w = fine_word(key, node, x);
+                    const float raw = RowIO<T>::scalar(row, (int)x);
+                    const float uu = fmaf((float)w, 2.3283064365386963e-10f, 1.1641532182693481e-10f);
+                    const float t_hat = -__logf(uu);
+                    const float t_lo = fmaxf(t_hat - fmaf(t_hat, 1e-6f, 2.5e-7f), 0.0f);
+                    const float y_hi = __expf(raw - tau) * 1.0002f;   // upper bound of exp(value - tau)
+                    keep = tk_base[i] + t_lo <= y_hi;
+                }
+                if (keep) {
+                    const int slot = atomicAdd(&n_fin, 1);
+                    if (slot < kFinCap) { fin_x[slot] = xe; fin_w[slot] = w; }
+                }
+            }
+            __syncthreads();
+            const int nf = n_fin;
+            general = nf > kFinCap;
+            if (!general) {
+                for (int i = tid; i < nf; i += kScanThreads) {
+                    const uint32_t xe = fin_x[i];
+                    const int x = (int)(xe & 0x7FFFFFFFu);
+                    const uint4 cw = philox_row(a, pr, (uint32_t)x >> 4);
+                    const float base = neg_log_uniform_f32(cw.x) * 0.0625f;
+                    const float raw = RowIO<T>::scalar(row, x);
+                    const float t_x = (xe & 0x80000000u) ? 0.0f : neg_log_uniform_f32(fin_w[i]);
+                    const float pert = raw - logf(base + t_x);
+                    if (pert >= tau) {
+                        const int sidx = atomicAdd(&n_surv, 1);
+                        if (sidx < kSurvCap) { sv_val[sidx] = pert; sv_idx[sidx] = x; sv_raw[sidx] = raw; }
+                    }
+                }
+                __syncthreads();
+                general = n_surv > kSurvCap;
+            }
+        }
+        if (general) {  // start over in the general path
+            __syncthreads();
+            if (tid == 0) n_surv = 0;
+            __syncthreads();
+        }
+    }
+
+    int ns = n_surv;
+    for (int attempt = 0; general && attempt < 16; ++attempt) {
         if (n_queued <= kCandCap) {
             for (int i = tid; i < n_queued; i += kScanThreads) process_group(cand[i]);
         } else {  // too many candidate groups for the queue: each thread handles its own
@@ -405,10 +501,8 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     if (ns > kSurvCap) ns = kSurvCap;
 
     float lse = 0.0f;
-    if (NEED_LSE) {  // the warps' maxima were published before the first barrier
-        float M = red_f[0];
-#pragma unroll
-        for (int w = 1; w < kScanWarps; ++w) M = fmaxf(M, red_f[w]);
+    if (NEED_LSE) {
+        const float M = lse_M;
         const float scaled = (lse_m > kNegInf) ? lse_s * ex2_approx((lse_m - M) * kLog2e) : 0.0f;
         const double S = block_sum<kScanThreads>((double)scaled, red_d);
         lse = (M > kNegInf && S > 0.0) ? (float)((double)M + log(S)) : kNegInf;
