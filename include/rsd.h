@@ -27,11 +27,14 @@
  *   - Randomness is a pure function of (seed, step, global sequence index, flat node id, stream tag, index), drawn
  *     from Philox4x32-10 (Salmon et al., SC'11): key = (seed low word, seed high word), counter = (index,
  *     node | tag << 28, sequence, step).  Global sequence index = seq_base + b, so a batch may be split over
- *     several GPUs without changing any result.  Streams (rsd_rng_layout() == 1):
- *       tag 0  Gumbel, coarse : index = x >> 4; output byte x & 15 (little-endian over the 4 words) is the top
- *                               byte of element x's 32 random bits
- *       tag 1  Gumbel, fine   : index = x >> 2; the upper 24 bits of output word x & 3 are the low 24 bits
- *              U = (bits + 1/2) / 2^32,  G = -ln(-ln U)
+ *     several GPUs without changing any result.  Streams (rsd_rng_layout() == 2), with t(w) = -ln((w + 1/2) / 2^32)
+ *     for a 32-bit word w:
+ *       tag 0  Gumbel, per group of 16 consecutive tokens : index = x >> 4; word 0 -> t_M, word 1 & 15 -> position a
+ *       tag 1  Gumbel, per token                          : index = x >> 2; word x & 3 -> t_x
+ *              G(x) = -ln( t_M / 16 + (x mod 16 != a ? t_x : 0) )
+ *              This draws the 16 noises of a group through the order statistics of 16 i.i.d. uniforms (largest
+ *              first, at a uniform position; the rest uniform below it), so they are i.i.d. standard Gumbel and
+ *              the group's largest noise is known from one generator call.
  *       tag 2  acceptance     : index = rank of the child among its siblings; U = (word0 >> 8) / 2^24
  *       tag 3  final token    : index = 0; u = (word0 + 1/2) / 2^32
  *     The same (seed, step, inputs) give bit-identical outputs whatever the launch shape.

@@ -69,7 +69,7 @@ void launch_scan_lse(const rsd_rows* rows, bool aligned, int blocks, const rsd::
 }
 
 void launch_scan(const rsd_rows* rows, bool need_lse, int blocks, rsd::ScanArgs& a, cudaStream_t s) {
-    const bool aligned = rows_aligned(rows);
+    const bool aligned = rows_aligned(rows) && a.V % 16 == 0;  // vector path: aligned rows made of whole groups
     for (int r = 0; r < 10; ++r) {
         a.rk0[r] = a.seed_lo + (uint32_t)r * 0x9E3779B9u;
         a.rk1[r] = a.seed_hi + (uint32_t)r * 0xBB67AE85u;

@@ -256,52 +256,58 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     float best = kNegInf;                  // largest exact sample of this thread (value(a) + lower bound of G_max)
     float lse_m = kNegInf, lse_s = 0.0f;   // running log-sum-exp of this thread's elements
     bool saw_nan = false;
-    Packed<T> nxt;
-    if (tid < n_groups) nxt.load(row, tid, V, ALIGNED && (tid + 1) * 16 <= V);
-    else nxt.fill_neg_inf();
-    for (int it = 0; it < n_iter; ++it) {
-        const int g = it * kScanThreads + tid;
-        const Packed<T> cur = nxt;
-        if (it + 1 < n_iter) {
-            const int g2 = g + kScanThreads;
-            if (g2 < n_groups) nxt.load(row, g2, V, ALIGNED && (g2 + 1) * 16 <= V);
-            else nxt.fill_neg_inf();
-        }
-        if (g < n_groups) {
-            const uint4 cw = philox_row(a, pr, (uint32_t)g);
-            float g_lo, g_hi;
-            group_noise_bounds(cw.x, g_lo, g_hi);
-            float gmax = group_max_nan(cur);
-            ub[g] = gmax + g_hi;                                   // NaN if the group holds a NaN: looked at later
-            best = fmaxf(best, group_element(cur, (int)(cw.y & 15u)) + g_lo);  // fmaxf drops NaN
-            if (NEED_LSE) {
-                float v[16];
-                cur.unpack(v);
-                if (gmax != gmax) {  // NaN counts as -inf
-                    gmax = kNegInf;
+    // work on one group whose 16 values are in `cur`
+    auto body = [&](const Packed<T>& cur, int g) {
+        const uint4 cw = philox_row(a, pr, (uint32_t)g);
+        float g_lo, g_hi;
+        group_noise_bounds(cw.x, g_lo, g_hi);
+        float gmax = group_max_nan(cur);
+        ub[g] = gmax + g_hi;                                   // NaN if the group holds a NaN: looked at later
+        best = fmaxf(best, group_element(cur, (int)(cw.y & 15u)) + g_lo);  // fmaxf drops NaN
+        if (NEED_LSE) {
+            float v[16];
+            cur.unpack(v);
+            if (gmax != gmax) {  // NaN counts as -inf
+                gmax = kNegInf;
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        if (v[j] != v[j]) v[j] = kNegInf;
-                        gmax = fmaxf(gmax, v[j]);
-                    }
-                }
-                if (gmax > lse_m) {  // rescale the running sum to the new reference
-                    lse_s *= ex2_approx((lse_m - gmax) * kLog2e);  // lse_m = -inf gives 0
-                    lse_m = gmax;
-                }
-                if (lse_m > kNegInf) {
-                    const float c = lse_m * kLog2e;
-                    float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-                    for (int j = 0; j < 16; j += 2) {
-                        s0 += ex2_approx(fmaf(v[j], kLog2e, -c));
-                        s1 += ex2_approx(fmaf(v[j + 1], kLog2e, -c));
-                    }
-                    lse_s += s0 + s1;
+                for (int j = 0; j < 16; ++j) {
+                    if (v[j] != v[j]) v[j] = kNegInf;
+                    gmax = fmaxf(gmax, v[j]);
                 }
             }
+            if (gmax > lse_m) {  // rescale the running sum to the new reference
+                lse_s *= ex2_approx((lse_m - gmax) * kLog2e);  // lse_m = -inf gives 0
+                lse_m = gmax;
+            }
+            // lse_m = -inf (nothing finite yet): every term is exp2(NaN or -inf), so skip
+            if (lse_m > kNegInf) {
+                const float c = lse_m * kLog2e;
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                    s0 += ex2_approx(fmaf(v[j], kLog2e, -c));
+                    s1 += ex2_approx(fmaf(v[j + 1], kLog2e, -c));
+                }
+                lse_s += s0 + s1;
+            }
         }
+    };
+    // Sweeps in which every thread has a group run without bounds checks, two per turn on alternating buffers
+    // (loads are issued one sweep ahead); the ragged last sweep is fetched first and handled last.
+    const int n_full = n_groups / kScanThreads;
+    const int g_last = n_full * kScanThreads + tid;
+    Packed<T> last, buf_a, buf_b;
+    if (g_last < n_groups) last.load(row, g_last, V, ALIGNED && (g_last + 1) * 16 <= V);
+    if (n_full > 0) buf_a.load(row, tid, V, ALIGNED);
+    int it = 0;
+    for (; it + 1 < n_full; it += 2) {
+        buf_b.load(row, (it + 1) * kScanThreads + tid, V, ALIGNED);
+        body(buf_a, it * kScanThreads + tid);
+        if (it + 2 < n_full) buf_a.load(row, (it + 2) * kScanThreads + tid, V, ALIGNED);
+        body(buf_b, (it + 1) * kScanThreads + tid);
     }
+    if (it < n_full) body(buf_a, it * kScanThreads + tid);
+    if (g_last < n_groups) body(last, g_last);
 
     // ---- tau: a lower bound of the k-th largest perturbed value from the threads' samples -------------------------
     // The samples belong to distinct elements.  They are folded into 32 bins (one per lane index, maximum over the
