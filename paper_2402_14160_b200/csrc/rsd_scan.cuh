@@ -44,6 +44,26 @@ struct ScanArgs {
     int32_t child_base[kMaxRows];
 };
 
+// Packed pairs of fp32 (sm_100 executes fma/add on two floats per instruction).
+__device__ __forceinline__ unsigned long long f32x2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ unsigned long long add_f32x2(unsigned long long a, unsigned long long b) {
+    unsigned long long r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ void split_f32x2(unsigned long long v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+
 // Coarse Gumbel stream of one row: counter words 1..3 and the key are fixed, only word 0 (the group index)
 // varies, so the parts of the first two rounds that do not depend on it are computed once per block.
 struct PhiloxRow {
@@ -282,12 +302,16 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
             // lse_m = -inf (nothing finite yet): every term is exp2(NaN or -inf), so skip
             if (lse_m > kNegInf) {
                 const float c = lse_m * kLog2e;
-                float s0 = 0.f, s1 = 0.f;
+                const unsigned long long l2 = f32x2(kLog2e, kLog2e), c2 = f32x2(-c, -c);
+                unsigned long long acc = f32x2(0.0f, 0.0f);
 #pragma unroll
-                for (int j = 0; j < 16; j += 2) {
-                    s0 += ex2_approx(fmaf(v[j], kLog2e, -c));
-                    s1 += ex2_approx(fmaf(v[j + 1], kLog2e, -c));
+                for (int j = 0; j < 16; j += 2) {  // two elements per fma / add
+                    float e0, e1;
+                    split_f32x2(fma_f32x2(f32x2(v[j], v[j + 1]), l2, c2), e0, e1);
+                    acc = add_f32x2(acc, f32x2(ex2_approx(e0), ex2_approx(e1)));
                 }
+                float s0, s1;
+                split_f32x2(acc, s0, s1);
                 lse_s += s0 + s1;
             }
         }
