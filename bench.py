@@ -26,6 +26,11 @@ if ROOT not in sys.path:
 
 import workloads  # noqa: E402
 
+# DRAM bytes moved per algorithmic byte by the scan kernel, from the ncu capture summarised in
+# profiles/scan_topk_kernel_workload5_256seq.md (dram__bytes_read + dram__bytes_write over rows x V x 2 bytes; the
+# traffic grows in proportion to the rows scanned).  Set to None whenever the kernel changes after a capture.
+SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.034
+
 METRIC = "verified tree nodes/sec"
 UNIT = "nodes/s"
 
@@ -279,7 +284,11 @@ def main():
     ver_gbs = ver_bytes / (ver_ms / K * 1e-3) / 1e9
     roofline = {"kernel": "scan_topk_kernel (Gumbel-Top-k / SBS parent-row scan)", "bound": "hbm",
                 "achieved": scan_gbs, "peak": peak, "unit": "GB/s", "frac": scan_gbs / peak, "peak_kind": peak_kind,
-                "traffic": None, "algorithmic_bytes_per_step": scan_bytes_per_step,
+                "traffic": (None if SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE is None else
+                            SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE * scan_bytes_per_step / n_scan),
+                "traffic_note": "DRAM bytes per scan launch (average over the step's launches), scaled by rows from a "
+                                "256-sequence ncu capture",
+                "algorithmic_bytes_per_step": scan_bytes_per_step,
                 "launches_per_step": n_scan, "avg_launch_ms": scan_ms / (K * n_scan),
                 "share_of_step": scan_ms / elapsed_ms,
                 "verify_walk": {"achieved": ver_gbs, "frac": ver_gbs / peak, "algorithmic_bytes_last_step": ver_bytes,
