@@ -13,7 +13,7 @@ from typing import Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "librsd.so")
+LIB_PATH = os.environ.get("RSD_LIB_PATH") or os.path.join(_HERE, "librsd.so")  # override: a variant build
 
 RSD_F32, RSD_BF16 = 0, 1
 ST_NAN_INPUT, ST_FEWER_THAN_K, ST_ZERO_RESIDUAL, ST_ZERO_DRAFT_PROB, ST_DRAFT_EXHAUSTED = 1, 2, 4, 8, 16

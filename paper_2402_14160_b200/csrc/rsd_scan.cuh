@@ -20,10 +20,16 @@ constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kQueueCap = 64;  // per-warp candidate queue (a push adds at most 32 to at most 31 pending)
 constexpr int kMaxRows = 256;
 constexpr int kIdxNone = 0x7FFFFFFF;
+// Queue sizes of the per-row stages.  Overflow of any of them is handled (general path, raised bound), so a build
+// with tiny sizes (-DRSD_SCAN_SMALL_QUEUES) gives the same results; the tests use one to exercise those paths.
+#ifdef RSD_SCAN_SMALL_QUEUES
+constexpr int kCandCap = 4, kTaskCap = 4, kFinCap = 2, kSurvCap = 40;
+#else
 constexpr int kCandCap = 512;           // candidate groups queued per row (more are handled in place)
 constexpr int kTaskCap = 512;           // elements of candidate groups that may reach the bound
 constexpr int kFinCap = 256;            // elements that pass the cheap noise test
-constexpr int kSurvCap = 256;           // elements whose exact perturbed value reaches the bound
+constexpr int kSurvCap = 256;           // elements whose exact perturbed value reaches the bound (>= RSD_MAX_K)
+#endif
 
 struct ScanArgs {
     const void* data;
