@@ -301,13 +301,13 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                     gmax = fmaxf(gmax, v[j]);
                 }
             }
-            if (gmax > lse_m) {  // rescale the running sum to the new reference
-                lse_s *= ex2_approx((lse_m - gmax) * kLog2e);  // lse_m = -inf gives 0
-                lse_m = gmax;
-            }
-            // lse_m = -inf (nothing finite yet): every term is exp2(NaN or -inf), so skip
-            if (lse_m > kNegInf) {
-                const float c = lse_m * kLog2e;
+            // branch-free online softmax: rescale by exp(old max - new max) (1 when the max does not grow; the
+            // running sum is 0 while the max is -inf), then add this group's exponentials
+            const float new_m = fmaxf(lse_m, gmax);
+            const float scale = (new_m > lse_m && lse_m > kNegInf) ? ex2_approx((lse_m - new_m) * kLog2e) : 1.0f;
+            lse_m = new_m;
+            {
+                const float c = (lse_m > kNegInf) ? lse_m * kLog2e : 0.0f;   // all -inf so far: terms are exp2(-inf) = 0
                 const unsigned long long l2 = f32x2(kLog2e, kLog2e), c2 = f32x2(-c, -c);
                 unsigned long long acc = f32x2(0.0f, 0.0f);
 #pragma unroll
@@ -318,7 +318,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                 }
                 float s0, s1;
                 split_f32x2(acc, s0, s1);
-                lse_s += s0 + s1;
+                lse_s = fmaf(lse_s, scale, s0 + s1);
             }
         }
     };
