@@ -29,7 +29,7 @@ import workloads  # noqa: E402
 # DRAM bytes moved per algorithmic byte by the scan kernel, from the ncu capture summarised in
 # profiles/scan_topk_kernel_workload5_256seq.md (dram__bytes_read + dram__bytes_write over rows x V x 2 bytes; the
 # traffic grows in proportion to the rows scanned).  Set to None whenever the kernel changes after a capture.
-SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.034
+SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.031
 
 METRIC = "verified tree nodes/sec"
 UNIT = "nodes/s"
@@ -290,6 +290,8 @@ def main():
                                 "256-sequence ncu capture",
                 "algorithmic_bytes_per_step": scan_bytes_per_step,
                 "launches_per_step": n_scan, "avg_launch_ms": scan_ms / (K * n_scan),
+                "launch_ms_by_level": [sum(scan_ev[s][l][0].elapsed_time(scan_ev[s][l][1]) for s in range(K)) / K
+                                       for l in range(n_scan)],
                 "share_of_step": scan_ms / elapsed_ms,
                 "verify_walk": {"achieved": ver_gbs, "frac": ver_gbs / peak, "algorithmic_bytes_last_step": ver_bytes,
                                 "avg_launch_ms": ver_ms / K, "share_of_step": ver_ms / elapsed_ms}}
