@@ -27,14 +27,15 @@
  *   - Randomness is a pure function of (seed, step, global sequence index, flat node id, stream tag, index), drawn
  *     from Philox4x32-10 (Salmon et al., SC'11): key = (seed low word, seed high word), counter = (index,
  *     node | tag << 28, sequence, step).  Global sequence index = seq_base + b, so a batch may be split over
- *     several GPUs without changing any result.  Streams (rsd_rng_layout() == 2), with t(w) = -ln((w + 1/2) / 2^32)
- *     for a 32-bit word w:
- *       tag 0  Gumbel, per group of 16 consecutive tokens : index = x >> 4; word 0 -> t_M, word 1 & 15 -> position a
- *       tag 1  Gumbel, per token                          : index = x >> 2; word x & 3 -> t_x
+ *     several GPUs without changing any result.  Streams (rsd_rng_layout() == 3), with t(u) = -ln u:
+ *       tag 0  Gumbel, one 32-bit word w per group g = x >> 4 of 16 consecutive tokens: word (g >> 5) & 3 of the
+ *              call with index = (g >> 7) * 32 + (g & 31) (one call serves four groups 32 apart);
+ *              t_M = t(((w >> 4) + 1/2) / 2^28), position a = w & 15
+ *       tag 1  Gumbel, per token: index = x >> 2, word w = word x & 3; t_x = t((w + 1/2) / 2^32)
  *              G(x) = -ln( t_M / 16 + (x mod 16 != a ? t_x : 0) )
  *              This draws the 16 noises of a group through the order statistics of 16 i.i.d. uniforms (largest
  *              first, at a uniform position; the rest uniform below it), so they are i.i.d. standard Gumbel and
- *              the group's largest noise is known from one generator call.
+ *              the group's largest noise is known from one word of the coarse stream.
  *       tag 2  acceptance     : index = rank of the child among its siblings; U = (word0 >> 8) / 2^24
  *       tag 3  final token    : index = 0; u = (word0 + 1/2) / 2^32
  *     The same (seed, step, inputs) give bit-identical outputs whatever the launch shape.

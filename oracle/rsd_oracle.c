@@ -92,15 +92,16 @@ static void draw(uint64_t seed, uint32_t step, uint32_t seq, uint32_t node, uint
     rsd_oracle_philox4x32_10(ctr, key, out);
 }
 
-int rsd_oracle_rng_layout(void) { return 2; }
+int rsd_oracle_rng_layout(void) { return 3; }
 
 /*
- * Gumbel noise of (sequence, node), RNG layout 2.  The noise of the V elements must be i.i.d. standard Gumbel
+ * Gumbel noise of (sequence, node), RNG layout 3.  The noise of the V elements must be i.i.d. standard Gumbel
  * (Eq. 6).  It is drawn group-wise, 16 consecutive elements per group, from the order statistics of 16 i.i.d.
  * uniforms: the largest of them is V^(1/16) for a uniform V, it sits at a uniformly random position a, and the
  * other 15 are i.i.d. uniform below it.  With t(U) = -ln U this reads
- *     coarse stream, index = group: word 0 -> U_M, word 1 (low 4 bits) -> a
- *     fine stream, index = x >> 2, word x & 3 -> U_x                  (32 bits each, U = (bits + 1/2) / 2^32)
+ *     coarse stream: one 32-bit word per group g = x >> 4, namely word (g >> 5) & 3 of the call with
+ *         index (g >> 7) * 32 + (g & 31); its upper 28 bits -> U_M = (bits + 1/2) / 2^28, its low 4 bits -> a
+ *     fine stream, index = x >> 2, word x & 3 -> U_x = (bits + 1/2) / 2^32
  *     G_x = -ln( t(U_M) / 16 + [x mod 16 != a] * t(U_x) ).
  * (max of 16 uniforms M = U_M^(1/16) has -ln M = t(U_M)/16; another element is M * U_x, so -ln of it is
  * t(U_M)/16 + t(U_x); G = -ln(-ln U).)  The element at position a carries the group's largest noise, which is
@@ -114,9 +115,11 @@ static double neg_log_uniform(uint32_t bits) {
 void rsd_oracle_gumbel_parts(uint64_t seed, uint32_t step, uint32_t seq, uint32_t node, uint32_t e,
                              double* t_group, int32_t* argmax_pos, double* t_elem) {
     uint32_t w[4];
-    draw(seed, step, seq, node, TAG_GUMBEL_COARSE, e >> 4, w);
-    *t_group = neg_log_uniform(w[0]);
-    *argmax_pos = (int32_t)(w[1] & 15u);
+    const uint32_t g = e >> 4;
+    draw(seed, step, seq, node, TAG_GUMBEL_COARSE, ((g >> 7) << 5) | (g & 31u), w);
+    const uint32_t word = w[(g >> 5) & 3u];
+    *t_group = -log(((double)(word >> 4) + 0.5) * (1.0 / 268435456.0));
+    *argmax_pos = (int32_t)(word & 15u);
     draw(seed, step, seq, node, TAG_GUMBEL_FINE, e >> 2, w);
     *t_elem = neg_log_uniform(w[e & 3u]);
 }

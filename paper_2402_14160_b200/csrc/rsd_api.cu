@@ -88,7 +88,7 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 extern "C" {
 
 int rsd_version(void) { return 100; }
-int rsd_rng_layout(void) { return 2; }
+int rsd_rng_layout(void) { return 3; }
 const char* rsd_last_error(void) { return g_err; }
 
 int rsd_profile_next_scan(void* before, void* after) {

@@ -42,12 +42,23 @@ __device__ __forceinline__ uint4 rng_draw(const RngKey& k, uint32_t node, uint32
     return philox4x32_10(index, (node & 0x0FFFFFFFu) | (tag << 28), k.seq, k.step, k.seed_lo, k.seed_hi);
 }
 
-// Gumbel noise, RNG layout 2: the 16 noises of a group of consecutive elements are drawn through the order
+// Gumbel noise, RNG layout 3: the 16 noises of a group of consecutive elements are drawn through the order
 // statistics of 16 i.i.d. uniforms.  With t(U) = -ln U,
-//     coarse stream (index = group):  word 0 -> U_M,  word 1 low 4 bits -> position a of the group's largest noise
-//     fine stream (index = x >> 2, word x & 3) -> U_x
+//     coarse stream: one 32-bit word per group; its upper 28 bits -> U_M = (bits + 1/2) / 2^28, its low 4 bits ->
+//         position a of the group's largest noise.  Group g reads word (g >> 5) & 3 of the call with index
+//         (g >> 7) * 32 + (g & 31): one call serves groups g, g + 32, g + 64, g + 96 of a block of 128 groups,
+//         i.e. the four groups a lane of a warp meets while the warp sweeps 2048 consecutive elements.
+//     fine stream (index = x >> 2, word x & 3) -> U_x = (bits + 1/2) / 2^32
 //     G_x = -ln( t(U_M) / 16 + [x mod 16 != a] t(U_x) ),
 // so the element at position a has the largest noise of its group, -ln(t(U_M) / 16), known from the coarse stream.
+__device__ __forceinline__ uint32_t coarse_index(uint32_t g) { return ((g >> 7) << 5) | (g & 31u); }
+__device__ __forceinline__ uint32_t coarse_select(const uint4& w, uint32_t g) {
+    const uint32_t sel = (g >> 5) & 3u;
+    return sel < 2 ? (sel == 0 ? w.x : w.y) : (sel == 2 ? w.z : w.w);
+}
+__device__ __forceinline__ uint32_t coarse_word(const RngKey& k, uint32_t node, uint32_t g) {
+    return coarse_select(rng_draw(k, node, kTagGumbelCoarse, coarse_index(g)), g);
+}
 __device__ __forceinline__ uint32_t fine_word(const RngKey& k, uint32_t node, uint32_t e) {
     const uint4 w = rng_draw(k, node, kTagGumbelFine, e >> 2);
     const uint32_t sel = e & 3u;
@@ -62,6 +73,15 @@ __device__ __forceinline__ float neg_log_uniform_f32(uint32_t bits) {
 }
 __device__ __forceinline__ double neg_log_uniform_f64(uint32_t bits) {
     return -log(((double)bits + 0.5) * (1.0 / 4294967296.0));
+}
+// the same for the group uniform: U_M = ((word >> 4) + 1/2) / 2^28
+__device__ __forceinline__ float neg_log_group_uniform_f32(uint32_t word) {
+    const uint32_t bits = word >> 4;
+    if (bits < 0x08000000u) return -logf(((float)bits + 0.5f) * 3.725290298461914e-09f);
+    return -log1pf(-(((float)(0x0FFFFFFFu - bits) + 0.5f) * 3.725290298461914e-09f));
+}
+__device__ __forceinline__ double neg_log_group_uniform_f64(uint32_t word) {
+    return -log(((double)(word >> 4) + 0.5) * (1.0 / 268435456.0));
 }
 
 // ---------------------------------------------------------------------------------------------------------

@@ -2,7 +2,8 @@
 // the per-sequence epilogue of a Stochastic Beam Search level (Eqs. 10-12, Algorithm 9).
 //
 // The noise of a group of 16 consecutive elements is drawn through its order statistics (see rsd_device.cuh): one
-// Philox call per group gives the group's largest noise and the element that carries it.  The streaming loop
+// word of a Philox call gives the group's largest noise and the element that carries it, and one call serves the
+// four groups a lane meets in a chunk of 128 groups.  The streaming loop
 // therefore needs, per group, only the largest value of the group: value_max + noise_max bounds every perturbed
 // value of the group from above, and value(a) + noise_max is the exact perturbed value of one element, i.e. a
 // sample from below.  The k-th largest of those samples is a true lower bound tau of the k-th largest perturbed
@@ -17,7 +18,6 @@ namespace rsd {
 
 constexpr int kScanThreads = 128;
 constexpr int kScanWarps = kScanThreads / 32;
-constexpr int kQueueCap = 64;  // per-warp candidate queue (a push adds at most 32 to at most 31 pending)
 constexpr int kMaxRows = 256;
 constexpr int kIdxNone = 0x7FFFFFFF;
 // Queue sizes of the per-row stages.  Overflow of any of them is handled (general path, raised bound), so a build
@@ -115,6 +115,22 @@ __device__ __forceinline__ uint4 philox_row(const ScanArgs& a, const PhiloxRow& 
     return make_uint4(y0, y1, y2, y3);
 }
 
+// Fine Gumbel stream word of element e, with the round keys taken from the kernel arguments.
+__device__ __forceinline__ uint32_t fine_word_rk(const ScanArgs& a, const RngKey& k, uint32_t node, uint32_t e) {
+    uint32_t c0 = e >> 2, c1 = (node & 0x0FFFFFFFu) | (kTagGumbelFine << 28), c2 = k.seq, c3 = k.step;
+#pragma unroll
+    for (int i = 0; i < 10; ++i) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ a.rk0[i];
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ a.rk1[i];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+    }
+    const uint32_t sel = e & 3u;
+    return sel < 2 ? (sel == 0 ? c0 : c1) : (sel == 2 ? c2 : c3);
+}
+
 __device__ __forceinline__ bool better(float v1, int i1, float v2, int i2) {
     return v1 > v2 || (v1 == v2 && i1 < i2);
 }
@@ -143,6 +159,10 @@ struct Packed<float> {
     __device__ __forceinline__ void fill_neg_inf() {
 #pragma unroll
         for (int i = 0; i < 4; ++i) w[i] = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
+    }
+    __device__ __forceinline__ void load_aligned(const void* group) {  // 64 bytes at a 16-byte aligned address
+#pragma unroll
+        for (int i = 0; i < 4; ++i) w[i] = ld_stream((const uint4*)group + i);
     }
     __device__ __forceinline__ void load(const void* row, int g, int V, bool aligned_full) {
         if (aligned_full) {
@@ -177,6 +197,10 @@ struct Packed<__nv_bfloat16> {
     }
     __device__ __forceinline__ void fill_neg_inf() {
         w[0] = w[1] = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+    }
+    __device__ __forceinline__ void load_aligned(const void* group) {  // 32 bytes at a 16-byte aligned address
+        w[0] = ld_stream((const uint4*)group);
+        w[1] = ld_stream((const uint4*)group + 1);
     }
     __device__ __forceinline__ void load(const void* row, int g, int V, bool aligned_full) {
         if (aligned_full) {
@@ -237,25 +261,72 @@ __device__ __forceinline__ float group_element(const Packed<__nv_bfloat16>& p, i
     return __uint_as_float((pos & 1) ? (w & 0xFFFF0000u) : (w << 16));
 }
 
-// Bounds of the group's largest noise G_max = -ln(t / 16), t = -ln((bits + 1/2) / 2^32), from fast logarithms:
-// lo <= G_max <= hi.  (|t_hat - t| <= 2.5e-7 + 1e-6 t covers the conversion and lg2.approx; the outer logarithm
-// adds at most 2e-6; hi is +huge when t_hat is too small to bound.)
+// Bounds of the group's largest noise G_max = -ln(t / 16), t = -ln((bits + 1/2) / 2^28), from two fast logarithms:
+// lo <= G_max <= hi.  With t_hat the fast value of t, |t_hat - t| <= 2.7e-7 + 3e-7 t (conversion, fma and lg2.approx
+// at 2^-22), so for t >= 2^-12 the relative error of t_hat / 16 is below 1.2e-3; the outer lg2.approx and the final
+// fma add less than 1e-5.  Below 2^-12 (one group in 4096) the bounds are -huge and +huge.
+constexpr float kNoiseMargin = 1.5e-3f;
+__device__ __forceinline__ float lg2_approx(float x) {
+    float r;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
 __device__ __forceinline__ void group_noise_bounds(uint32_t bits, float& lo, float& hi) {
-    const float u = fmaf((float)bits, 2.3283064365386963e-10f, 1.1641532182693481e-10f);
-    const float t_hat = -__logf(u);
-    const float dt = fmaf(t_hat, 1e-6f, 2.5e-7f);
-    hi = -__logf(fmaxf(t_hat - dt, 1e-37f) * 0.0625f) + 2e-4f;
-    lo = -__logf((t_hat + dt) * 0.0625f) - 2e-4f;
+    const float u = fmaf((float)bits, 3.725290298461914e-09f, 1.862645149230957e-09f);  // (bits + 1/2) / 2^28
+    const float ts = fmaf(lg2_approx(u), -0.04332169878499658f, 1e-30f);                // t / 16 (> 0), -ln2 / 16
+    const float margin = ts >= 1.52587890625e-05f ? kNoiseMargin : 1e30f;               // t / 16 >= 2^-16
+    const float l2 = lg2_approx(ts);
+    hi = fmaf(l2, -0.6931471805599453f, margin);
+    lo = fmaf(l2, -0.6931471805599453f, -margin);
+}
+
+// Shared-memory slot of one thread for the group it is working on: the 16 values as loaded, so that the one at a
+// position known only at run time can be read back with one load instead of a select tree.  The stride of 16 bytes
+// more than the data keeps the 16-byte stores of a quarter warp on distinct banks.
+template <typename T>
+struct GroupSlot {
+    static constexpr int kStride = (int)sizeof(Packed<T>) + 16;
+};
+__device__ __forceinline__ void slot_store(uint32_t addr, const Packed<float>& p) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr + 16u * i), "r"(p.w[i].x), "r"(p.w[i].y),
+                     "r"(p.w[i].z), "r"(p.w[i].w));
+}
+__device__ __forceinline__ void slot_store(uint32_t addr, const Packed<__nv_bfloat16>& p) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr + 16u * i), "r"(p.w[i].x), "r"(p.w[i].y),
+                     "r"(p.w[i].z), "r"(p.w[i].w));
+}
+template <typename T>
+__device__ __forceinline__ float slot_element(uint32_t addr, uint32_t pos);
+template <>
+__device__ __forceinline__ float slot_element<float>(uint32_t addr, uint32_t pos) {
+    float r;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(r) : "r"(addr + 4u * pos));
+    return r;
+}
+template <>
+__device__ __forceinline__ float slot_element<__nv_bfloat16>(uint32_t addr, uint32_t pos) {
+    uint32_t r;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(r) : "r"(addr + 2u * pos));
+    return __uint_as_float(r << 16);
 }
 
 // One block per row.
 template <typename T, bool ALIGNED, bool NEED_LSE>
 __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanArgs a) {
     extern __shared__ float ub[];                    // [n_groups] upper bound of each group's perturbed values
-    __shared__ int cand[kCandCap];                   // groups whose bound reaches tau
-    __shared__ uint32_t tk_x[kTaskCap];              // element index | (it carries the group's largest noise) << 31
-    __shared__ float tk_base[kTaskCap];              // lower bound of t(U_M) / 16 of the element's group
-    __shared__ uint32_t fin_x[kFinCap], fin_w[kFinCap];  // element (same encoding) and its fine-stream word
+    // One buffer, two uses: the threads' group slots during the streaming loop, the queues of the stages after it.
+    constexpr int kQueueBytes = 4 * (kCandCap + 2 * kTaskCap + 2 * kFinCap);
+    constexpr int kSlotBytes = kScanThreads * GroupSlot<T>::kStride;
+    __shared__ __align__(16) unsigned char shared_buf[kQueueBytes > kSlotBytes ? kQueueBytes : kSlotBytes];
+    int* const cand = (int*)shared_buf;                              // groups whose bound reaches tau
+    uint32_t* const tk_x = (uint32_t*)(cand + kCandCap);             // element index | (it carries the group's largest noise) << 31
+    float* const tk_base = (float*)(tk_x + kTaskCap);                // lower bound of t(U_M) / 16 of the element's group
+    uint32_t* const fin_x = (uint32_t*)(tk_base + kTaskCap);         // element (same encoding) ...
+    uint32_t* const fin_w = fin_x + kFinCap;                         // ... and its fine-stream word
     __shared__ int n_task, n_fin;
     __shared__ float sv_val[kSurvCap], sv_raw[kSurvCap];
     __shared__ int sv_idx[kSurvCap];
@@ -263,6 +334,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     __shared__ float red_f[kScanWarps];
     __shared__ double red_d[kScanWarps];
     __shared__ int n_cand, n_surv, nan_flag;
+    __shared__ float lse_sh;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / a.R, r = blockIdx.x % a.R;
@@ -278,81 +350,118 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     if (tid < 32) bin_max[tid] = float_to_ordered(kNegInf);
     __syncthreads();
 
-    // ---- streaming loop: one group per thread per sweep ------------------------------------------------------------
+    // ---- streaming loop ----------------------------------------------------------------------------------------------
+    // A warp takes chunks of 128 consecutive groups; lane l meets groups l, l + 32, l + 64, l + 96 of the chunk, whose
+    // coarse-stream words are the four words of one Philox call.
     float best = kNegInf;                  // largest exact sample of this thread (value(a) + lower bound of G_max)
-    float lse_m = kNegInf, lse_s = 0.0f;   // running log-sum-exp of this thread's elements
+    // Running log-sum-exp of this thread's elements: sum of 2^(value * log2(e) - c) with an integer c, fixed at the
+    // first finite group maximum and moved up only when a group maximum exceeds it by more than 40.
+    float lse_thr = kNegInf;               // group maxima above this move the reference (-inf: nothing finite yet)
+    float lse_negc = 0.0f;                 // -c
+    unsigned long long acc0 = f32x2(0.0f, 0.0f), acc1 = acc0;
     bool saw_nan = false;
-    // work on one group whose 16 values are in `cur`
-    auto body = [&](const Packed<T>& cur, int g) {
-        const uint4 cw = philox_row(a, pr, (uint32_t)g);
+    const uint32_t slot = (uint32_t)__cvta_generic_to_shared(shared_buf) + (uint32_t)tid * GroupSlot<T>::kStride;
+    // work on one group whose 16 values are in `cur`; `word` is the group's coarse-stream word, `ub_g` = &ub[group]
+    auto body = [&](const Packed<T>& cur, float* ub_g, uint32_t word) {
+        slot_store(slot, cur);
         float g_lo, g_hi;
-        group_noise_bounds(cw.x, g_lo, g_hi);
+        group_noise_bounds(word >> 4, g_lo, g_hi);
         float gmax = group_max_nan(cur);
-        ub[g] = gmax + g_hi;                                   // NaN if the group holds a NaN: looked at later
-        best = fmaxf(best, group_element(cur, (int)(cw.y & 15u)) + g_lo);  // fmaxf drops NaN
+        *ub_g = gmax + g_hi;                                   // NaN if the group holds a NaN: looked at later
+        best = fmaxf(best, slot_element<T>(slot, word & 15u) + g_lo);  // fmaxf drops NaN
         if (NEED_LSE) {
             float v[16];
             cur.unpack(v);
-            if (gmax != gmax) {  // NaN counts as -inf
-                gmax = kNegInf;
+            if (!(gmax <= lse_thr)) {  // rare: a NaN in the group, the first finite group, or a jump of more than 40
+                if (gmax != gmax) {    // NaN counts as -inf
+                    gmax = kNegInf;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    if (v[j] != v[j]) v[j] = kNegInf;
-                    gmax = fmaxf(gmax, v[j]);
+                    for (int j = 0; j < 16; ++j) {
+                        if (v[j] != v[j]) v[j] = kNegInf;
+                        gmax = fmaxf(gmax, v[j]);
+                    }
+                }
+                if (gmax > lse_thr) {
+                    const float c_new = ceilf(gmax * kLog2e);
+                    const float sc = lse_thr > kNegInf ? ex2_approx(-(lse_negc + c_new)) : 0.0f;  // 2^(c_old - c_new) <= 1
+                    float s0, s1, s2, s3;
+                    split_f32x2(acc0, s0, s1);
+                    split_f32x2(acc1, s2, s3);
+                    acc0 = f32x2(s0 * sc, s1 * sc);
+                    acc1 = f32x2(s2 * sc, s3 * sc);
+                    lse_negc = -c_new;
+                    lse_thr = gmax + 40.0f;
                 }
             }
-            // branch-free online softmax: rescale by exp(old max - new max) (1 when the max does not grow; the
-            // running sum is 0 while the max is -inf), then add this group's exponentials
-            const float new_m = fmaxf(lse_m, gmax);
-            const float scale = (new_m > lse_m && lse_m > kNegInf) ? ex2_approx((lse_m - new_m) * kLog2e) : 1.0f;
-            lse_m = new_m;
-            {
-                const float c = (lse_m > kNegInf) ? lse_m * kLog2e : 0.0f;   // all -inf so far: terms are exp2(-inf) = 0
-                const unsigned long long l2 = f32x2(kLog2e, kLog2e), c2 = f32x2(-c, -c);
-                unsigned long long acc = f32x2(0.0f, 0.0f);
+            const unsigned long long l2 = f32x2(kLog2e, kLog2e), c2 = f32x2(lse_negc, lse_negc);
 #pragma unroll
-                for (int j = 0; j < 16; j += 2) {  // two elements per fma / add
-                    float e0, e1;
-                    split_f32x2(fma_f32x2(f32x2(v[j], v[j + 1]), l2, c2), e0, e1);
-                    acc = add_f32x2(acc, f32x2(ex2_approx(e0), ex2_approx(e1)));
-                }
-                float s0, s1;
-                split_f32x2(acc, s0, s1);
-                lse_s = fmaf(lse_s, scale, s0 + s1);
+            for (int j = 0; j < 16; j += 4) {  // two elements per fma / add, two accumulators
+                float e0, e1, e2, e3;
+                split_f32x2(fma_f32x2(f32x2(v[j], v[j + 1]), l2, c2), e0, e1);
+                split_f32x2(fma_f32x2(f32x2(v[j + 2], v[j + 3]), l2, c2), e2, e3);
+                acc0 = add_f32x2(acc0, f32x2(ex2_approx(e0), ex2_approx(e1)));
+                acc1 = add_f32x2(acc1, f32x2(ex2_approx(e2), ex2_approx(e3)));
             }
         }
     };
-    // Sweeps in which every thread has a group run without bounds checks, two per turn on alternating buffers
-    // (loads are issued one sweep ahead); the ragged last sweep is fetched first and handled last.
-    const int n_full = n_groups / kScanThreads;
-    const int g_last = n_full * kScanThreads + tid;
-    Packed<T> last, buf_a, buf_b;
-    if (g_last < n_groups) last.load(row, g_last, V, ALIGNED && (g_last + 1) * 16 <= V);
-    if (n_full > 0) buf_a.load(row, tid, V, ALIGNED);
-    int it = 0;
-    for (; it + 1 < n_full; it += 2) {
-        buf_b.load(row, (it + 1) * kScanThreads + tid, V, ALIGNED);
-        body(buf_a, it * kScanThreads + tid);
-        if (it + 2 < n_full) buf_a.load(row, (it + 2) * kScanThreads + tid, V, ALIGNED);
-        body(buf_b, (it + 1) * kScanThreads + tid);
+    // Two buffers: the group two turns ahead is requested as soon as a buffer has been consumed.  Chunks that lie
+    // wholly inside the row run without bounds checks; the row's last, partial chunk runs the same steps guarded.
+    {
+        constexpr int kGroupBytes = 16 * RowIO<T>::kBytes;
+        const int n_full = n_groups >> 7;                    // whole chunks
+        auto fetch = [&](Packed<T>& q, int g) {              // guarded
+            if (g < n_groups) q.load(row, g, V, ALIGNED);
+        };
+        auto fetch_at = [&](Packed<T>& q, const char* p, int g) {   // group g lies inside the row; p = its address
+            if (ALIGNED) q.load_aligned(p);
+            else q.load(row, g, V, false);
+        };
+        Packed<T> q0, q1;
+        int c = warp;
+        fetch(q0, c * 128 + lane);
+        fetch(q1, c * 128 + 32 + lane);
+        for (; c < n_full; c += kScanWarps) {
+            const int g0 = c * 128 + lane, gn = g0 + kScanWarps * 128;
+            const char* p = row + (size_t)g0 * kGroupBytes;
+            float* ub_g = ub + g0;
+            const uint4 cw = philox_row(a, pr, (uint32_t)(c * 32 + lane));
+            body(q0, ub_g, cw.x);
+            fetch_at(q0, p + 64 * kGroupBytes, g0 + 64);
+            body(q1, ub_g + 32, cw.y);
+            fetch_at(q1, p + 96 * kGroupBytes, g0 + 96);
+            body(q0, ub_g + 64, cw.z);
+            fetch(q0, gn);
+            body(q1, ub_g + 96, cw.w);
+            fetch(q1, gn + 32);
+        }
+        if (c == n_full && (n_groups & 127)) {   // this warp owns the partial chunk; q0 and q1 are on their way
+            const int g0 = c * 128 + lane;
+            float* ub_g = ub + g0;
+            const uint4 cw = philox_row(a, pr, (uint32_t)(c * 32 + lane));
+            if (g0 < n_groups) body(q0, ub_g, cw.x);
+            fetch(q0, g0 + 64);
+            if (g0 + 32 < n_groups) body(q1, ub_g + 32, cw.y);
+            fetch(q1, g0 + 96);
+            if (g0 + 64 < n_groups) body(q0, ub_g + 64, cw.z);
+            if (g0 + 96 < n_groups) body(q1, ub_g + 96, cw.w);
+        }
     }
-    if (it < n_full) body(buf_a, it * kScanThreads + tid);
-    if (g_last < n_groups) body(last, g_last);
 
     // ---- tau: a lower bound of the k-th largest perturbed value from the threads' samples -------------------------
     // The samples belong to distinct elements.  They are folded into 32 bins (one per lane index, maximum over the
     // warps); the k-th largest bin maximum is at most the k-th largest sample, hence at most the k-th largest
     // perturbed value of the row.  Every warp sorts the 32 bin maxima itself, so one barrier is enough.
     if (best > kNegInf) atomicMax(&bin_max[lane], float_to_ordered(best));
+    const float lse_c = lse_thr > kNegInf ? -lse_negc : kNegInf;  // this thread's reference exponent
     if (NEED_LSE) {
-        const float wm = warp_max(lse_m);
+        const float wm = warp_max(lse_c);
         if (lane == 0) red_f[warp] = wm;
     }
-    __syncthreads();
-    float lse_M = kNegInf;
+    __syncthreads();   // also: every thread is done with its group slot, the queues may take the buffer over
+    float lse_C = kNegInf;
     if (NEED_LSE) {
 #pragma unroll
-        for (int w = 0; w < kScanWarps; ++w) lse_M = fmaxf(lse_M, red_f[w]);
+        for (int w = 0; w < kScanWarps; ++w) lse_C = fmaxf(lse_C, red_f[w]);
     }
     float tau;
     {
@@ -370,13 +479,37 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     }
 
     // ---- candidate groups ---------------------------------------------------------------------------------------------
-    for (int it = 0; it < n_iter; ++it) {
-        const int g = it * kScanThreads + tid;
-        if (g < n_groups) {
-            const float u = ub[g];
-            if (u >= tau || u != u) {
-                const int slot = atomicAdd(&n_cand, 1);
-                if (slot < kCandCap) cand[slot] = g;
+    // (a NaN bound compares false: the group is kept)
+    if (n_iter <= 32) {
+        // one bit per sweep, then one queue reservation per warp
+        uint32_t mine = 0;
+        for (int it = 0; it < n_iter; ++it) {
+            const int g = it * kScanThreads + tid;
+            if (g < n_groups && !(ub[g] < tau)) mine |= 1u << it;
+        }
+        const int cnt = __popc(mine);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        int base = 0;
+        if (lane == 31) base = atomicAdd(&n_cand, incl);
+        base = __shfl_sync(0xFFFFFFFFu, base, 31);
+        int slot_c = base + incl - cnt;
+        while (mine) {
+            const int it = __ffs(mine) - 1;
+            mine &= mine - 1;
+            if (slot_c < kCandCap) cand[slot_c] = it * kScanThreads + tid;
+            ++slot_c;
+        }
+    } else {
+        for (int it = 0; it < n_iter; ++it) {
+            const int g = it * kScanThreads + tid;
+            if (g < n_groups && !(ub[g] < tau)) {
+                const int slot_c = atomicAdd(&n_cand, 1);
+                if (slot_c < kCandCap) cand[slot_c] = g;
             }
         }
     }
@@ -387,10 +520,10 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     auto process_group = [&](int g) {
         Packed<T> grp;
         grp.load(row, g, V, ALIGNED && (g + 1) * 16 <= V);
-        const uint4 cw = philox_row(a, pr, (uint32_t)g);
-        const float base = neg_log_uniform_f32(cw.x) * 0.0625f;   // t(U_M) / 16
+        const uint32_t word = coarse_select(philox_row(a, pr, coarse_index((uint32_t)g)), (uint32_t)g);
+        const float base = neg_log_group_uniform_f32(word) * 0.0625f;   // t(U_M) / 16
         const float g_max = -logf(base);
-        const int apos = (int)(cw.y & 15u);
+        const int apos = (int)(word & 15u);
         // elements whose value plus the group's largest noise reaches tau (NaN compares false both ways: flagged)
         uint32_t todo = 0;
         {
@@ -409,7 +542,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
             const int x = g * 16 + j;
             const float raw = group_element(grp, j);
             float pert = raw + g_max;
-            if (j != apos) pert = raw - logf(base + neg_log_uniform_f32(fine_word(key, node, (uint32_t)x)));
+            if (j != apos) pert = raw - logf(base + neg_log_uniform_f32(fine_word_rk(a, key, node, (uint32_t)x)));
             if (pert >= tau) {
                 const int sidx = atomicAdd(&n_surv, 1);
                 if (sidx < kSurvCap) { sv_val[sidx] = pert; sv_idx[sidx] = x; sv_raw[sidx] = raw; }
@@ -427,27 +560,30 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
             const int g = cand[i];
             Packed<T> grp;
             grp.load(row, g, V, ALIGNED && (g + 1) * 16 <= V);
-            const uint4 cw = philox_row(a, pr, (uint32_t)g);
-            const float u = fmaf((float)cw.x, 2.3283064365386963e-10f, 1.1641532182693481e-10f);
+            const uint32_t word = coarse_select(philox_row(a, pr, coarse_index((uint32_t)g)), (uint32_t)g);
+            const float u = fmaf((float)(word >> 4), 3.725290298461914e-09f, 1.862645149230957e-09f);
             const float t_hat = -__logf(u);
             const float base_lo = fmaxf(t_hat - fmaf(t_hat, 1e-6f, 2.5e-7f), 0.0f) * 0.0625f;
             const float need = tau + __logf(fmaxf(base_lo, 1e-37f)) - 2e-4f;   // tau - (upper bound of G_max)
-            const uint32_t apos = cw.y & 15u;
+            const uint32_t apos = word & 15u;
+            if (ub[g] != ub[g]) saw_nan = true;                  // the bound is NaN exactly when the group holds one
+            const float need_f = fmaxf(need, -3.4028234663852886e38f);   // finite: -inf and NaN never pass
             float v[16];
             grp.unpack(v);
             uint32_t todo = 0;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                if (v[j] != v[j]) saw_nan = true;
-                else if (v[j] > kNegInf && v[j] >= need) todo |= 1u << j;
-            }
-            while (todo) {
-                const uint32_t j = (uint32_t)__ffs(todo) - 1u;
-                todo &= todo - 1;
-                const int slot = atomicAdd(&n_task, 1);
-                if (slot < kTaskCap) {
-                    tk_x[slot] = (uint32_t)(g * 16) + j + (j == apos ? 0x80000000u : 0u);
-                    tk_base[slot] = base_lo;
+            for (int j = 0; j < 16; ++j)
+                if (v[j] >= need_f) todo |= 1u << j;
+            if (todo) {
+                int slot_t = atomicAdd(&n_task, __popc(todo));
+                while (todo) {
+                    const uint32_t j = (uint32_t)__ffs(todo) - 1u;
+                    todo &= todo - 1;
+                    if (slot_t < kTaskCap) {
+                        tk_x[slot_t] = (uint32_t)(g * 16) + j + (j == apos ? 0x80000000u : 0u);
+                        tk_base[slot_t] = base_lo;
+                    }
+                    ++slot_t;
                 }
             }
         }
@@ -461,7 +597,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                 uint32_t w = 0;
                 bool keep = true;
                 if (!(xe & 0x80000000u)) {
-                    w = fine_word(key, node, x);
+                    w = fine_word_rk(a, key, node, x);
                     const float raw = RowIO<T>::scalar(row, (int)x);
                     const float uu = fmaf((float)w, 2.3283064365386963e-10f, 1.1641532182693481e-10f);
                     const float t_hat = -__logf(uu);
@@ -481,8 +617,8 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                 for (int i = tid; i < nf; i += kScanThreads) {
                     const uint32_t xe = fin_x[i];
                     const int x = (int)(xe & 0x7FFFFFFFu);
-                    const uint4 cw = philox_row(a, pr, (uint32_t)x >> 4);
-                    const float base = neg_log_uniform_f32(cw.x) * 0.0625f;
+                    const uint32_t gx = (uint32_t)x >> 4;
+                    const float base = neg_log_group_uniform_f32(coarse_select(philox_row(a, pr, coarse_index(gx)), gx)) * 0.0625f;
                     const float raw = RowIO<T>::scalar(row, x);
                     const float t_x = (xe & 0x80000000u) ? 0.0f : neg_log_uniform_f32(fin_w[i]);
                     const float pert = raw - logf(base + t_x);
@@ -538,13 +674,20 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
 
     float lse = 0.0f;
     if (NEED_LSE) {
-        const float M = lse_M;
-        const float scaled = (lse_m > kNegInf) ? lse_s * ex2_approx((lse_m - M) * kLog2e) : 0.0f;
-        const double S = block_sum<kScanThreads>((double)scaled, red_d);
-        lse = (M > kNegInf && S > 0.0) ? (float)((double)M + log(S)) : kNegInf;
+        // sum over the threads of s_t * 2^(c_t - C), C the largest reference exponent: exact scaling, summed in double
+        float s0, s1, s2, s3;
+        split_f32x2(acc0, s0, s1);
+        split_f32x2(acc1, s2, s3);
+        const float C = lse_C, d = lse_c - C;   // d <= 0, an integer (or NaN / -inf when there is nothing to add)
+        double term = 0.0;
+        if (lse_c > kNegInf && d > -1000.0f) term = ldexp((double)((s0 + s1) + (s2 + s3)), (int)d);
+        if (C == -kNegInf) term = (double)(C - C);  // a +inf value: the sum is not a number
+        const double S = block_sum<kScanThreads>(term, red_d);
+        if (tid == 0) lse_sh = (C > kNegInf && (S > 0.0 || S != S)) ? (float)((double)C * 0.6931471805599453 + log(S)) : kNegInf;
     }
     if (saw_nan) nan_flag = 1;
     __syncthreads();
+    if (NEED_LSE) lse = lse_sh;
 
     // ---- rank the survivors, write the picks ----------------------------------------------------------------------------
     const int total = ns < k ? ns : k;
@@ -624,11 +767,11 @@ __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const Sb
             const double sigma = a.sum_in ? (double)a.sum_in[(int64_t)b * a.n_par + kpar] : 0.0;
             const double lse = a.is_logprob ? 0.0 : (double)a.fin_lse[(int64_t)b * a.n_par + kpar];
             const uint32_t node = (uint32_t)(a.first_parent_node + kpar);
-            const uint4 cw = rng_draw(key, node, kTagGumbelCoarse, (uint32_t)x >> 4);
-            const double t_elem = (((uint32_t)x & 15u) != (cw.y & 15u))
+            const uint32_t word = coarse_word(key, node, (uint32_t)x >> 4);
+            const double t_elem = (((uint32_t)x & 15u) != (word & 15u))
                                       ? neg_log_uniform_f64(fine_word(key, node, (uint32_t)x)) : 0.0;
             phi = sigma + ((double)a.fin_value[(int64_t)b * F + f] - lse);
-            pert = phi - log(neg_log_uniform_f64(cw.x) * 0.0625 + t_elem);
+            pert = phi - log(neg_log_group_uniform_f64(word) * 0.0625 + t_elem);
         }
         s_tok[f] = x;
         s_phi[f] = phi;

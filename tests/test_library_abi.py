@@ -18,7 +18,7 @@ def test_library_builds_and_exports_every_declared_symbol():
     assert declared == set(api.EXPORTS)
     for name in declared:
         assert hasattr(lib, name), name
-    assert lib.rsd_rng_layout() == 2
+    assert lib.rsd_rng_layout() == 3
     lib.rsd_sbs_workspace_bytes.restype = ctypes.c_size_t
     assert lib.rsd_sbs_workspace_bytes(4, 8, 8) >= 4 * 8 * 8 * 8 + 4 * 8 * 4
 

@@ -61,18 +61,24 @@ def test_philox_avalanche():
 
 
 def test_gumbel_stream_layout():
-    """Group uniform and position from the coarse stream (16 elements per call), element uniform from the fine one."""
+    """Group uniform (28 bits) and position (4 bits) from one word of the coarse stream, four groups 32 apart per
+    call; element uniform from the fine stream, four elements per call."""
     seed, step, seq, node = 0x1234567811223344, 5, 17, 9
     key = [seed & MASK, seed >> 32]
-    for e in [0, 1, 3, 4, 15, 16, 17, 31999, 50271]:
-        coarse = oracle.philox4x32_10([e >> 4, node | (0 << 28), seq, step], key)
+    for e in [0, 1, 3, 4, 15, 16, 17, 511, 512, 1023, 1535, 1536, 2047, 2048, 2049, 31999, 50271]:
+        g = e >> 4
+        coarse = oracle.philox4x32_10([(g >> 7) * 32 + (g & 31), node | (0 << 28), seq, step], key)
+        word = int(coarse[(g >> 5) & 3])
         fine = oracle.philox4x32_10([e >> 2, node | (1 << 28), seq, step], key)
         tg, a, te = oracle.gumbel_parts(seed, step, seq, node, e)
-        assert math.isclose(tg, -math.log((int(coarse[0]) + 0.5) / 2.0 ** 32), rel_tol=1e-14)
-        assert a == int(coarse[1]) & 15
+        assert math.isclose(tg, -math.log(((word >> 4) + 0.5) / 2.0 ** 28), rel_tol=1e-14)
+        assert a == word & 15
         assert math.isclose(te, -math.log((int(fine[e & 3]) + 0.5) / 2.0 ** 32), rel_tol=1e-14)
-        g = oracle.gumbel(seed, step, seq, node, e)
-        assert math.isclose(g, -math.log(tg / 16 + (te if (e & 15) != a else 0.0)), rel_tol=1e-13)
+        g_noise = oracle.gumbel(seed, step, seq, node, e)
+        assert math.isclose(g_noise, -math.log(tg / 16 + (te if (e & 15) != a else 0.0)), rel_tol=1e-13)
+    # every group of a row reads its own word: (call, word) pairs are distinct
+    pairs = {((g >> 7) * 32 + (g & 31), (g >> 5) & 3) for g in range(4096)}
+    assert len(pairs) == 4096
 
 
 def test_streams_are_keyed_by_every_coordinate():
@@ -129,4 +135,4 @@ def test_uniform_streams():
     assert stats.kstest(ua, "uniform").pvalue > 1e-3
     assert stats.kstest(ur, "uniform").pvalue > 1e-3
     assert abs(np.corrcoef(ua, ur)[0, 1]) < 0.02
-    assert oracle.lib().rsd_oracle_rng_layout() == 2
+    assert oracle.lib().rsd_oracle_rng_layout() == 3
