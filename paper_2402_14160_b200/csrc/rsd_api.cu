@@ -35,9 +35,9 @@ int check_rows(const char* name, const rsd_rows* r, int V, bool need_row_stride)
     return RSD_OK;
 }
 
-bool rows_aligned(const rsd_rows* r) {
+bool rows_aligned(const rsd_rows* r, int bytes = 16) {
     const int64_t eb = r->dtype == RSD_F32 ? 4 : 2;
-    return ((uintptr_t)r->data % 16 == 0) && ((r->seq_stride * eb) % 16 == 0) && ((r->row_stride * eb) % 16 == 0);
+    return ((uintptr_t)r->data % bytes == 0) && ((r->seq_stride * eb) % bytes == 0) && ((r->row_stride * eb) % bytes == 0);
 }
 
 int check_vocab(int V) {
@@ -45,31 +45,34 @@ int check_vocab(int V) {
     return RSD_OK;
 }
 
-template <typename T, bool ALIGNED, bool NEED_LSE>
+template <typename T, bool ALIGNED, bool WIDE, bool NEED_LSE>
 void launch_scan_one(int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
-    const size_t smem = sizeof(float) * (size_t)((a.V + 15) / 16);  // one bound per group of 16 elements
+    const size_t smem = sizeof(float) * (size_t)((((a.V + 15) / 16) + 3) / 4 * 4);  // one bound per group of 16 elements, padded to fours
     static bool raised = false;  // per instantiation: allow the largest vocabulary's dynamic shared memory
     if (!raised) {
-        cudaFuncSetAttribute(rsd::scan_topk_kernel<T, ALIGNED, NEED_LSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(rsd::scan_topk_kernel<T, ALIGNED, WIDE, NEED_LSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(sizeof(float) * (RSD_MAX_VOCAB / 16)));
         raised = true;
     }
-    rsd::scan_topk_kernel<T, ALIGNED, NEED_LSE><<<blocks, rsd::kScanThreads, smem, s>>>(a);
+    rsd::scan_topk_kernel<T, ALIGNED, WIDE, NEED_LSE><<<blocks, rsd::kScanThreads, smem, s>>>(a);
 }
 
 template <bool NEED_LSE>
-void launch_scan_lse(const rsd_rows* rows, bool aligned, int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
+void launch_scan_lse(const rsd_rows* rows, int align, int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
     if (rows->dtype == RSD_F32) {
-        if (aligned) launch_scan_one<float, true, NEED_LSE>(blocks, a, s);
-        else launch_scan_one<float, false, NEED_LSE>(blocks, a, s);
+        if (align == 32) launch_scan_one<float, true, true, NEED_LSE>(blocks, a, s);
+        else if (align == 16) launch_scan_one<float, true, false, NEED_LSE>(blocks, a, s);
+        else launch_scan_one<float, false, false, NEED_LSE>(blocks, a, s);
     } else {
-        if (aligned) launch_scan_one<__nv_bfloat16, true, NEED_LSE>(blocks, a, s);
-        else launch_scan_one<__nv_bfloat16, false, NEED_LSE>(blocks, a, s);
+        if (align == 32) launch_scan_one<__nv_bfloat16, true, true, NEED_LSE>(blocks, a, s);
+        else if (align == 16) launch_scan_one<__nv_bfloat16, true, false, NEED_LSE>(blocks, a, s);
+        else launch_scan_one<__nv_bfloat16, false, false, NEED_LSE>(blocks, a, s);
     }
 }
 
 void launch_scan(const rsd_rows* rows, bool need_lse, int blocks, rsd::ScanArgs& a, cudaStream_t s) {
-    const bool aligned = rows_aligned(rows) && a.V % 16 == 0;  // vector path: aligned rows made of whole groups
+    // vector paths: rows made of whole groups that start on 32- or 16-byte boundaries
+    const int aligned = a.V % 16 != 0 ? 0 : rows_aligned(rows, 32) ? 32 : rows_aligned(rows, 16) ? 16 : 0;
     for (int r = 0; r < 10; ++r) {
         a.rk0[r] = a.seed_lo + (uint32_t)r * 0x9E3779B9u;
         a.rk1[r] = a.seed_hi + (uint32_t)r * 0xBB67AE85u;

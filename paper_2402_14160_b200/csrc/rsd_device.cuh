@@ -101,6 +101,13 @@ __device__ __forceinline__ uint4 ld_stream(const void* p) {
     return v;
 }
 
+// 32 bytes at a 32-byte aligned address in one request (sm_100: 256-bit global loads)
+__device__ __forceinline__ void ld_stream_256(const void* p, uint4& lo, uint4& hi) {
+    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w), "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w)
+                 : "l"(p));
+}
+
 template <typename T>
 struct RowIO;
 

@@ -160,15 +160,18 @@ struct Packed<float> {
 #pragma unroll
         for (int i = 0; i < 4; ++i) w[i] = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
     }
-    __device__ __forceinline__ void load_aligned(const void* group) {  // 64 bytes at a 16-byte aligned address
+    __device__ __forceinline__ void load_aligned(const void* group, bool wide) {  // 64 bytes, 16- or 32-byte aligned
+        if (wide) {
+            ld_stream_256(group, w[0], w[1]);
+            ld_stream_256((const char*)group + 32, w[2], w[3]);
+        } else {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) w[i] = ld_stream((const uint4*)group + i);
+            for (int i = 0; i < 4; ++i) w[i] = ld_stream((const uint4*)group + i);
+        }
     }
-    __device__ __forceinline__ void load(const void* row, int g, int V, bool aligned_full) {
+    __device__ __forceinline__ void load(const void* row, int g, int V, bool aligned_full, bool wide = false) {
         if (aligned_full) {
-            const uint4* p = (const uint4*)((const float*)row + (size_t)g * 16);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) w[i] = ld_stream(p + i);
+            load_aligned((const float*)row + (size_t)g * 16, wide);
         } else {
             uint32_t u[16];
 #pragma unroll
@@ -198,15 +201,17 @@ struct Packed<__nv_bfloat16> {
     __device__ __forceinline__ void fill_neg_inf() {
         w[0] = w[1] = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
     }
-    __device__ __forceinline__ void load_aligned(const void* group) {  // 32 bytes at a 16-byte aligned address
-        w[0] = ld_stream((const uint4*)group);
-        w[1] = ld_stream((const uint4*)group + 1);
+    __device__ __forceinline__ void load_aligned(const void* group, bool wide) {  // 32 bytes, 16- or 32-byte aligned
+        if (wide) {
+            ld_stream_256(group, w[0], w[1]);
+        } else {
+            w[0] = ld_stream((const uint4*)group);
+            w[1] = ld_stream((const uint4*)group + 1);
+        }
     }
-    __device__ __forceinline__ void load(const void* row, int g, int V, bool aligned_full) {
+    __device__ __forceinline__ void load(const void* row, int g, int V, bool aligned_full, bool wide = false) {
         if (aligned_full) {
-            const uint4* p = (const uint4*)((const uint16_t*)row + (size_t)g * 16);
-            w[0] = ld_stream(p);
-            w[1] = ld_stream(p + 1);
+            load_aligned((const uint16_t*)row + (size_t)g * 16, wide);
         } else {
             uint32_t u[8];
 #pragma unroll
@@ -259,6 +264,32 @@ __device__ __forceinline__ float group_element(const Packed<__nv_bfloat16>& p, i
     const uint32_t a = pick_word(p.w[0], wi), b = pick_word(p.w[1], wi);
     const uint32_t w = (wi & 4) ? b : a;
     return __uint_as_float((pos & 1) ? (w & 0xFFFF0000u) : (w << 16));
+}
+
+// bit j set when element j of the group is >= need (need finite; NaN and -inf elements never pass)
+__device__ __forceinline__ uint32_t group_mask_ge(const Packed<float>& p, float need) {
+    float v[16];
+    p.unpack(v);
+    uint32_t m = 0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+        if (v[j] >= need) m |= 1u << j;
+    return m;
+}
+__device__ __forceinline__ uint32_t group_mask_ge(const Packed<__nv_bfloat16>& p, float need) {
+    // the values lie on the bf16 grid, so v >= need exactly when v >= need rounded up to that grid
+    uint16_t nb;
+    asm("cvt.rp.bf16.f32 %0, %1;" : "=h"(nb) : "f"(need));
+    const uint32_t need2 = (uint32_t)nb * 0x00010001u;
+    const uint32_t q[8] = {p.w[0].x, p.w[0].y, p.w[0].z, p.w[0].w, p.w[1].x, p.w[1].y, p.w[1].z, p.w[1].w};
+    uint32_t acc = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        uint32_t ge;   // 0xFFFF per half that passes
+        asm("set.ge.u32.bf16x2 %0, %1, %2;" : "=r"(ge) : "r"(q[i]), "r"(need2));
+        acc |= ge & ((1u << (2 * i)) | (1u << (2 * i + 17)));
+    }
+    return (acc | (acc >> 16)) & 0xFFFFu;
 }
 
 // Bounds of the group's largest noise G_max = -ln(t / 16), t = -ln((bits + 1/2) / 2^28), from two fast logarithms:
@@ -315,18 +346,22 @@ __device__ __forceinline__ float slot_element<__nv_bfloat16>(uint32_t addr, uint
 }
 
 // One block per row.
-template <typename T, bool ALIGNED, bool NEED_LSE>
+// ALIGNED: rows start on 16-byte boundaries and V is a multiple of 16 (vector loads); WIDE: 32-byte boundaries as well.
+template <typename T, bool ALIGNED, bool WIDE, bool NEED_LSE>
 __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanArgs a) {
     extern __shared__ float ub[];                    // [n_groups] upper bound of each group's perturbed values
     // One buffer, two uses: the threads' group slots during the streaming loop, the queues of the stages after it.
-    constexpr int kQueueBytes = 4 * (kCandCap + 2 * kTaskCap + 2 * kFinCap);
+    constexpr int kQueueBytes = 4 * (kCandCap + 3 * kTaskCap + 4 * kFinCap);
     constexpr int kSlotBytes = kScanThreads * GroupSlot<T>::kStride;
     __shared__ __align__(16) unsigned char shared_buf[kQueueBytes > kSlotBytes ? kQueueBytes : kSlotBytes];
     int* const cand = (int*)shared_buf;                              // groups whose bound reaches tau
     uint32_t* const tk_x = (uint32_t*)(cand + kCandCap);             // element index | (it carries the group's largest noise) << 31
     float* const tk_base = (float*)(tk_x + kTaskCap);                // lower bound of t(U_M) / 16 of the element's group
-    uint32_t* const fin_x = (uint32_t*)(tk_base + kTaskCap);         // element (same encoding) ...
-    uint32_t* const fin_w = fin_x + kFinCap;                         // ... and its fine-stream word
+    uint32_t* const tk_word = (uint32_t*)(tk_base + kTaskCap);       // coarse-stream word of its group
+    uint32_t* const fin_x = tk_word + kTaskCap;                      // element (same encoding as tk_x) ...
+    uint32_t* const fin_w = fin_x + kFinCap;                         // ... its fine-stream word,
+    float* const fin_raw = (float*)(fin_w + kFinCap);                // value
+    uint32_t* const fin_word = (uint32_t*)(fin_raw + kFinCap);       // and coarse-stream word
     __shared__ int n_task, n_fin;
     __shared__ float sv_val[kSurvCap], sv_raw[kSurvCap];
     __shared__ int sv_idx[kSurvCap];
@@ -348,6 +383,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
 
     if (tid == 0) { n_cand = 0; n_surv = 0; nan_flag = 0; n_task = 0; n_fin = 0; }
     if (tid < 32) bin_max[tid] = float_to_ordered(kNegInf);
+    if (tid < 4 && n_groups + tid < ((n_groups + 3) & ~3)) ub[n_groups + tid] = kNegInf;   // padding of the bounds
     __syncthreads();
 
     // ---- streaming loop ----------------------------------------------------------------------------------------------
@@ -359,7 +395,6 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     float lse_thr = kNegInf;               // group maxima above this move the reference (-inf: nothing finite yet)
     float lse_negc = 0.0f;                 // -c
     unsigned long long acc0 = f32x2(0.0f, 0.0f), acc1 = acc0;
-    bool saw_nan = false;
     const uint32_t slot = (uint32_t)__cvta_generic_to_shared(shared_buf) + (uint32_t)tid * GroupSlot<T>::kStride;
     // work on one group whose 16 values are in `cur`; `word` is the group's coarse-stream word, `ub_g` = &ub[group]
     auto body = [&](const Packed<T>& cur, float* ub_g, uint32_t word) {
@@ -410,10 +445,10 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
         constexpr int kGroupBytes = 16 * RowIO<T>::kBytes;
         const int n_full = n_groups >> 7;                    // whole chunks
         auto fetch = [&](Packed<T>& q, int g) {              // guarded
-            if (g < n_groups) q.load(row, g, V, ALIGNED);
+            if (g < n_groups) q.load(row, g, V, ALIGNED, WIDE);
         };
         auto fetch_at = [&](Packed<T>& q, const char* p, int g) {   // group g lies inside the row; p = its address
-            if (ALIGNED) q.load_aligned(p);
+            if (ALIGNED) q.load_aligned(p, WIDE);
             else q.load(row, g, V, false);
         };
         Packed<T> q0, q1;
@@ -452,40 +487,59 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     // warps); the k-th largest bin maximum is at most the k-th largest sample, hence at most the k-th largest
     // perturbed value of the row.  Every warp sorts the 32 bin maxima itself, so one barrier is enough.
     if (best > kNegInf) atomicMax(&bin_max[lane], float_to_ordered(best));
-    const float lse_c = lse_thr > kNegInf ? -lse_negc : kNegInf;  // this thread's reference exponent
     if (NEED_LSE) {
-        const float wm = warp_max(lse_c);
-        if (lane == 0) red_f[warp] = wm;
+        // the warp's share of the log-sum-exp: largest reference exponent C_w and sum of s_t * 2^(c_t - C_w) (exact
+        // scaling, summed in double); the last thread combines the warps' shares after the barrier
+        const float lse_c = lse_thr > kNegInf ? -lse_negc : kNegInf;  // this thread's reference exponent
+        const float cw_max = warp_max(lse_c);
+        float s0, s1, s2, s3;
+        split_f32x2(acc0, s0, s1);
+        split_f32x2(acc1, s2, s3);
+        const float d = lse_c - cw_max;   // <= 0, an integer (NaN or -inf when there is nothing to add)
+        double term = 0.0;
+        if (lse_c > kNegInf && d > -1000.0f) term = ldexp((double)((s0 + s1) + (s2 + s3)), (int)d);
+        if (cw_max == -kNegInf) term = (double)(cw_max - cw_max);  // a +inf value: the sum is not a number
+        term = warp_sum(term);
+        if (lane == 0) { red_f[warp] = cw_max; red_d[warp] = term; }
     }
     __syncthreads();   // also: every thread is done with its group slot, the queues may take the buffer over
-    float lse_C = kNegInf;
-    if (NEED_LSE) {
+    if (NEED_LSE && tid == kScanThreads - 1) {
+        float C = red_f[0];
 #pragma unroll
-        for (int w = 0; w < kScanWarps; ++w) lse_C = fmaxf(lse_C, red_f[w]);
+        for (int w = 1; w < kScanWarps; ++w) C = fmaxf(C, red_f[w]);
+        double S = 0.0;
+#pragma unroll
+        for (int w = 0; w < kScanWarps; ++w) {
+            const float d = red_f[w] - C;
+            if (red_f[w] > kNegInf && d > -1000.0f) S += ldexp(red_d[w], (int)d);
+            else if (d != d) S = (double)d;
+        }
+        lse_sh = (C > kNegInf && (S > 0.0 || S != S)) ? (float)((double)C * 0.6931471805599453 + log(S)) : kNegInf;
     }
     float tau;
     {
-        float v = ordered_to_float(bin_max[lane]);  // bitonic sort across the warp, ascending
-#pragma unroll
-        for (int k2 = 2; k2 <= 32; k2 <<= 1) {
-#pragma unroll
-            for (int j = k2 >> 1; j > 0; j >>= 1) {
-                const float other = __shfl_xor_sync(0xFFFFFFFFu, v, j);
-                const bool up = (lane & k2) == 0, lower = (lane & j) == 0;
-                v = (lower == up) ? fminf(v, other) : fmaxf(v, other);
-            }
+        // k-th largest of the 32 bin maxima: take the maximum k times, dropping it (and its equals, which can only
+        // lower the result: still a lower bound) after each turn
+        uint32_t v = bin_max[lane], top = 0;
+        for (int i = 0; i < k; ++i) {
+            top = __reduce_max_sync(0xFFFFFFFFu, v);
+            if (v == top) v = 0;
         }
-        tau = __shfl_sync(0xFFFFFFFFu, v, 32 - k);  // k-th largest (k <= 32)
+        tau = top ? ordered_to_float(top) : kNegInf;
     }
 
     // ---- candidate groups ---------------------------------------------------------------------------------------------
-    // (a NaN bound compares false: the group is kept)
-    if (n_iter <= 32) {
-        // one bit per sweep, then one queue reservation per warp
+    // (a NaN bound compares false: the group is kept; the bounds are padded with -inf to a multiple of four)
+    const int n_quads = (n_groups + 3) >> 2;
+    if (n_quads <= 8 * kScanThreads) {
+        // four bounds per load, one bit per group, then one queue reservation per warp
+        const float4* ub4 = (const float4*)ub;
         uint32_t mine = 0;
-        for (int it = 0; it < n_iter; ++it) {
-            const int g = it * kScanThreads + tid;
-            if (g < n_groups && !(ub[g] < tau)) mine |= 1u << it;
+        for (int sw = 0, q = tid; q < n_quads; ++sw, q += kScanThreads) {
+            const float4 u = ub4[q];
+            const uint32_t m = (!(u.x < tau) ? 1u : 0u) | (!(u.y < tau) ? 2u : 0u) | (!(u.z < tau) ? 4u : 0u) |
+                               (!(u.w < tau) ? 8u : 0u);
+            mine |= m << (4 * sw);
         }
         const int cnt = __popc(mine);
         int incl = cnt;
@@ -499,9 +553,9 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
         base = __shfl_sync(0xFFFFFFFFu, base, 31);
         int slot_c = base + incl - cnt;
         while (mine) {
-            const int it = __ffs(mine) - 1;
+            const int bit = __ffs(mine) - 1;
             mine &= mine - 1;
-            if (slot_c < kCandCap) cand[slot_c] = it * kScanThreads + tid;
+            if (slot_c < kCandCap) cand[slot_c] = (((bit >> 2) * kScanThreads + tid) << 2) + (bit & 3);
             ++slot_c;
         }
     } else {
@@ -519,7 +573,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     // exact perturbed values of the elements of group g that can reach tau
     auto process_group = [&](int g) {
         Packed<T> grp;
-        grp.load(row, g, V, ALIGNED && (g + 1) * 16 <= V);
+        grp.load(row, g, V, ALIGNED && (g + 1) * 16 <= V, WIDE);
         const uint32_t word = coarse_select(philox_row(a, pr, coarse_index((uint32_t)g)), (uint32_t)g);
         const float base = neg_log_group_uniform_f32(word) * 0.0625f;   // t(U_M) / 16
         const float g_max = -logf(base);
@@ -532,7 +586,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
             const float need = tau - g_max - 1e-5f;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-                if (v[j] != v[j]) saw_nan = true;
+                if (v[j] != v[j]) nan_flag = 1;
                 else if (v[j] > kNegInf && v[j] >= need) todo |= 1u << j;
             }
         }
@@ -559,21 +613,16 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
         for (int i = tid; i < n_queued; i += kScanThreads) {
             const int g = cand[i];
             Packed<T> grp;
-            grp.load(row, g, V, ALIGNED && (g + 1) * 16 <= V);
+            grp.load(row, g, V, ALIGNED && (g + 1) * 16 <= V, WIDE);
             const uint32_t word = coarse_select(philox_row(a, pr, coarse_index((uint32_t)g)), (uint32_t)g);
             const float u = fmaf((float)(word >> 4), 3.725290298461914e-09f, 1.862645149230957e-09f);
             const float t_hat = -__logf(u);
             const float base_lo = fmaxf(t_hat - fmaf(t_hat, 1e-6f, 2.5e-7f), 0.0f) * 0.0625f;
             const float need = tau + __logf(fmaxf(base_lo, 1e-37f)) - 2e-4f;   // tau - (upper bound of G_max)
             const uint32_t apos = word & 15u;
-            if (ub[g] != ub[g]) saw_nan = true;                  // the bound is NaN exactly when the group holds one
+            if (ub[g] != ub[g]) nan_flag = 1;                  // the bound is NaN exactly when the group holds one
             const float need_f = fmaxf(need, -3.4028234663852886e38f);   // finite: -inf and NaN never pass
-            float v[16];
-            grp.unpack(v);
-            uint32_t todo = 0;
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-                if (v[j] >= need_f) todo |= 1u << j;
+            uint32_t todo = group_mask_ge(grp, need_f);
             if (todo) {
                 int slot_t = atomicAdd(&n_task, __popc(todo));
                 while (todo) {
@@ -582,6 +631,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                     if (slot_t < kTaskCap) {
                         tk_x[slot_t] = (uint32_t)(g * 16) + j + (j == apos ? 0x80000000u : 0u);
                         tk_base[slot_t] = base_lo;
+                        tk_word[slot_t] = word;
                     }
                     ++slot_t;
                 }
@@ -596,9 +646,9 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                 const uint32_t x = xe & 0x7FFFFFFFu;
                 uint32_t w = 0;
                 bool keep = true;
+                const float raw = RowIO<T>::scalar(row, (int)x);   // an L2 hit, in flight during the Philox rounds below
                 if (!(xe & 0x80000000u)) {
                     w = fine_word_rk(a, key, node, x);
-                    const float raw = RowIO<T>::scalar(row, (int)x);
                     const float uu = fmaf((float)w, 2.3283064365386963e-10f, 1.1641532182693481e-10f);
                     const float t_hat = -__logf(uu);
                     const float t_lo = fmaxf(t_hat - fmaf(t_hat, 1e-6f, 2.5e-7f), 0.0f);
@@ -607,7 +657,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                 }
                 if (keep) {
                     const int slot = atomicAdd(&n_fin, 1);
-                    if (slot < kFinCap) { fin_x[slot] = xe; fin_w[slot] = w; }
+                    if (slot < kFinCap) { fin_x[slot] = xe; fin_w[slot] = w; fin_raw[slot] = raw; fin_word[slot] = tk_word[i]; }
                 }
             }
             __syncthreads();
@@ -617,9 +667,8 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                 for (int i = tid; i < nf; i += kScanThreads) {
                     const uint32_t xe = fin_x[i];
                     const int x = (int)(xe & 0x7FFFFFFFu);
-                    const uint32_t gx = (uint32_t)x >> 4;
-                    const float base = neg_log_group_uniform_f32(coarse_select(philox_row(a, pr, coarse_index(gx)), gx)) * 0.0625f;
-                    const float raw = RowIO<T>::scalar(row, x);
+                    const float base = neg_log_group_uniform_f32(fin_word[i]) * 0.0625f;
+                    const float raw = fin_raw[i];
                     const float t_x = (xe & 0x80000000u) ? 0.0f : neg_log_uniform_f32(fin_w[i]);
                     const float pert = raw - logf(base + t_x);
                     if (pert >= tau) {
@@ -672,22 +721,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     }
     if (ns > kSurvCap) ns = kSurvCap;
 
-    float lse = 0.0f;
-    if (NEED_LSE) {
-        // sum over the threads of s_t * 2^(c_t - C), C the largest reference exponent: exact scaling, summed in double
-        float s0, s1, s2, s3;
-        split_f32x2(acc0, s0, s1);
-        split_f32x2(acc1, s2, s3);
-        const float C = lse_C, d = lse_c - C;   // d <= 0, an integer (or NaN / -inf when there is nothing to add)
-        double term = 0.0;
-        if (lse_c > kNegInf && d > -1000.0f) term = ldexp((double)((s0 + s1) + (s2 + s3)), (int)d);
-        if (C == -kNegInf) term = (double)(C - C);  // a +inf value: the sum is not a number
-        const double S = block_sum<kScanThreads>(term, red_d);
-        if (tid == 0) lse_sh = (C > kNegInf && (S > 0.0 || S != S)) ? (float)((double)C * 0.6931471805599453 + log(S)) : kNegInf;
-    }
-    if (saw_nan) nan_flag = 1;
-    __syncthreads();
-    if (NEED_LSE) lse = lse_sh;
+    const float lse = NEED_LSE ? lse_sh : 0.0f;   // written before the barriers that end the stages above
 
     // ---- rank the survivors, write the picks ----------------------------------------------------------------------------
     const int total = ns < k ? ns : k;
