@@ -442,50 +442,46 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     // Two buffers: the group two turns ahead is requested as soon as a buffer has been consumed.  Chunks that lie
     // wholly inside the row run without bounds checks; the row's last, partial chunk runs the same steps guarded.
     {
-        constexpr int kGroupBytes = 16 * RowIO<T>::kBytes;
         const int n_full = n_groups >> 7;                    // whole chunks
         auto fetch = [&](Packed<T>& q, int g) {              // guarded
             if (g < n_groups) q.load(row, g, V, ALIGNED, WIDE);
-        };
-        auto fetch_at = [&](Packed<T>& q, const char* p, int g) {   // group g lies inside the row; p = its address
-            if (ALIGNED) q.load_aligned(p, WIDE);
-            else q.load(row, g, V, false);
         };
         Packed<T> q0, q1;
         int c = warp;
         fetch(q0, c * 128 + lane);
         fetch(q1, c * 128 + 32 + lane);
         for (; c < n_full; c += kScanWarps) {
-            const int g0 = c * 128 + lane, gn = g0 + kScanWarps * 128;
-            const char* p = row + (size_t)g0 * kGroupBytes;
+            const int g0 = c * 128 + lane;
             float* ub_g = ub + g0;
             const uint4 cw = philox_row(a, pr, (uint32_t)(c * 32 + lane));
-            body(q0, ub_g, cw.x);
-            fetch_at(q0, p + 64 * kGroupBytes, g0 + 64);
-            body(q1, ub_g + 32, cw.y);
-            fetch_at(q1, p + 96 * kGroupBytes, g0 + 96);
-            body(q0, ub_g + 64, cw.z);
-            fetch(q0, gn);
-            body(q1, ub_g + 96, cw.w);
-            fetch(q1, gn + 32);
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {   // two turns of two groups: keeps the loop's code small
+                const int g_next = h ? g0 + kScanWarps * 128 : g0 + 64;   // first turn: inside this chunk
+                body(q0, ub_g + 64 * h, h ? cw.z : cw.x);
+                fetch(q0, g_next);
+                body(q1, ub_g + 64 * h + 32, h ? cw.w : cw.y);
+                fetch(q1, g_next + 32);
+            }
         }
         if (c == n_full && (n_groups & 127)) {   // this warp owns the partial chunk; q0 and q1 are on their way
             const int g0 = c * 128 + lane;
             float* ub_g = ub + g0;
             const uint4 cw = philox_row(a, pr, (uint32_t)(c * 32 + lane));
-            if (g0 < n_groups) body(q0, ub_g, cw.x);
-            fetch(q0, g0 + 64);
-            if (g0 + 32 < n_groups) body(q1, ub_g + 32, cw.y);
-            fetch(q1, g0 + 96);
-            if (g0 + 64 < n_groups) body(q0, ub_g + 64, cw.z);
-            if (g0 + 96 < n_groups) body(q1, ub_g + 96, cw.w);
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+                const int g = g0 + 64 * h;
+                if (g < n_groups) body(q0, ub_g + 64 * h, h ? cw.z : cw.x);
+                if (h == 0) fetch(q0, g0 + 64);
+                if (g + 32 < n_groups) body(q1, ub_g + 64 * h + 32, h ? cw.w : cw.y);
+                if (h == 0) fetch(q1, g0 + 96);
+            }
         }
     }
 
     // ---- tau: a lower bound of the k-th largest perturbed value from the threads' samples -------------------------
     // The samples belong to distinct elements.  They are folded into 32 bins (one per lane index, maximum over the
     // warps); the k-th largest bin maximum is at most the k-th largest sample, hence at most the k-th largest
-    // perturbed value of the row.  Every warp sorts the 32 bin maxima itself, so one barrier is enough.
+    // perturbed value of the row.  Every warp finds it from the 32 bin maxima itself, so one barrier is enough.
     if (best > kNegInf) atomicMax(&bin_max[lane], float_to_ordered(best));
     if (NEED_LSE) {
         // the warp's share of the log-sum-exp: largest reference exponent C_w and sum of s_t * 2^(c_t - C_w) (exact
@@ -689,16 +685,14 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
 
     int ns = n_surv;
     for (int attempt = 0; general && attempt < 16; ++attempt) {
-        if (n_queued <= kCandCap) {
-            for (int i = tid; i < n_queued; i += kScanThreads) process_group(cand[i]);
-        } else {  // too many candidate groups for the queue: each thread handles its own
-            for (int it = 0; it < n_iter; ++it) {
-                const int g = it * kScanThreads + tid;
-                if (g < n_groups) {
-                    const float u = ub[g];
-                    if (u >= tau || u != u) process_group(g);
-                }
-            }
+        // the queued candidate groups, or (when they did not fit the queue) every group whose bound reaches tau
+        const bool queued = n_queued <= kCandCap;
+        const int n_items = queued ? n_queued : n_groups;
+        for (int i = tid; i < n_items; i += kScanThreads) {
+            int g = i;
+            if (queued) g = cand[i];
+            else if (ub[i] < tau) continue;
+            process_group(g);
         }
         __syncthreads();
         ns = n_surv;
