@@ -143,7 +143,7 @@ int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int3
 size_t rsd_sbs_workspace_bytes(int B, int n_par, int W) {
     if (B < 0 || n_par < 1 || W < 1) return 0;
     const size_t f = (size_t)B * n_par * W;
-    return align_up(f * 4, 256) * 2 + align_up((size_t)B * n_par * 4, 256);
+    return align_up(f * 4, 256) * 3 + align_up((size_t)B * n_par * 4, 256);
 }
 
 int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, int32_t first_parent_node,
@@ -174,7 +174,8 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     char* w = (char*)ws;
     int32_t* fin_token = (int32_t*)w;
     float* fin_value = (float*)(w + align_up(f * 4, 256));
-    float* fin_lse = (float*)(w + 2 * align_up(f * 4, 256));
+    float* fin_pert = (float*)(w + 2 * align_up(f * 4, 256));
+    float* fin_lse = (float*)(w + 3 * align_up(f * 4, 256));
 
     rsd::ScanArgs a;
     memset(&a, 0, sizeof(a));
@@ -183,7 +184,7 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     a.R = n_par; a.V = V; a.max_k = W;
     a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
     a.subtract_lse = 0;
-    a.out_token = fin_token; a.out_perturbed = nullptr; a.out_value = fin_value; a.out_lse = fin_lse;
+    a.out_token = fin_token; a.out_perturbed = fin_pert; a.out_value = fin_value; a.out_lse = fin_lse;
     a.status = status;
     launch_scan(draft_level, !draft_level->is_logprob, B * n_par, a, s);
     if (int e = check_launch("rsd_sbs_step(scan)")) return e;
@@ -191,12 +192,12 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     rsd::SbsEpilogueArgs e;
     e.n_par = n_par; e.W = W; e.is_logprob = draft_level->is_logprob; e.first_parent_node = first_parent_node;
     e.seed_lo = (uint32_t)seed; e.seed_hi = (uint32_t)(seed >> 32); e.step = step; e.seq_base = seq_base;
-    e.fin_token = fin_token; e.fin_value = fin_value; e.fin_lse = fin_lse;
+    e.fin_token = fin_token; e.fin_value = fin_value; e.fin_pert = fin_pert; e.fin_lse = fin_lse;
     e.sum_in = sum_logprob_in; e.gamma_in = trunc_gumbel_in;
     e.out_token = out_token; e.out_parent = out_parent; e.out_stride = out_stride; e.parent_base = parent_base;
     e.sum_out = sum_logprob_out; e.gamma_out = trunc_gumbel_out;
     e.out_count = out_count; e.status = status;
-    const size_t smem = (size_t)n_par * W * (8 + 8 + 4);
+    const size_t smem = (size_t)n_par * W * (8 + 8 + 4) + (size_t)n_par * 4;
     rsd::sbs_epilogue_kernel<<<B, rsd::kEpilogueThreads, smem, s>>>(e);
     return check_launch("rsd_sbs_step(epilogue)");
 }

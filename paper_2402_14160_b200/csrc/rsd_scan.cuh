@@ -762,6 +762,7 @@ struct SbsEpilogueArgs {
     uint32_t seed_lo, seed_hi, step, seq_base;
     const int32_t* fin_token;  // [B][n_par][W]
     const float* fin_value;    // [B][n_par][W] the row's own value at the finalist
+    const float* fin_pert;     // [B][n_par][W] value + noise in fp32 (decreasing within a parent)
     const float* fin_lse;      // [B][n_par]
     const float* sum_in;       // [B][n_par] or null
     const float* gamma_in;     // [B][n_par] or null
@@ -787,9 +788,50 @@ __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const Sb
     const RngKey key = {a.seed_lo, a.seed_hi, a.step, a.seq_base + (uint32_t)b};
     const double ninf = -__longlong_as_double(0x7FF0000000000000LL);
 
+    // A child enters the beam only if its psi reaches the W-th best psi of the level.  The best child of parent j has
+    // psi = Gamma_j exactly, so that bound is at least L = the W-th largest Gamma among the parents that deliver a
+    // child (valid parent, at least one finalist); L = -inf when fewer than W do.  Finalists that a cheap fp32 test
+    // shows to lie clearly below L are dropped before the double-precision work; a parent's best finalist is
+    // always kept (it defines Z).
+    float* s_gam = (float*)(s_tok + F);   // [n_par]
+    __shared__ float s_L;
+    if (tid == 0) s_L = kNegInf;
+    for (int kp = tid; kp < a.n_par; kp += kEpilogueThreads) {
+        const float sg = a.sum_in ? a.sum_in[(int64_t)b * a.n_par + kp] : 0.0f;
+        const float gm = a.gamma_in ? a.gamma_in[(int64_t)b * a.n_par + kp] : 0.0f;
+        const bool delivers = a.fin_token[(int64_t)b * F + (int64_t)kp * a.W] >= 0 && sg > kNegInf && gm > kNegInf;
+        s_gam[kp] = delivers ? gm : kNegInf;
+    }
+    __syncthreads();
+    for (int kp = tid; kp < a.n_par; kp += kEpilogueThreads) {
+        const float g = s_gam[kp];
+        int rank = 0;
+        for (int j = 0; j < a.n_par; ++j) {
+            const float o = s_gam[j];
+            rank += (o > g || (o == g && j < kp)) ? 1 : 0;
+        }
+        if (rank == a.W - 1 && g > kNegInf) s_L = g;
+    }
+    __syncthreads();
+    const float L = s_L;
+
     for (int f = tid; f < F; f += kEpilogueThreads) {
         const int kpar = f / a.W;
-        const int x = a.fin_token[(int64_t)b * F + f];
+        int x = a.fin_token[(int64_t)b * F + f];
+        if (x >= 0 && L > kNegInf && f != kpar * a.W) {
+            // psi_f < L  <=>  exp(-phi~_f) - exp(-Z) > exp(-L) - exp(-Gamma_k), with Z - phi~_f = the gap d between
+            // the parent's best and this finalist's fp32 perturbed values; margins cover the fp32 arithmetic
+            const float sg = a.sum_in ? a.sum_in[(int64_t)b * a.n_par + kpar] : 0.0f;
+            const float gm = a.gamma_in ? a.gamma_in[(int64_t)b * a.n_par + kpar] : 0.0f;
+            const float lse = a.is_logprob ? 0.0f : a.fin_lse[(int64_t)b * a.n_par + kpar];
+            const float u0 = a.fin_pert[(int64_t)b * F + (int64_t)kpar * a.W];
+            const float d_lo = (u0 - a.fin_pert[(int64_t)b * F + f]) - 1e-4f;
+            if (d_lo > 0.0f) {
+                const float z = sg - lse + u0;
+                const float rhs = expf(-L + 1e-3f) - expf(-gm);
+                if (rhs <= 0.0f || -z + logf(expm1f(d_lo)) > logf(rhs) + 1e-2f) x = -1;   // cannot reach the beam
+            }
+        }
         double phi = ninf, pert = ninf;
         if (x >= 0) {
             const double sigma = a.sum_in ? (double)a.sum_in[(int64_t)b * a.n_par + kpar] : 0.0;

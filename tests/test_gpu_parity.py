@@ -173,6 +173,36 @@ def test_sbs_drops_minus_infinity_candidates(rsd):
     assert close(g["trunc_gumbel"][0, :3], o["trunc_gumbel"][0, :3]).all()
 
 
+@pytest.mark.parametrize("dtype,V,W,L,sigma", [("f32", 200, 8, 5, 3.5), ("bf16", 4099, 8, 4, 4.5), ("f32", 64, 4, 6, 3.0)])
+def test_sbs_peaked_rows_branch_inside_a_parent(rsd, dtype, V, W, L, sigma):
+    # peaked next-token distributions: several children of one parent enter the beam and other parents drop out, so
+    # the epilogue's early rejection of finalists (psi below the W-th largest Gamma) has to keep exactly the right ones
+    B = 16
+    draft = _rows((B, 1 + (L - 1) * W, V), dtype, sigma, 900 + V)
+    t, g_levels, o_levels, _ = _sbs_chain(rsd, draft, W, L, seed=5, step=1, is_logprob=False)
+    t.check()
+    parents = np.concatenate([o["parent"] for o in o_levels[1:]])
+    counts = [len(set(row.tolist())) for row in parents]
+    assert min(counts) < W and np.mean(counts) < W - 0.25      # parents really are shared and dropped
+
+
+def test_sbs_parent_with_a_fully_masked_row(rsd):
+    # W valid parents, one of which has no selectable child: only W - 1 parents deliver their best child, so second
+    # and third children of the others must still be found
+    W, V = 4, 96
+    rows = _rows((3, W, V), "f32", 2.0, 77)
+    rows[:, 2, :] = float("-inf")
+    sig = _rows((3, W), "f32", 1.0, 78) - 3.0
+    gam = _rows((3, W), "f32", 1.0, 79)
+    g = _np(rsd.rsd_sbs_step(rows, W, 1, sig, gam, 11, 0))
+    o = oracle.sbs_step(workloads.as_oracle_rows(rows), W, 1, sig.cpu().numpy().astype(np.float64),
+                        gam.cpu().numpy().astype(np.float64), 11, 0)
+    t = Tally()
+    compare_sbs_level(t, g, o, W, set())
+    t.check()
+    assert np.all(g["count"] == W) and not np.any(g["parent"] == 2)
+
+
 # ---------------------------------------------------------------------------------------------------------
 # verification
 # ---------------------------------------------------------------------------------------------------------
