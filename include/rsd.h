@@ -157,7 +157,7 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
  * device image, which every GPU that loads the library holds until the process exits.  The call itself allocates
  * and frees nothing.
  *   - Sizes: rsd_sbs_workspace_bytes(B, n_par, W) must not exceed RSD_SBS_STATIC_SCRATCH_BYTES (for example
- *     B = 1024, n_par = 8, W = 8 needs 819,200 bytes); larger calls return RSD_ERR_WORKSPACE with a message.
+ *     B = 1024, n_par = 8, W = 8 needs 851,968 bytes); larger calls return RSD_ERR_WORKSPACE with a message.
  *   - The first call on each device looks up the array's device address (with that device current) and keeps it;
  *     make that first call outside any stream capture.
  *   - All calls on a device share the one array.  Nothing in it has to start at zero (every entry is written before

@@ -143,7 +143,7 @@ int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int3
 size_t rsd_sbs_workspace_bytes(int B, int n_par, int W) {
     if (B < 0 || n_par < 1 || W < 1) return 0;
     const size_t f = (size_t)B * n_par * W;
-    return align_up(f * 4, 256) * 3 + align_up((size_t)B * n_par * 4, 256);
+    return align_up(f * 4, 256) * 3 + align_up((size_t)B * n_par * 4, 256) * 2;
 }
 
 int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, int32_t first_parent_node,
@@ -168,7 +168,6 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     if (!ws || ws_bytes < need) return fail(RSD_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
     if ((uintptr_t)ws % 256 != 0) return fail(RSD_ERR_WORKSPACE, "workspace must be 256-byte aligned");
     cudaStream_t s = (cudaStream_t)stream;
-    if (cudaMemsetAsync(status, 0, sizeof(int32_t) * (size_t)B, s) != cudaSuccess) return check_launch("memset(status)");
 
     const size_t f = (size_t)B * n_par * W;
     char* w = (char*)ws;
@@ -176,6 +175,7 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     float* fin_value = (float*)(w + align_up(f * 4, 256));
     float* fin_pert = (float*)(w + 2 * align_up(f * 4, 256));
     float* fin_lse = (float*)(w + 3 * align_up(f * 4, 256));
+    int32_t* row_status = (int32_t*)(w + 3 * align_up(f * 4, 256) + align_up((size_t)B * n_par * 4, 256));
 
     rsd::ScanArgs a;
     memset(&a, 0, sizeof(a));
@@ -185,7 +185,7 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
     a.subtract_lse = 0;
     a.out_token = fin_token; a.out_perturbed = fin_pert; a.out_value = fin_value; a.out_lse = fin_lse;
-    a.status = status;
+    a.status = status; a.row_status = row_status;   // status[b] is written by the epilogue
     launch_scan(draft_level, !draft_level->is_logprob, B * n_par, a, s);
     if (int e = check_launch("rsd_sbs_step(scan)")) return e;
 
@@ -193,6 +193,7 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     e.n_par = n_par; e.W = W; e.is_logprob = draft_level->is_logprob; e.first_parent_node = first_parent_node;
     e.seed_lo = (uint32_t)seed; e.seed_hi = (uint32_t)(seed >> 32); e.step = step; e.seq_base = seq_base;
     e.fin_token = fin_token; e.fin_value = fin_value; e.fin_pert = fin_pert; e.fin_lse = fin_lse;
+    e.row_status = row_status;
     e.sum_in = sum_logprob_in; e.gamma_in = trunc_gumbel_in;
     e.out_token = out_token; e.out_parent = out_parent; e.out_stride = out_stride; e.parent_base = parent_base;
     e.sum_out = sum_logprob_out; e.gamma_out = trunc_gumbel_out;

@@ -42,6 +42,8 @@ struct ScanArgs {
     float* out_value;     // [B][R][max_k] or null: the row's own value at each pick
     float* out_lse;       // [B][R] or null
     int32_t* status;      // [B], OR-ed into
+    int32_t* row_status;  // [B][R] or null; when set, the row's NaN flag is stored here instead (beam search level:
+                          // the epilogue assembles status[b], and a row with fewer than k picks is not an event)
     int32_t* node_token;  // [B][node_stride] or null: pick j of row r also goes to node child_base[r] + j
     int node_stride;
     uint32_t rk0[10], rk1[10];  // Philox round keys: seed_lo + r * 0x9E3779B9, seed_hi + r * 0xBB67AE85
@@ -744,7 +746,8 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
         int st = 0;
         if (nan_flag) st |= 1;       // RSD_ST_NAN_INPUT
         if (total < k) st |= 2;      // RSD_ST_FEWER_THAN_K
-        if (st) atomicOr(&a.status[b], st);
+        if (a.row_status) a.row_status[(int64_t)b * a.R + r] = st & 1;
+        else if (st) atomicOr(&a.status[b], st);
     }
 }
 
@@ -764,6 +767,7 @@ struct SbsEpilogueArgs {
     const float* fin_value;    // [B][n_par][W] the row's own value at the finalist
     const float* fin_pert;     // [B][n_par][W] value + noise in fp32 (decreasing within a parent)
     const float* fin_lse;      // [B][n_par]
+    const int32_t* row_status; // [B][n_par] status bits of the row scans
     const float* sum_in;       // [B][n_par] or null
     const float* gamma_in;     // [B][n_par] or null
     int32_t* out_token;   // [B][out_stride]
@@ -908,8 +912,13 @@ __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const Sb
         a.sum_out[o] = kNegInf;
         a.gamma_out[o] = kNegInf;
     }
-    if (tid == 0 && cnt < a.W) atomicOr(&a.status[b], 2);  // RSD_ST_FEWER_THAN_K
-    if (tid == 0) a.out_count[b] = cnt;
+    int row_bits = 0;
+    for (int kp = tid; kp < a.n_par; kp += kEpilogueThreads) row_bits |= a.row_status[(int64_t)b * a.n_par + kp];
+    row_bits = __syncthreads_or(row_bits);
+    if (tid == 0) {
+        a.status[b] = (row_bits & 1) | (cnt < a.W ? 2 : 0);  // RSD_ST_NAN_INPUT, RSD_ST_FEWER_THAN_K
+        a.out_count[b] = cnt;
+    }
 }
 
 }  // namespace rsd
