@@ -369,7 +369,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     __shared__ int sv_idx[kSurvCap];
     __shared__ uint32_t bin_max[32];                 // per lane index: largest sample over the warps (ordered encoding)
     __shared__ float red_f[kScanWarps];
-    __shared__ double red_d[kScanWarps];
+    __shared__ float red_s[kScanWarps];
     __shared__ int n_cand, n_surv, nan_flag;
     __shared__ float lse_sh;
 
@@ -487,32 +487,35 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     if (best > kNegInf) atomicMax(&bin_max[lane], float_to_ordered(best));
     if (NEED_LSE) {
         // the warp's share of the log-sum-exp: largest reference exponent C_w and sum of s_t * 2^(c_t - C_w) (exact
-        // scaling, summed in double); the last thread combines the warps' shares after the barrier
+        // scaling); the last thread combines the warps' shares after the barrier.  All in fp32: the threads' sums
+        // already are, and double-precision instructions are slow enough to show on every row's critical path.
         const float lse_c = lse_thr > kNegInf ? -lse_negc : kNegInf;  // this thread's reference exponent
         const float cw_max = warp_max(lse_c);
         float s0, s1, s2, s3;
         split_f32x2(acc0, s0, s1);
         split_f32x2(acc1, s2, s3);
         const float d = lse_c - cw_max;   // <= 0, an integer (NaN or -inf when there is nothing to add)
-        double term = 0.0;
-        if (lse_c > kNegInf && d > -1000.0f) term = ldexp((double)((s0 + s1) + (s2 + s3)), (int)d);
-        if (cw_max == -kNegInf) term = (double)(cw_max - cw_max);  // a +inf value: the sum is not a number
-        term = warp_sum(term);
-        if (lane == 0) { red_f[warp] = cw_max; red_d[warp] = term; }
+        float term = 0.0f;
+        if (lse_c > kNegInf && d > -120.0f) term = ((s0 + s1) + (s2 + s3)) * exp2f(d);
+        if (cw_max == -kNegInf) term = cw_max - cw_max;  // a +inf value: the sum is not a number
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) term += __shfl_xor_sync(0xFFFFFFFFu, term, o);
+        if (lane == 0) { red_f[warp] = cw_max; red_s[warp] = term; }
     }
     __syncthreads();   // also: every thread is done with its group slot, the queues may take the buffer over
     if (NEED_LSE && tid == kScanThreads - 1) {
         float C = red_f[0];
 #pragma unroll
         for (int w = 1; w < kScanWarps; ++w) C = fmaxf(C, red_f[w]);
-        double S = 0.0;
+        float S = 0.0f;
 #pragma unroll
         for (int w = 0; w < kScanWarps; ++w) {
             const float d = red_f[w] - C;
-            if (red_f[w] > kNegInf && d > -1000.0f) S += ldexp(red_d[w], (int)d);
-            else if (d != d) S = (double)d;
+            if (red_f[w] > kNegInf && d > -120.0f) S += red_s[w] * exp2f(d);
+            else if (d != d) S = d;
         }
-        lse_sh = (C > kNegInf && (S > 0.0 || S != S)) ? (float)((double)C * 0.6931471805599453 + log(S)) : kNegInf;
+        // C ln 2 + ln S with ln 2 split so that C * hi is exact (C is a small integer)
+        lse_sh = (C > kNegInf && (S > 0.0f || S != S)) ? fmaf(C, 0.693145751953125f, fmaf(C, 1.4286068203094172e-06f, logf(S))) : kNegInf;
     }
     float tau;
     {
