@@ -135,7 +135,8 @@ def rrs_chain(p, q, tokens):
     return theta, res, st
 
 
-def gumbel_topk(rows, k_per_row, rng_node, seed, step, *, is_logprob=False, seq_base=0, max_k=None):
+def gumbel_topk(rows, k_per_row, rng_node, seed, step, *, is_logprob=False, seq_base=0, max_k=None,
+                temperature=1.0):
     """rows [B,R,V]; returns dict(token[B,R,max_k], perturbed, logprob, margin[B,R], status[B])."""
     a, dt = _rows(rows)
     B, R, V = a.shape
@@ -148,7 +149,7 @@ def gumbel_topk(rows, k_per_row, rng_node, seed, step, *, is_logprob=False, seq_
     logp = np.zeros((B, R, max_k), np.float64)
     margin = np.zeros((B, R), np.float64)
     status = np.zeros(B, np.int32)
-    lib().rsd_oracle_gumbel_topk(_ptr(a), C.c_int(dt), C.c_int(int(is_logprob)),
+    lib().rsd_oracle_gumbel_topk(_ptr(a), C.c_int(dt), C.c_int(int(is_logprob)), C.c_double(temperature),
                                  C.c_int64(a.strides[0] // a.itemsize), C.c_int64(a.strides[1] // a.itemsize),
                                  C.c_int(B), C.c_int(R), C.c_int(V), _ptr(k), _ptr(nodes), C.c_int(max_k),
                                  C.c_uint64(seed), C.c_uint32(step), C.c_uint32(seq_base),
@@ -157,7 +158,7 @@ def gumbel_topk(rows, k_per_row, rng_node, seed, step, *, is_logprob=False, seq_
 
 
 def sbs_step(rows, W, first_parent_node, sum_logprob_in, trunc_gumbel_in, seed, step, *, is_logprob=False,
-             seq_base=0):
+             seq_base=0, temperature=1.0):
     """rows [B,n_par,V]; one Stochastic Beam Search level."""
     a, dt = _rows(rows)
     B, n_par, V = a.shape
@@ -171,7 +172,7 @@ def sbs_step(rows, W, first_parent_node, sum_logprob_in, trunc_gumbel_in, seed, 
     cnt = np.zeros(B, np.int32)
     margin = np.zeros(B, np.float64)
     status = np.zeros(B, np.int32)
-    lib().rsd_oracle_sbs_step(_ptr(a), C.c_int(dt), C.c_int(int(is_logprob)),
+    lib().rsd_oracle_sbs_step(_ptr(a), C.c_int(dt), C.c_int(int(is_logprob)), C.c_double(temperature),
                               C.c_int64(a.strides[0] // a.itemsize), C.c_int64(a.strides[1] // a.itemsize),
                               C.c_int(B), C.c_int(n_par), C.c_int(V), C.c_int(W), C.c_int32(first_parent_node),
                               _ptr(sig), _ptr(gam), C.c_uint64(seed), C.c_uint32(step), C.c_uint32(seq_base),
@@ -179,7 +180,8 @@ def sbs_step(rows, W, first_parent_node, sum_logprob_in, trunc_gumbel_in, seed, 
     return dict(token=tok, parent=par, sum_logprob=so, trunc_gumbel=go, count=cnt, margin=margin, status=status)
 
 
-def verify_tree(draft, target, parent, token, num_levels, seed, step, *, seq_base=0, want_weights=False):
+def verify_tree(draft, target, parent, token, num_levels, seed, step, *, seq_base=0, want_weights=False,
+                draft_temperature=1.0, target_temperature=1.0):
     """draft [B,P,V], target [B,N+1,V], parent [N+1] or [B,N+1] (flat, root -1), token [B,N+1]."""
     d, ddt = _rows(draft)
     t, tdt = _rows(target)
@@ -200,9 +202,9 @@ def verify_tree(draft, target, parent, token, num_levels, seed, step, *, seq_bas
     weights = np.zeros((B, V), np.float64) if want_weights else None
     status = np.zeros(B, np.int32)
     lib().rsd_oracle_verify_tree(_ptr(d), C.c_int(ddt), C.c_int64(d.strides[0] // d.itemsize),
-                                 C.c_int64(d.strides[1] // d.itemsize),
+                                 C.c_int64(d.strides[1] // d.itemsize), C.c_double(draft_temperature),
                                  _ptr(t), C.c_int(tdt), C.c_int64(t.strides[0] // t.itemsize),
-                                 C.c_int64(t.strides[1] // t.itemsize),
+                                 C.c_int64(t.strides[1] // t.itemsize), C.c_double(target_temperature),
                                  C.c_int(B), C.c_int(V), C.c_int(n_nodes), C.c_int(L),
                                  _ptr(par), C.c_int(shared), _ptr(tok),
                                  C.c_uint64(seed), C.c_uint32(step), C.c_uint32(seq_base),
@@ -212,7 +214,8 @@ def verify_tree(draft, target, parent, token, num_levels, seed, step, *, seq_bas
                 theta=theta, margin=margin, final_margin=fmargin, final_weights=weights, status=status)
 
 
-def resample_residual(draft, target, rejected, rng_node, seed, step, *, seq_base=0):
+def resample_residual(draft, target, rejected, rng_node, seed, step, *, seq_base=0, draft_temperature=1.0,
+                      target_temperature=1.0):
     """draft/target [B,V] (draft may be None when nothing was rejected); rejected [B,max_k] (-1 padded)."""
     t, tdt = _rows(target)
     B, V = t.shape
@@ -227,8 +230,9 @@ def resample_residual(draft, target, rejected, rng_node, seed, step, *, seq_base
     res = np.zeros((B, V), np.float64)
     margin = np.zeros(B, np.float64)
     status = np.zeros(B, np.int32)
-    lib().rsd_oracle_resample_residual(_ptr(d), C.c_int(ddt), C.c_int64(dstride),
+    lib().rsd_oracle_resample_residual(_ptr(d), C.c_int(ddt), C.c_int64(dstride), C.c_double(draft_temperature),
                                        _ptr(t), C.c_int(tdt), C.c_int64(t.strides[0] // t.itemsize),
+                                       C.c_double(target_temperature),
                                        C.c_int(B), C.c_int(V), _ptr(rej), C.c_int(rej.shape[1]), _ptr(nodes),
                                        C.c_uint64(seed), C.c_uint32(step), C.c_uint32(seq_base),
                                        _ptr(out), _ptr(res), _ptr(margin), _ptr(status))

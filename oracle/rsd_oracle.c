@@ -156,13 +156,16 @@ static double read_elem(const void* base, int dtype, int64_t idx) {
     return (double)f;
 }
 
-/* copy a row to double; NaN becomes -inf and is reported */
-static int load_row(const void* base, int dtype, int64_t off, int V, double* out) {
+/* sampling temperature (Section 4: 0.3 or 1.0): a value <= 0 or == 1 means "none" */
+static int has_temperature(double t) { return t > 0.0 && t != 1.0; }
+
+/* copy a row to double, divided by the temperature; NaN becomes -inf and is reported */
+static int load_row(const void* base, int dtype, int64_t off, int V, double temperature, double* out) {
     int saw_nan = 0;
     for (int x = 0; x < V; ++x) {
         double v = read_elem(base, dtype, off + x);
         if (isnan(v)) { v = -INFINITY; saw_nan = 1; }
-        out[x] = v;
+        out[x] = has_temperature(temperature) ? v / temperature : v;
     }
     return saw_nan;
 }
@@ -201,7 +204,8 @@ static void softmax_row(const double* logits, int V, double* prob) {
  * selected; missing picks are -1.  out_margin[b][r] = the smallest gap between
  * consecutive sorted values v_1 >= ... >= v_{k+1} (v_{k+1} = best loser).
  */
-int rsd_oracle_gumbel_topk(const void* data, int dtype, int is_logprob, int64_t seq_stride, int64_t row_stride,
+int rsd_oracle_gumbel_topk(const void* data, int dtype, int is_logprob, double temperature, int64_t seq_stride,
+                           int64_t row_stride,
                            int B, int R, int V, const int32_t* k_per_row, const int32_t* rng_node, int max_k,
                            uint64_t seed, uint32_t step, uint32_t seq_base,
                            int32_t* out_token, double* out_perturbed, double* out_logprob, double* out_margin,
@@ -214,8 +218,8 @@ int rsd_oracle_gumbel_topk(const void* data, int dtype, int is_logprob, int64_t 
             double* pert = (double*)malloc(sizeof(double) * (size_t)V);
             char* taken = (char*)calloc((size_t)V, 1);
             int st = 0;
-            if (load_row(data, dtype, b * seq_stride + r * row_stride, V, phi)) st |= ORC_ST_NAN_INPUT;
-            log_softmax_row(phi, V, is_logprob);
+            if (load_row(data, dtype, b * seq_stride + r * row_stride, V, temperature, phi)) st |= ORC_ST_NAN_INPUT;
+            log_softmax_row(phi, V, is_logprob && !has_temperature(temperature));   /* scaled rows are scores again */
             for (int x = 0; x < V; ++x)
                 pert[x] = phi[x] + rsd_oracle_gumbel(seed, step, seq_base + (uint32_t)b, (uint32_t)rng_node[r], (uint32_t)x);
             int k = k_per_row[r];
@@ -280,7 +284,8 @@ double rsd_oracle_truncated_gumbel(double u, double phi, double z) {
  * root).  Outputs the W best (token, parent) pairs by psi, decreasing; equal
  * values go to the smaller parent, then the smaller token.
  */
-int rsd_oracle_sbs_step(const void* data, int dtype, int is_logprob, int64_t seq_stride, int64_t row_stride,
+int rsd_oracle_sbs_step(const void* data, int dtype, int is_logprob, double temperature, int64_t seq_stride,
+                        int64_t row_stride,
                         int B, int n_par, int V, int W, int32_t first_parent_node,
                         const double* sum_logprob_in, const double* trunc_gumbel_in,
                         uint64_t seed, uint32_t step, uint32_t seq_base,
@@ -295,8 +300,8 @@ int rsd_oracle_sbs_step(const void* data, int dtype, int is_logprob, int64_t seq
         int st = 0;
         for (int k = 0; k < n_par; ++k) {
             double* row = phi + (size_t)k * V;
-            if (load_row(data, dtype, b * seq_stride + k * row_stride, V, row)) st |= ORC_ST_NAN_INPUT;
-            log_softmax_row(row, V, is_logprob);
+            if (load_row(data, dtype, b * seq_stride + k * row_stride, V, temperature, row)) st |= ORC_ST_NAN_INPUT;
+            log_softmax_row(row, V, is_logprob && !has_temperature(temperature));
             double sigma = sum_logprob_in ? sum_logprob_in[(int64_t)b * n_par + k] : 0.0;
             double gamma = trunc_gumbel_in ? trunc_gumbel_in[(int64_t)b * n_par + k] : 0.0;
             double* pert = psi + (size_t)k * V;
@@ -457,7 +462,9 @@ int rsd_oracle_rrs_chain(const double* p_in, const double* q_in, int V, const in
  * token was drawn from.
  */
 int rsd_oracle_verify_tree(const void* draft, int draft_dtype, int64_t draft_seq_stride, int64_t draft_row_stride,
+                           double draft_temperature,
                            const void* target, int target_dtype, int64_t target_seq_stride, int64_t target_row_stride,
+                           double target_temperature,
                            int B, int V, int n_nodes /* N+1 */, int num_levels,
                            const int32_t* parent, int topology_is_shared, const int32_t* token,
                            uint64_t seed, uint32_t step, uint32_t seq_base,
@@ -485,13 +492,13 @@ int rsd_oracle_verify_tree(const void* draft, int draft_dtype, int64_t draft_seq
         for (;;) {
             int n_children = 0;
             for (int c = 1; c < n_nodes; ++c) if (par[c] == cur && tok[c] >= 0) ++n_children;
-            if (load_row(target, target_dtype, b * target_seq_stride + cur * target_row_stride, V, lt)) st |= ORC_ST_NAN_INPUT;
+            if (load_row(target, target_dtype, b * target_seq_stride + cur * target_row_stride, V, target_temperature, lt)) st |= ORC_ST_NAN_INPUT;
             softmax_row(lt, V, q);
             if (n_children == 0 || len >= num_levels) {
                 reason = (len >= num_levels) ? ORC_STOP_LEAF : ORC_STOP_NO_CHILDREN;
                 break;
             }
-            if (load_row(draft, draft_dtype, b * draft_seq_stride + cur * draft_row_stride, V, ld)) st |= ORC_ST_NAN_INPUT;
+            if (load_row(draft, draft_dtype, b * draft_seq_stride + cur * draft_row_stride, V, draft_temperature, ld)) st |= ORC_ST_NAN_INPUT;
             softmax_row(ld, V, p);
             int accepted_child = -1, j = 0, alive = 1;
             for (int c = 1; c < n_nodes && alive; ++c) {
@@ -534,8 +541,9 @@ int rsd_oracle_verify_tree(const void* draft, int draft_dtype, int64_t draft_seq
  * (sequence, rng_node[b]).  With no rejected token this is a plain draw from
  * the target row (draft may then be NULL).
  */
-int rsd_oracle_resample_residual(const void* draft, int draft_dtype, int64_t draft_seq_stride,
+int rsd_oracle_resample_residual(const void* draft, int draft_dtype, int64_t draft_seq_stride, double draft_temperature,
                                  const void* target, int target_dtype, int64_t target_seq_stride,
+                                 double target_temperature,
                                  int B, int V, const int32_t* rejected, int max_k, const int32_t* rng_node,
                                  uint64_t seed, uint32_t step, uint32_t seq_base,
                                  int32_t* out_token, double* out_residual, double* out_margin, int32_t* status) {
@@ -545,12 +553,12 @@ int rsd_oracle_resample_residual(const void* draft, int draft_dtype, int64_t dra
         double* q = (double*)malloc(sizeof(double) * (size_t)V);
         double* p = (double*)malloc(sizeof(double) * (size_t)V);
         int st = 0;
-        if (load_row(target, target_dtype, b * target_seq_stride, V, l)) st |= ORC_ST_NAN_INPUT;
+        if (load_row(target, target_dtype, b * target_seq_stride, V, target_temperature, l)) st |= ORC_ST_NAN_INPUT;
         softmax_row(l, V, q);
         int n_rej = 0;
         for (int i = 0; i < max_k; ++i) if (rejected && rejected[(int64_t)b * max_k + i] >= 0) ++n_rej;
         if (n_rej > 0) {
-            if (load_row(draft, draft_dtype, b * draft_seq_stride, V, l)) st |= ORC_ST_NAN_INPUT;
+            if (load_row(draft, draft_dtype, b * draft_seq_stride, V, draft_temperature, l)) st |= ORC_ST_NAN_INPUT;
             softmax_row(l, V, p);
             for (int i = 0; i < max_k; ++i) {
                 int x = rejected[(int64_t)b * max_k + i];
