@@ -80,6 +80,10 @@ typedef struct rsd_rows {
     int32_t is_logprob; /* 1: rows are log-probabilities already (drafting uses them as given) */
     int64_t seq_stride; /* elements between sequences */
     int64_t row_stride; /* elements between rows of one sequence, >= V */
+    float temperature;  /* sampling temperature (Section 4 uses 0.3 and 1.0): every value is divided by it before the
+                           log-softmax; 0 or 1 = none.  With a temperature, rows flagged is_logprob are re-scored
+                           (their log-softmax is taken again after the division).  Negative, infinite or NaN values
+                           are refused. */
 } rsd_rows;
 
 typedef struct rsd_tree {

@@ -26,7 +26,7 @@ EXPORTS = ["rsd_version", "rsd_rng_layout", "rsd_last_error", "rsd_profile_next_
 
 class RsdRows(C.Structure):
     _fields_ = [("data", C.c_void_p), ("dtype", C.c_int32), ("is_logprob", C.c_int32),
-                ("seq_stride", C.c_int64), ("row_stride", C.c_int64)]
+                ("seq_stride", C.c_int64), ("row_stride", C.c_int64), ("temperature", C.c_float)]
 
 
 class RsdTree(C.Structure):
@@ -87,7 +87,7 @@ def _ptr(t: Optional[torch.Tensor]):
     return None if t is None else t.data_ptr()
 
 
-def rows_of(t: torch.Tensor, is_logprob: bool = False) -> RsdRows:
+def rows_of(t: torch.Tensor, is_logprob: bool = False, temperature: float = 1.0) -> RsdRows:
     """Describe a [B, R, V] (or [B, V]) CUDA tensor of fp32 or bf16 rows; the last dimension must be dense."""
     if not t.is_cuda:
         raise RsdError("rows must live on a CUDA device")
@@ -100,9 +100,9 @@ def rows_of(t: torch.Tensor, is_logprob: bool = False) -> RsdRows:
     if t.stride(-1) != 1:
         raise RsdError("rows must be dense along the vocabulary")
     if t.dim() == 3:
-        return RsdRows(t.data_ptr(), dt, int(is_logprob), t.stride(0), t.stride(1))
+        return RsdRows(t.data_ptr(), dt, int(is_logprob), t.stride(0), t.stride(1), float(temperature))
     if t.dim() == 2:
-        return RsdRows(t.data_ptr(), dt, int(is_logprob), t.stride(0), t.shape[1])
+        return RsdRows(t.data_ptr(), dt, int(is_logprob), t.stride(0), t.shape[1], float(temperature))
     raise RsdError("rows must be [B, R, V] or [B, V]")
 
 
@@ -114,7 +114,8 @@ def _host_i32(values: Sequence[int]):
 def rsd_gumbel_topk_draft(draft: torch.Tensor, k_per_row: Sequence[int], rng_node: Sequence[int], seed: int,
                           step: int, *, is_logprob: bool = False, seq_base: int = 0, max_k: Optional[int] = None,
                           want_values: bool = False, child_base: Optional[Sequence[int]] = None,
-                          node_token: Optional[torch.Tensor] = None, out: Optional[dict] = None):
+                          node_token: Optional[torch.Tensor] = None, out: Optional[dict] = None,
+                          temperature: float = 1.0):
     """draft [B, R, V] -> dict(token [B, R, max_k], status [B], and perturbed/logprob when want_values).
 
     With child_base [R] and node_token [B, N+1] (int32) the picks also land in the tree's per-node token array.
@@ -127,7 +128,7 @@ def rsd_gumbel_topk_draft(draft: torch.Tensor, k_per_row: Sequence[int], rng_nod
                    status=torch.empty((B,), dtype=torch.int32, device=dev),
                    perturbed=torch.empty((B, R, max_k), dtype=torch.float32, device=dev) if want_values else None,
                    logprob=torch.empty((B, R, max_k), dtype=torch.float32, device=dev) if want_values else None)
-    rows = rows_of(draft, is_logprob)
+    rows = rows_of(draft, is_logprob, temperature)
     if node_token is not None and (node_token.dtype != torch.int32 or not node_token.is_contiguous()):
         raise RsdError("node_token must be contiguous int32")
     _check(lib().rsd_gumbel_topk_draft(C.byref(rows), B, R, V, _host_i32(k_per_row), _host_i32(rng_node), max_k,
@@ -151,7 +152,7 @@ def rsd_sbs_workspace_bytes(B: int, n_par: int, W: int) -> int:
 def rsd_sbs_step(draft_level: torch.Tensor, W: int, first_parent_node: int, sum_logprob_in: Optional[torch.Tensor],
                  trunc_gumbel_in: Optional[torch.Tensor], seed: int, step: int, *, is_logprob: bool = False,
                  seq_base: int = 0, workspace: Optional[torch.Tensor] = None, out: Optional[dict] = None,
-                 parent_base: int = 0):
+                 parent_base: int = 0, temperature: float = 1.0):
     """draft_level [B, n_par, V] -> dict(token, parent, sum_logprob, trunc_gumbel [B, W], count [B], status [B]).
 
     out["token"] / out["parent"] may be [B, W] views into wider [B, N+1] tree arrays (row stride kept); parent_base
@@ -169,7 +170,7 @@ def rsd_sbs_step(draft_level: torch.Tensor, W: int, first_parent_node: int, sum_
                    trunc_gumbel=torch.empty((B, W), dtype=torch.float32, device=dev),
                    count=torch.empty((B,), dtype=torch.int32, device=dev),
                    status=torch.empty((B,), dtype=torch.int32, device=dev))
-    rows = rows_of(draft_level, is_logprob)
+    rows = rows_of(draft_level, is_logprob, temperature)
     if out["token"].stride(0) != out["parent"].stride(0) or out["token"].stride(1) != 1 or out["parent"].stride(1) != 1:
         raise RsdError("out token/parent must share a row stride and be dense along the picks")
     _check(lib().rsd_sbs_step(C.byref(rows), B, n_par, V, W, first_parent_node, _ptr(sum_logprob_in),
@@ -184,7 +185,8 @@ SBS_STATIC_SCRATCH_BYTES = 1 << 20
 
 def rsd_sbs_step_static(draft_level: torch.Tensor, W: int, first_parent_node: int,
                         sum_logprob_in: Optional[torch.Tensor], trunc_gumbel_in: Optional[torch.Tensor], seed: int,
-                        step: int, out: dict, *, is_logprob: bool = False, seq_base: int = 0, parent_base: int = 0):
+                        step: int, out: dict, *, is_logprob: bool = False, seq_base: int = 0, parent_base: int = 0,
+                        temperature: float = 1.0):
     """rsd_sbs_step with the library's built-in scratch, for callers that may not allocate device memory.
 
     `out` must hold the caller's own tensors (token, parent, sum_logprob, trunc_gumbel [B, W]; count, status [B]):
@@ -192,7 +194,7 @@ def rsd_sbs_step_static(draft_level: torch.Tensor, W: int, first_parent_node: in
     scratch.  Calls that overlap on one GPU share that scratch and race.
     """
     B, n_par, V = draft_level.shape
-    rows = rows_of(draft_level, is_logprob)
+    rows = rows_of(draft_level, is_logprob, temperature)
     if out["token"].stride(0) != out["parent"].stride(0) or out["token"].stride(1) != 1 or out["parent"].stride(1) != 1:
         raise RsdError("out token/parent must share a row stride and be dense along the picks")
     _check(lib().rsd_sbs_step_static(C.byref(rows), B, n_par, V, W, first_parent_node, _ptr(sum_logprob_in),
@@ -205,7 +207,7 @@ def rsd_sbs_step_static(draft_level: torch.Tensor, W: int, first_parent_node: in
 
 def rsd_verify_tree(draft: torch.Tensor, target: torch.Tensor, parent: torch.Tensor, token: torch.Tensor,
                     num_levels: int, seed: int, step: int, *, seq_base: int = 0, want_theta: bool = False,
-                    out: Optional[dict] = None):
+                    out: Optional[dict] = None, draft_temperature: float = 1.0, target_temperature: float = 1.0):
     """draft [B, P, V], target [B, N+1, V], parent [N+1] or [B, N+1] int32, token [B, N+1] int32."""
     B, _, V = target.shape
     dev = target.device
@@ -224,7 +226,7 @@ def rsd_verify_tree(draft: torch.Tensor, target: torch.Tensor, parent: torch.Ten
                    status=torch.empty((B,), dtype=torch.int32, device=dev))
         out["theta"] = torch.empty((B, n_nodes), dtype=torch.float32, device=dev) if want_theta else None
     tree = RsdTree(L, n_nodes, parent.data_ptr(), token.data_ptr(), 1 if parent.dim() == 1 else 0)
-    d, t = rows_of(draft), rows_of(target)
+    d, t = rows_of(draft, False, draft_temperature), rows_of(target, False, target_temperature)
     _check(lib().rsd_verify_tree(C.byref(d), C.byref(t), C.byref(tree), B, V, seed, step, seq_base,
                                  _ptr(out["accepted_len"]), _ptr(out["accepted_node"]), _ptr(out["accepted_token"]),
                                  _ptr(out["last_token"]), _ptr(out["stop_reason"]), _ptr(out.get("theta")),
@@ -234,15 +236,16 @@ def rsd_verify_tree(draft: torch.Tensor, target: torch.Tensor, parent: torch.Ten
 
 def rsd_resample_residual(draft_row: Optional[torch.Tensor], target_row: torch.Tensor,
                           rejected: Optional[torch.Tensor], rng_node: torch.Tensor, seed: int, step: int, *,
-                          seq_base: int = 0, want_residual: bool = False):
+                          seq_base: int = 0, want_residual: bool = False, draft_temperature: float = 1.0,
+                          target_temperature: float = 1.0):
     """draft_row/target_row [B, V]; rejected [B, max_k] int32 (-1 padded) or None; rng_node [B] int32."""
     B, V = target_row.shape
     dev = target_row.device
     token = torch.empty((B,), dtype=torch.int32, device=dev)
     status = torch.empty((B,), dtype=torch.int32, device=dev)
     residual = torch.empty((B, V), dtype=torch.float32, device=dev) if want_residual else None
-    t = rows_of(target_row)
-    d = rows_of(draft_row) if draft_row is not None else t
+    t = rows_of(target_row, False, target_temperature)
+    d = rows_of(draft_row, False, draft_temperature) if draft_row is not None else t
     max_k = 0 if rejected is None else rejected.shape[1]
     if rejected is not None and (rejected.dtype != torch.int32 or not rejected.is_contiguous()):
         raise RsdError("rejected must be contiguous int32")

@@ -32,8 +32,15 @@ int check_rows(const char* name, const rsd_rows* r, int V, bool need_row_stride)
     if (r->dtype != RSD_F32 && r->dtype != RSD_BF16) return fail(RSD_ERR_UNSUPPORTED, "%s: unknown dtype %d", name, r->dtype);
     if (need_row_stride && r->row_stride < V) return fail(RSD_ERR_INVALID_ARG, "%s: row_stride %lld < V %d", name, (long long)r->row_stride, V);
     if (r->seq_stride < 0 || r->row_stride < 0) return fail(RSD_ERR_INVALID_ARG, "%s: negative stride", name);
+    if (!(r->temperature >= 0.0f) || r->temperature > 3.0e38f)
+        return fail(RSD_ERR_INVALID_ARG, "%s: temperature %g must be a finite number >= 0 (0 or 1: none)", name, (double)r->temperature);
     return RSD_OK;
 }
+
+// temperature that applies (1 when the rows ask for none)
+float temperature_of(const rsd_rows* r) { return (r->temperature > 0.0f && r->temperature != 1.0f) ? r->temperature : 1.0f; }
+// rows usable as log-probabilities as they are: flagged so and not re-scored by a temperature
+bool rows_are_logprob(const rsd_rows* r) { return r->is_logprob && temperature_of(r) == 1.0f; }
 
 bool rows_aligned(const rsd_rows* r, int bytes = 16) {
     const int64_t eb = r->dtype == RSD_F32 ? 4 : 2;
@@ -45,16 +52,22 @@ int check_vocab(int V) {
     return RSD_OK;
 }
 
-template <typename T, bool ALIGNED, bool WIDE, bool NEED_LSE>
-void launch_scan_one(int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
+template <typename T, bool ALIGNED, bool WIDE, bool NEED_LSE, bool TEMP>
+void launch_scan_temp(int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
     const size_t smem = sizeof(float) * (size_t)((((a.V + 15) / 16) + 3) / 4 * 4);  // one bound per group of 16 elements, padded to fours
     static bool raised = false;  // per instantiation: allow the largest vocabulary's dynamic shared memory
     if (!raised) {
-        cudaFuncSetAttribute(rsd::scan_topk_kernel<T, ALIGNED, WIDE, NEED_LSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(rsd::scan_topk_kernel<T, ALIGNED, WIDE, NEED_LSE, TEMP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)(sizeof(float) * (RSD_MAX_VOCAB / 16)));
         raised = true;
     }
-    rsd::scan_topk_kernel<T, ALIGNED, WIDE, NEED_LSE><<<blocks, rsd::kScanThreads, smem, s>>>(a);
+    rsd::scan_topk_kernel<T, ALIGNED, WIDE, NEED_LSE, TEMP><<<blocks, rsd::kScanThreads, smem, s>>>(a);
+}
+
+template <typename T, bool ALIGNED, bool WIDE, bool NEED_LSE>
+void launch_scan_one(int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
+    if (a.temp != 1.0f) launch_scan_temp<T, ALIGNED, WIDE, NEED_LSE, true>(blocks, a, s);
+    else launch_scan_temp<T, ALIGNED, WIDE, NEED_LSE, false>(blocks, a, s);
 }
 
 template <bool NEED_LSE>
@@ -135,7 +148,8 @@ int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int3
     a.subtract_lse = 1;
     a.out_token = out_token; a.out_perturbed = out_perturbed; a.out_value = out_logprob; a.out_lse = nullptr;
     a.status = status; a.node_token = node_token; a.node_stride = node_stride;
-    const bool need_lse = !draft->is_logprob && (out_perturbed || out_logprob);
+    a.temp = temperature_of(draft); a.inv_temp = 1.0f / a.temp;
+    const bool need_lse = !rows_are_logprob(draft) && (out_perturbed || out_logprob);
     launch_scan(draft, need_lse, B * R, a, s);
     return check_launch("rsd_gumbel_topk_draft");
 }
@@ -186,11 +200,12 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     a.subtract_lse = 0;
     a.out_token = fin_token; a.out_perturbed = fin_pert; a.out_value = fin_value; a.out_lse = fin_lse;
     a.status = status; a.row_status = row_status;   // status[b] is written by the epilogue
-    launch_scan(draft_level, !draft_level->is_logprob, B * n_par, a, s);
+    a.temp = temperature_of(draft_level); a.inv_temp = 1.0f / a.temp; a.raw_values = 1;
+    launch_scan(draft_level, !rows_are_logprob(draft_level), B * n_par, a, s);
     if (int e = check_launch("rsd_sbs_step(scan)")) return e;
 
     rsd::SbsEpilogueArgs e;
-    e.n_par = n_par; e.W = W; e.is_logprob = draft_level->is_logprob; e.first_parent_node = first_parent_node;
+    e.n_par = n_par; e.W = W; e.is_logprob = rows_are_logprob(draft_level); e.inv_temp = 1.0 / (double)temperature_of(draft_level); e.first_parent_node = first_parent_node;
     e.seed_lo = (uint32_t)seed; e.seed_hi = (uint32_t)(seed >> 32); e.step = step; e.seq_base = seq_base;
     e.fin_token = fin_token; e.fin_value = fin_value; e.fin_pert = fin_pert; e.fin_lse = fin_lse;
     e.row_status = row_status;
@@ -219,8 +234,8 @@ int rsd_verify_tree(const rsd_rows* draft, const rsd_rows* target, const rsd_tre
     if (!accepted_len || !accepted_node || !accepted_token || !last_token || !stop_reason || !status) return fail(RSD_ERR_INVALID_ARG, "null output");
     if (B == 0) return RSD_OK;
     rsd::VerifyArgs a;
-    a.draft = {draft->data, draft->seq_stride, draft->row_stride};
-    a.target = {target->data, target->seq_stride, target->row_stride};
+    a.draft = {draft->data, draft->seq_stride, draft->row_stride, 1.0f / temperature_of(draft)};
+    a.target = {target->data, target->seq_stride, target->row_stride, 1.0f / temperature_of(target)};
     a.V = V; a.L = tree->num_levels; a.num_nodes = tree->num_nodes; a.shared_topology = tree->topology_is_shared;
     a.parent = tree->parent; a.token = tree->token;
     a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
@@ -254,8 +269,8 @@ int rsd_resample_residual(const rsd_rows* draft_row, const rsd_rows* target_row,
     if (!rng_node || !out_token || !status) return fail(RSD_ERR_INVALID_ARG, "null argument");
     if (B == 0) return RSD_OK;
     rsd::ResampleArgs a;
-    a.target = {target_row->data, target_row->seq_stride, 0};
-    a.draft = rejected ? rsd::RowsDev{draft_row->data, draft_row->seq_stride, 0} : a.target;
+    a.target = {target_row->data, target_row->seq_stride, 0, 1.0f / temperature_of(target_row)};
+    a.draft = rejected ? rsd::RowsDev{draft_row->data, draft_row->seq_stride, 0, 1.0f / temperature_of(draft_row)} : a.target;
     a.V = V; a.max_k = rejected ? max_k : 0; a.rejected = rejected; a.rng_node = rng_node;
     a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
     a.out_token = out_token; a.out_residual = out_residual; a.status = status;

@@ -37,6 +37,9 @@ struct ScanArgs {
     int R, V, max_k;
     uint32_t seed_lo, seed_hi, step, seq_base;
     int subtract_lse;     // 1: outputs in log-probability units (value - LSE)
+    float inv_temp, temp; // every value is multiplied by inv_temp = 1 / temperature before anything else (1: none)
+    int raw_values;       // 1: out_value receives the rows' own values as stored (the beam search epilogue scales them
+                          // in double); 0: value * inv_temp - shift
     int32_t* out_token;   // [B][R][max_k]
     float* out_perturbed; // [B][R][max_k] or null
     float* out_value;     // [B][R][max_k] or null: the row's own value at each pick
@@ -349,7 +352,8 @@ __device__ __forceinline__ float slot_element<__nv_bfloat16>(uint32_t addr, uint
 
 // One block per row.
 // ALIGNED: rows start on 16-byte boundaries and V is a multiple of 16 (vector loads); WIDE: 32-byte boundaries as well.
-template <typename T, bool ALIGNED, bool WIDE, bool NEED_LSE>
+// TEMP: a sampling temperature other than 1 applies (otherwise the scale factors are compile-time constants).
+template <typename T, bool ALIGNED, bool WIDE, bool NEED_LSE, bool TEMP>
 __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanArgs a) {
     extern __shared__ float ub[];                    // [n_groups] upper bound of each group's perturbed values
     // One buffer, two uses: the threads' group slots during the streaming loop, the queues of the stages after it.
@@ -394,6 +398,8 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     float best = kNegInf;                  // largest exact sample of this thread (value(a) + lower bound of G_max)
     // Running log-sum-exp of this thread's elements: sum of 2^(value * log2(e) - c) with an integer c, fixed at the
     // first finite group maximum and moved up only when a group maximum exceeds it by more than 40.
+    const float inv_temp = TEMP ? a.inv_temp : 1.0f, temp = TEMP ? a.temp : 1.0f;   // values enter as value * inv_temp
+    const float log2e_t = kLog2e * inv_temp;
     float lse_thr = kNegInf;               // group maxima above this move the reference (-inf: nothing finite yet)
     float lse_negc = 0.0f;                 // -c
     unsigned long long acc0 = f32x2(0.0f, 0.0f), acc1 = acc0;
@@ -404,8 +410,8 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
         float g_lo, g_hi;
         group_noise_bounds(word >> 4, g_lo, g_hi);
         float gmax = group_max_nan(cur);
-        *ub_g = gmax + g_hi;                                   // NaN if the group holds a NaN: looked at later
-        best = fmaxf(best, slot_element<T>(slot, word & 15u) + g_lo);  // fmaxf drops NaN
+        *ub_g = fmaf(gmax, inv_temp, g_hi);                    // NaN if the group holds a NaN: looked at later
+        best = fmaxf(best, fmaf(slot_element<T>(slot, word & 15u), inv_temp, g_lo));  // fmaxf drops NaN
         if (NEED_LSE) {
             float v[16];
             cur.unpack(v);
@@ -419,7 +425,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                     }
                 }
                 if (gmax > lse_thr) {
-                    const float c_new = ceilf(gmax * kLog2e);
+                    const float c_new = ceilf(gmax * log2e_t);
                     const float sc = lse_thr > kNegInf ? ex2_approx(-(lse_negc + c_new)) : 0.0f;  // 2^(c_old - c_new) <= 1
                     float s0, s1, s2, s3;
                     split_f32x2(acc0, s0, s1);
@@ -427,10 +433,10 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                     acc0 = f32x2(s0 * sc, s1 * sc);
                     acc1 = f32x2(s2 * sc, s3 * sc);
                     lse_negc = -c_new;
-                    lse_thr = gmax + 40.0f;
+                    lse_thr = fmaf(40.0f, temp, gmax);   // 40 in scaled units
                 }
             }
-            const unsigned long long l2 = f32x2(kLog2e, kLog2e), c2 = f32x2(lse_negc, lse_negc);
+            const unsigned long long l2 = f32x2(log2e_t, log2e_t), c2 = f32x2(lse_negc, lse_negc);
 #pragma unroll
             for (int j = 0; j < 16; j += 4) {  // two elements per fma / add, two accumulators
                 float e0, e1, e2, e3;
@@ -584,7 +590,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
         {
             float v[16];
             grp.unpack(v);
-            const float need = tau - g_max - 1e-5f;
+            const float need = (tau - g_max - 1e-5f) * temp - 1e-6f * fabsf((tau - g_max) * temp);   // in raw units
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
                 if (v[j] != v[j]) nan_flag = 1;
@@ -595,12 +601,13 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
             const int j = __ffs(todo) - 1;
             todo &= todo - 1;
             const int x = g * 16 + j;
-            const float raw = group_element(grp, j);
+            const float raw_u = group_element(grp, j);
+            const float raw = raw_u * inv_temp;
             float pert = raw + g_max;
             if (j != apos) pert = raw - logf(base + neg_log_uniform_f32(fine_word_rk(a, key, node, (uint32_t)x)));
             if (pert >= tau) {
                 const int sidx = atomicAdd(&n_surv, 1);
-                if (sidx < kSurvCap) { sv_val[sidx] = pert; sv_idx[sidx] = x; sv_raw[sidx] = raw; }
+                if (sidx < kSurvCap) { sv_val[sidx] = pert; sv_idx[sidx] = x; sv_raw[sidx] = raw_u; }
             }
         }
     };
@@ -622,7 +629,8 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
             const float need = tau + __logf(fmaxf(base_lo, 1e-37f)) - 2e-4f;   // tau - (upper bound of G_max)
             const uint32_t apos = word & 15u;
             if (ub[g] != ub[g]) nan_flag = 1;                  // the bound is NaN exactly when the group holds one
-            const float need_f = fmaxf(need, -3.4028234663852886e38f);   // finite: -inf and NaN never pass
+            // the same bound for the raw values (value * inv_temp >= need), rounded down; finite: -inf, NaN never pass
+            const float need_f = fmaxf(need * temp - 2e-6f * fabsf(need * temp), -3.4028234663852886e38f);
             uint32_t todo = group_mask_ge(grp, need_f);
             if (todo) {
                 int slot_t = atomicAdd(&n_task, __popc(todo));
@@ -647,7 +655,8 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                 const uint32_t x = xe & 0x7FFFFFFFu;
                 uint32_t w = 0;
                 bool keep = true;
-                const float raw = RowIO<T>::scalar(row, (int)x);   // an L2 hit, in flight during the Philox rounds below
+                const float raw_u = RowIO<T>::scalar(row, (int)x);   // an L2 hit, in flight during the Philox rounds
+                const float raw = raw_u * inv_temp;
                 if (!(xe & 0x80000000u)) {
                     w = fine_word_rk(a, key, node, x);
                     const float uu = fmaf((float)w, 2.3283064365386963e-10f, 1.1641532182693481e-10f);
@@ -658,7 +667,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                 }
                 if (keep) {
                     const int slot = atomicAdd(&n_fin, 1);
-                    if (slot < kFinCap) { fin_x[slot] = xe; fin_w[slot] = w; fin_raw[slot] = raw; fin_word[slot] = tk_word[i]; }
+                    if (slot < kFinCap) { fin_x[slot] = xe; fin_w[slot] = w; fin_raw[slot] = raw_u; fin_word[slot] = tk_word[i]; }
                 }
             }
             __syncthreads();
@@ -669,12 +678,13 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                     const uint32_t xe = fin_x[i];
                     const int x = (int)(xe & 0x7FFFFFFFu);
                     const float base = neg_log_group_uniform_f32(fin_word[i]) * 0.0625f;
-                    const float raw = fin_raw[i];
+                    const float raw_u = fin_raw[i];
+                    const float raw = raw_u * inv_temp;
                     const float t_x = (xe & 0x80000000u) ? 0.0f : neg_log_uniform_f32(fin_w[i]);
                     const float pert = raw - logf(base + t_x);
                     if (pert >= tau) {
                         const int sidx = atomicAdd(&n_surv, 1);
-                        if (sidx < kSurvCap) { sv_val[sidx] = pert; sv_idx[sidx] = x; sv_raw[sidx] = raw; }
+                        if (sidx < kSurvCap) { sv_val[sidx] = pert; sv_idx[sidx] = x; sv_raw[sidx] = raw_u; }
                     }
                 }
                 __syncthreads();
@@ -735,7 +745,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
             a.out_token[o + rnk] = mi;
             if (a.node_token) a.node_token[(int64_t)b * a.node_stride + a.child_base[r] + rnk] = mi;
             if (a.out_perturbed) a.out_perturbed[o + rnk] = mv - shift;
-            if (a.out_value) a.out_value[o + rnk] = sv_raw[e] - shift;
+            if (a.out_value) a.out_value[o + rnk] = a.raw_values ? sv_raw[e] : fmaf(sv_raw[e], inv_temp, -shift);
         }
     }
     if (tid >= total && tid < a.max_k) {
@@ -764,6 +774,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
 // ---------------------------------------------------------------------------------------------------------
 struct SbsEpilogueArgs {
     int n_par, W, is_logprob;
+    double inv_temp;           // 1 / temperature of the parents' rows (1: none)
     int32_t first_parent_node;
     uint32_t seed_lo, seed_hi, step, seq_base;
     const int32_t* fin_token;  // [B][n_par][W]
@@ -847,7 +858,7 @@ __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const Sb
             const uint32_t word = coarse_word(key, node, (uint32_t)x >> 4);
             const double t_elem = (((uint32_t)x & 15u) != (word & 15u))
                                       ? neg_log_uniform_f64(fine_word(key, node, (uint32_t)x)) : 0.0;
-            phi = sigma + ((double)a.fin_value[(int64_t)b * F + f] - lse);
+            phi = sigma + ((double)a.fin_value[(int64_t)b * F + f] * a.inv_temp - lse);
             pert = phi - log(neg_log_group_uniform_f64(word) * 0.0625 + t_elem);
         }
         s_tok[f] = x;

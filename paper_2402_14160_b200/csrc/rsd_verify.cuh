@@ -31,6 +31,7 @@ constexpr float kRefSlack = 60.0f;    // redo a pass if the row maximum exceeds 
 struct RowsDev {
     const void* data;
     int64_t seq_stride, row_stride;
+    float inv_temp;   // 1 / sampling temperature of these rows (1: none); values enter as value * inv_temp
 };
 
 struct VerifyArgs {
@@ -123,12 +124,13 @@ __device__ float row_reference(const char* row, int V, bool whole_row, VerifySme
 // (a = 0, no draft row: plain exponentials of the target).  Leaves the sum of every 512-element tile in
 // sm.tile_sum, returns their total (summed in tile order, identically on all threads) and the true row maxima.
 template <typename T, bool ALIGNED, bool WITH_DRAFT>
-__device__ double weight_pass(const char* rowq, const char* rowp, int V, float mq, float mp, float a_hi, float a_lo,
+__device__ double weight_pass(const char* rowq, const char* rowp, int V, float mq, float mp, float kq, float kp,
+                              float a_hi, float a_lo,
                               VerifySmem& sm, bool& saw_nan, float* true_max_q, float* true_max_p) {
     const int n_groups = (V + 15) >> 4;
     const int n_tiles = (n_groups + 31) >> 5;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float cq = mq * kLog2e, cp = mp * kLog2e;
+    const float cq = mq * kq, cp = mp * kp;   // kq, kp = log2(e) / temperature of the row
     float tmq = kNegInf, tmp_ = kNegInf;
     const int n_iter = (n_groups + kVerifyThreads - 1) / kVerifyThreads;
     for (int it = 0; it < n_iter; ++it) {
@@ -142,13 +144,13 @@ __device__ double weight_pass(const char* rowq, const char* rowp, int V, float m
                 tmp_ = fmaxf(tmp_, load_clean<T, ALIGNED>(rowp, g, V, p, saw_nan));
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
-                    const float qh = ex2_approx(fmaf(q[j], kLog2e, -cq));
-                    const float ph = ex2_approx(fmaf(p[j], kLog2e, -cp));
+                    const float qh = ex2_approx(fmaf(q[j], kq, -cq));
+                    const float ph = ex2_approx(fmaf(p[j], kp, -cp));
                     w[j] = residual_weight(qh, ph, a_hi, a_lo);
                 }
             } else {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) w[j] = ex2_approx(fmaf(q[j], kLog2e, -cq));
+                for (int j = 0; j < 16; ++j) w[j] = ex2_approx(fmaf(q[j], kq, -cq));
             }
             gs = tree_sum16(w);
         }
@@ -175,10 +177,11 @@ __device__ double weight_pass(const char* rowq, const char* rowp, int V, float m
 
 // Both normalisers of a node in one pass: S_q = sum exp(lt - m_q), S_p = sum exp(ld - m_p).
 template <typename T, bool ALIGNED>
-__device__ void softmax_sums(const char* rowq, const char* rowp, int V, float mq, float mp, VerifySmem& sm,
+__device__ void softmax_sums(const char* rowq, const char* rowp, int V, float mq, float mp, float kq, float kp,
+                             VerifySmem& sm,
                              bool& saw_nan, double* Sq, double* Sp, float* true_max_q, float* true_max_p) {
     const int n_groups = (V + 15) >> 4;
-    const float cq = mq * kLog2e, cp = mp * kLog2e;
+    const float cq = mq * kq, cp = mp * kp;   // kq, kp = log2(e) / temperature of the row
     float tmq = kNegInf, tmp_ = kNegInf;
     double accq = 0.0, accp = 0.0;
     for (int g = threadIdx.x; g < n_groups; g += kVerifyThreads) {
@@ -187,8 +190,8 @@ __device__ void softmax_sums(const char* rowq, const char* rowp, int V, float mq
         tmp_ = fmaxf(tmp_, load_clean<T, ALIGNED>(rowp, g, V, p, saw_nan));
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-            q[j] = ex2_approx(fmaf(q[j], kLog2e, -cq));
-            p[j] = ex2_approx(fmaf(p[j], kLog2e, -cp));
+            q[j] = ex2_approx(fmaf(q[j], kq, -cq));
+            p[j] = ex2_approx(fmaf(p[j], kp, -cp));
         }
         accq += (double)tree_sum16(q);
         accp += (double)tree_sum16(p);
@@ -202,7 +205,8 @@ __device__ void softmax_sums(const char* rowq, const char* rowp, int V, float mq
 // Inverse CDF over the weights of the last weight_pass: the smallest y whose running sum exceeds u * total; if
 // rounding leaves none, the largest y with positive weight; -1 if there is no weight at all.
 template <typename T, bool ALIGNED, bool WITH_DRAFT>
-__device__ int inverse_cdf_pick(const char* rowq, const char* rowp, int V, float mq, float mp, float a_hi, float a_lo,
+__device__ int inverse_cdf_pick(const char* rowq, const char* rowp, int V, float mq, float mp, float kq, float kp,
+                                float a_hi, float a_lo,
                                 double total, double u, VerifySmem& sm) {
     const int n_groups = (V + 15) >> 4;
     const int n_tiles = (n_groups + 31) >> 5;
@@ -232,14 +236,14 @@ __device__ int inverse_cdf_pick(const char* rowq, const char* rowp, int V, float
             float q[16];
             bool dummy = false;
             load_clean<T, ALIGNED>(rowq, g, V, q, dummy);
-            const float cq = mq * kLog2e, cp = mp * kLog2e;
+            const float cq = mq * kq, cp = mp * kp;   // kq, kp = log2(e) / temperature of the row
             if (WITH_DRAFT) {
                 float p[16];
                 load_clean<T, ALIGNED>(rowp, g, V, p, dummy);
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
-                    const float qh = ex2_approx(fmaf(q[j], kLog2e, -cq));
-                    const float ph = ex2_approx(fmaf(p[j], kLog2e, -cp));
+                    const float qh = ex2_approx(fmaf(q[j], kq, -cq));
+                    const float ph = ex2_approx(fmaf(p[j], kp, -cp));
                     w[j] = residual_weight(qh, ph, a_hi, a_lo);
                 }
                 for (int i = 0; i < sm.n_removed; ++i) {
@@ -250,7 +254,7 @@ __device__ int inverse_cdf_pick(const char* rowq, const char* rowp, int V, float
                 }
             } else {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) w[j] = ex2_approx(fmaf(q[j], kLog2e, -cq));
+                for (int j = 0; j < 16; ++j) w[j] = ex2_approx(fmaf(q[j], kq, -cq));
             }
         }
         const double gs = (double)tree_sum16(w);
@@ -291,7 +295,8 @@ struct NodeChain {
     const char* rowq;
     const char* rowp;
     int V;
-    float mq, mp;
+    float mq, mp;       // reference values (raw units)
+    float kq, kp;       // log2(e) / temperature of the target and draft rows
     double Sq, Sp;      // normalisers relative to the references
     double A, P, Z;     // closed-form chain state
     double total;       // sum of the weights of the last weight_pass (valid if tiles_current)
@@ -305,8 +310,8 @@ struct NodeChain {
     }
 
     // reference maxima and normalisers of the node (both rows)
-    __device__ void open_both(const char* q, const char* p, int V_, VerifySmem& sm, bool& saw_nan) {
-        rowq = q; rowp = p; V = V_; with_draft = true; tiles_current = false;
+    __device__ void open_both(const char* q, const char* p, int V_, float kq_, float kp_, VerifySmem& sm, bool& saw_nan) {
+        rowq = q; rowp = p; V = V_; kq = kq_; kp = kp_; with_draft = true; tiles_current = false;
         A = 0.0; P = 0.0; Z = 1.0; a_hi = a_lo = 0.0f;
         __syncthreads();
         if (threadIdx.x == 0) sm.n_removed = 0;
@@ -317,16 +322,16 @@ struct NodeChain {
         if (!(mp > kNegInf)) mp = row_reference<T, ALIGNED>(rowp, V, true, sm, saw_nan);
         for (int attempt = 0; attempt < 2; ++attempt) {
             float tq, tp;
-            softmax_sums<T, ALIGNED>(rowq, rowp, V, mq, mp, sm, saw_nan, &Sq, &Sp, &tq, &tp);
-            const bool redo = (tq > mq + kRefSlack) || (tp > mp + kRefSlack);
+            softmax_sums<T, ALIGNED>(rowq, rowp, V, mq, mp, kq, kp, sm, saw_nan, &Sq, &Sp, &tq, &tp);
+            const bool redo = ((tq - mq) * kq > kRefSlack * kLog2e) || ((tp - mp) * kp > kRefSlack * kLog2e);
             if (!redo) break;
             mq = tq; mp = tp;
         }
     }
 
     // plain target row: weights exp(lt - m_q), total = S_q, tile sums ready for the draw
-    __device__ void open_target_only(const char* q, int V_, VerifySmem& sm, bool& saw_nan) {
-        rowq = q; rowp = q; V = V_; with_draft = false; tiles_current = true;
+    __device__ void open_target_only(const char* q, int V_, float kq_, VerifySmem& sm, bool& saw_nan) {
+        rowq = q; rowp = q; V = V_; kq = kq_; kp = kq_; with_draft = false; tiles_current = true;
         A = 0.0; P = 0.0; Z = 1.0; a_hi = a_lo = 0.0f; Sp = 1.0; mp = 0.0f;
         __syncthreads();
         if (threadIdx.x == 0) sm.n_removed = 0;
@@ -335,8 +340,8 @@ struct NodeChain {
         if (!(mq > kNegInf)) mq = row_reference<T, ALIGNED>(rowq, V, true, sm, saw_nan);
         for (int attempt = 0; attempt < 2; ++attempt) {
             float tq;
-            total = weight_pass<T, ALIGNED, false>(rowq, rowq, V, mq, 0.0f, 0.0f, 0.0f, sm, saw_nan, &tq, nullptr);
-            if (!(tq > mq + kRefSlack)) break;
+            total = weight_pass<T, ALIGNED, false>(rowq, rowq, V, mq, 0.0f, kq, kq, 0.0f, 0.0f, sm, saw_nan, &tq, nullptr);
+            if (!((tq - mq) * kq > kRefSlack * kLog2e)) break;
             mq = tq;
         }
         Sq = total;
@@ -344,11 +349,11 @@ struct NodeChain {
 
     __device__ double prob_q(int x) const {
         const float l = RowIO<T>::scalar(rowq, x);
-        return (l == l) ? (double)ex2_approx(fmaf(l, kLog2e, -mq * kLog2e)) / Sq : 0.0;
+        return (l == l) ? (double)ex2_approx(fmaf(l, kq, -mq * kq)) / Sq : 0.0;
     }
     __device__ double prob_p(int x) const {
         const float l = RowIO<T>::scalar(rowp, x);
-        return (l == l) ? (double)ex2_approx(fmaf(l, kLog2e, -mp * kLog2e)) / Sp : 0.0;
+        return (l == l) ? (double)ex2_approx(fmaf(l, kp, -mp * kp)) / Sp : 0.0;
     }
 
     // Eq. 3 for the next child x
@@ -367,7 +372,7 @@ struct NodeChain {
         const double A_old = A;
         A = A_new;
         split_a();
-        const double zhat = weight_pass<T, ALIGNED, true>(rowq, rowp, V, mq, mp, a_hi, a_lo, sm, saw_nan, nullptr, nullptr);
+        const double zhat = weight_pass<T, ALIGNED, true>(rowq, rowp, V, mq, mp, kq, kp, a_hi, a_lo, sm, saw_nan, nullptr, nullptr);
         const double Z_new = zhat / Sq;
         if (Z_new > 0.0 && Z_new < 1.7e308) {
             Z = Z_new;
@@ -385,8 +390,8 @@ struct NodeChain {
             const int i = sm.n_removed++;
             const float lq = RowIO<T>::scalar(rowq, x), lp = RowIO<T>::scalar(rowp, x);
             sm.rem_x[i] = x;
-            sm.rem_qh[i] = (lq == lq) ? ex2_approx(fmaf(lq, kLog2e, -mq * kLog2e)) : 0.0f;
-            sm.rem_ph[i] = (lp == lp) ? ex2_approx(fmaf(lp, kLog2e, -mp * kLog2e)) : 0.0f;
+            sm.rem_qh[i] = (lq == lq) ? ex2_approx(fmaf(lq, kq, -mq * kq)) : 0.0f;
+            sm.rem_ph[i] = (lp == lp) ? ex2_approx(fmaf(lp, kp, -mp * kp)) : 0.0f;
             sm.rem_w[i] = residual_weight(sm.rem_qh[i], sm.rem_ph[i], a_hi, a_lo);
         }
         __syncthreads();
@@ -399,13 +404,13 @@ struct NodeChain {
         if (!with_draft || A == 0.0) {
             if (!tiles_current || with_draft) {
                 float tq;
-                total = weight_pass<T, ALIGNED, false>(rowq, rowq, V, mq, 0.0f, 0.0f, 0.0f, sm, saw_nan, &tq, nullptr);
+                total = weight_pass<T, ALIGNED, false>(rowq, rowq, V, mq, 0.0f, kq, kq, 0.0f, 0.0f, sm, saw_nan, &tq, nullptr);
             }
-            return inverse_cdf_pick<T, ALIGNED, false>(rowq, rowq, V, mq, 0.0f, 0.0f, 0.0f, total, u, sm);
+            return inverse_cdf_pick<T, ALIGNED, false>(rowq, rowq, V, mq, 0.0f, kq, kq, 0.0f, 0.0f, total, u, sm);
         }
         if (!tiles_current)
-            total = weight_pass<T, ALIGNED, true>(rowq, rowp, V, mq, mp, a_hi, a_lo, sm, saw_nan, nullptr, nullptr);
-        return inverse_cdf_pick<T, ALIGNED, true>(rowq, rowp, V, mq, mp, a_hi, a_lo, total, u, sm);
+            total = weight_pass<T, ALIGNED, true>(rowq, rowp, V, mq, mp, kq, kp, a_hi, a_lo, sm, saw_nan, nullptr, nullptr);
+        return inverse_cdf_pick<T, ALIGNED, true>(rowq, rowp, V, mq, mp, kq, kp, a_hi, a_lo, total, u, sm);
     }
 };
 
@@ -427,7 +432,7 @@ __device__ int next_child(const int32_t* par, const int32_t* tok, int num_nodes,
 }
 
 template <typename T, bool ALIGNED>
-__global__ void __launch_bounds__(kVerifyThreads) verify_tree_kernel(const VerifyArgs a) {
+__global__ void __launch_bounds__(kVerifyThreads, 4) verify_tree_kernel(const VerifyArgs a) {
     __shared__ VerifySmem sm;
     const int b = blockIdx.x, tid = threadIdx.x;
     const int32_t* par = a.parent + (a.shared_topology ? 0 : (int64_t)b * a.num_nodes);
@@ -450,10 +455,11 @@ __global__ void __launch_bounds__(kVerifyThreads) verify_tree_kernel(const Verif
         int c = next_child(par, tok, a.num_nodes, a.V, cur, 0, sm);
         if (c < 0 || len >= a.L) {
             reason = (len >= a.L) ? 2 : 1;  // RSD_STOP_LEAF : RSD_STOP_NO_CHILDREN
-            chain.open_target_only(row_ptr<T>(a.target, b, cur), a.V, sm, saw_nan);
+            chain.open_target_only(row_ptr<T>(a.target, b, cur), a.V, kLog2e * a.target.inv_temp, sm, saw_nan);
             break;
         }
-        chain.open_both(row_ptr<T>(a.target, b, cur), row_ptr<T>(a.draft, b, cur), a.V, sm, saw_nan);
+        chain.open_both(row_ptr<T>(a.target, b, cur), row_ptr<T>(a.draft, b, cur), a.V, kLog2e * a.target.inv_temp,
+                        kLog2e * a.draft.inv_temp, sm, saw_nan);
         int accepted = -1, j = 0;
         while (c >= 0) {
             const int x = tok[c];
@@ -502,9 +508,9 @@ __global__ void __launch_bounds__(kVerifyThreads) resample_residual_kernel(const
     NodeChain<T, ALIGNED> chain;
     const char* rowq = row_ptr<T>(a.target, b, 0);
     if (n_rej == 0) {
-        chain.open_target_only(rowq, a.V, sm, saw_nan);
+        chain.open_target_only(rowq, a.V, kLog2e * a.target.inv_temp, sm, saw_nan);
     } else {
-        chain.open_both(rowq, row_ptr<T>(a.draft, b, 0), a.V, sm, saw_nan);
+        chain.open_both(rowq, row_ptr<T>(a.draft, b, 0), a.V, kLog2e * a.target.inv_temp, kLog2e * a.draft.inv_temp, sm, saw_nan);
         for (int i = 0; i < a.max_k; ++i) {
             const int x = a.rejected[(int64_t)b * a.max_k + i];
             if (x < 0 || x >= a.V) continue;
@@ -517,16 +523,16 @@ __global__ void __launch_bounds__(kVerifyThreads) resample_residual_kernel(const
     if (a.out_residual) {
         // normalised weights, recomputed element by element
         const bool with_draft = chain.with_draft && chain.A != 0.0;
-        const float cq = chain.mq * kLog2e, cp = chain.mp * kLog2e;
+        const float cq = chain.mq * chain.kq, cp = chain.mp * chain.kp;
         const double inv = chain.total > 0.0 ? 1.0 / chain.total : 0.0;
         for (int x = tid; x < a.V; x += kVerifyThreads) {
             float lq = RowIO<T>::scalar(rowq, x);
             if (lq != lq) lq = kNegInf;
-            float w = ex2_approx(fmaf(lq, kLog2e, -cq));
+            float w = ex2_approx(fmaf(lq, chain.kq, -cq));
             if (with_draft) {
                 float lp = RowIO<T>::scalar(chain.rowp, x);
                 if (lp != lp) lp = kNegInf;
-                const float ph = ex2_approx(fmaf(lp, kLog2e, -cp));
+                const float ph = ex2_approx(fmaf(lp, chain.kp, -cp));
                 w = residual_weight(w, ph, chain.a_hi, chain.a_lo);
                 for (int i = 0; i < sm.n_removed; ++i)
                     if (sm.rem_x[i] == x) w = sm.rem_w[i];

@@ -37,8 +37,12 @@ def close(gpu, ref, rel=REL_TOL, abs_tol=1e-6):
     return ok
 
 
-def compare_topk(tally, gpu_token, ora, k_per_row, gpu_perturbed=None, gpu_logprob=None, skip_seq=None):
-    """Row-wise: picks must match in order; a mismatching row is borderline iff the oracle's smallest gap <= MARGIN."""
+def compare_topk(tally, gpu_token, ora, k_per_row, gpu_perturbed=None, gpu_logprob=None, skip_seq=None,
+                 logprob_abs_tol=1e-6):
+    """Row-wise: picks must match in order; a mismatching row is borderline iff the oracle's smallest gap <= MARGIN.
+
+    logprob_abs_tol: a log-probability (and a perturbed one) is value / T - LSE in fp32; when those two terms are large
+    (low temperature) each carries half an ulp of its own size, which the caller passes here."""
     B, R, _ = gpu_token.shape
     bad_seq = set()
     for b in range(B):
@@ -49,11 +53,11 @@ def compare_topk(tally, gpu_token, ora, k_per_row, gpu_perturbed=None, gpu_logpr
             tally.decisions += k
             if np.array_equal(gpu_token[b, r], ora["token"][b, r]):
                 if gpu_perturbed is not None:
-                    ok = close(gpu_perturbed[b, r, :k], ora["perturbed"][b, r, :k])
+                    ok = close(gpu_perturbed[b, r, :k], ora["perturbed"][b, r, :k], abs_tol=logprob_abs_tol)
                     if not ok.all():
                         tally.failures.append(("perturbed", b, r, gpu_perturbed[b, r, :k], ora["perturbed"][b, r, :k]))
                 if gpu_logprob is not None:
-                    ok = close(gpu_logprob[b, r, :k], ora["logprob"][b, r, :k])
+                    ok = close(gpu_logprob[b, r, :k], ora["logprob"][b, r, :k], abs_tol=logprob_abs_tol)
                     if not ok.all():
                         tally.failures.append(("logprob", b, r, gpu_logprob[b, r, :k], ora["logprob"][b, r, :k]))
                 continue

@@ -300,3 +300,85 @@ def test_resample_residual_matches_oracle(rsd, dtype, V):
     o2 = oracle.resample_residual(None, workloads.as_oracle_rows(tg), None, nodes.cpu().numpy(), 13, 2, seq_base=1)
     assert np.all(np.abs(plain["residual"] - o2["residual"]) <= 1e-5 * o2["residual"].max(axis=1, keepdims=True))
     assert (plain["token"] != o2["token"]).sum() <= 1
+
+
+# ---------------------------------------------------------------------------------------------------------
+# sampling temperature (Section 4: 0.3 and 1.0)
+# ---------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,V,T", [("f32", 4099, 0.3), ("bf16", 32000, 0.3), ("bf16", 515, 0.7), ("f32", 1000, 2.0)])
+def test_gumbel_topk_with_temperature(rsd, dtype, V, T):
+    B, R = 3, 4
+    rows = _rows((B, R, V), dtype, 2.0, 1200 + V)
+    k = [min(V, x) for x in (1, 4, 8, 32)]
+    T = float(np.float32(T))                                     # the library takes the temperature as fp32
+    # value / T and the log-sum-exp are fp32 numbers of this size: two ulps of it bound their difference's error
+    tol = 2.0 * float(np.spacing(np.float32(rows.float().abs().max().item() / T)))
+    g = rsd.rsd_gumbel_topk_draft(rows, k, [0, 3, 7, 11], 9, 2, max_k=max(k), want_values=True, temperature=T)
+    o = oracle.gumbel_topk(workloads.as_oracle_rows(rows), k, [0, 3, 7, 11], 9, 2, max_k=max(k), temperature=T)
+    t = Tally()
+    compare_topk(t, g["token"].cpu().numpy(), o, k, g["perturbed"].cpu().numpy(), g["logprob"].cpu().numpy(),
+                 logprob_abs_tol=tol)
+    t.check()
+    # log-probability rows are re-scored under a temperature: same picks as the raw rows give
+    lp = torch.log_softmax(rows.float(), -1)
+    g2 = rsd.rsd_gumbel_topk_draft(lp, k, [0, 3, 7, 11], 9, 2, max_k=max(k), want_values=True, is_logprob=True,
+                                   temperature=T)
+    o2 = oracle.gumbel_topk(workloads.as_oracle_rows(lp), k, [0, 3, 7, 11], 9, 2, max_k=max(k), is_logprob=True,
+                            temperature=T)
+    t = Tally()
+    compare_topk(t, g2["token"].cpu().numpy(), o2, k, g2["perturbed"].cpu().numpy(), g2["logprob"].cpu().numpy(),
+                 logprob_abs_tol=tol)
+    t.check()
+
+
+@pytest.mark.parametrize("dtype,V,W,L,T", [("bf16", 4099, 8, 4, 0.3), ("f32", 1000, 4, 4, 0.3), ("bf16", 32000, 6, 3, 0.5)])
+def test_sbs_and_walk_with_temperature(rsd, dtype, V, W, L, T):
+    # low temperature sharpens the rows: beams branch inside parents, acceptance tests see tempered ratios
+    B = 8
+    T = float(np.float32(T))
+    P = 1 + (L - 1) * W
+    draft = _rows((B, P, V), dtype, 1.5, 1300 + V)
+    target = (torch.cat([draft.float(), _rows((B, W, V), "f32", 1.5, 1301 + V)], 1)
+              + _rows((B, P + W, V), "f32", 0.5, 1302 + V)).to(draft.dtype)
+    host = workloads.as_oracle_rows(draft)
+    t = Tally()
+    skip = set()
+    g_prev = o_prev = None
+    o_levels = []
+    for l in range(L):
+        first = 0 if l == 0 else 1 + (l - 1) * W
+        n_par = 1 if l == 0 else W
+        g = rsd.rsd_sbs_step(draft[:, first:first + n_par], W, first, None if l == 0 else g_prev["sum_logprob"],
+                             None if l == 0 else g_prev["trunc_gumbel"], 21, 3, temperature=T)
+        o = oracle.sbs_step(host[:, first:first + n_par], W, first, None if l == 0 else o_prev["sum_logprob"],
+                            None if l == 0 else o_prev["trunc_gumbel"], 21, 3, temperature=T)
+        skip |= compare_sbs_level(t, _np(g), o, W, skip)
+        g_prev, o_prev = g, o
+        o_levels.append(o)
+    t.check()
+    parent, token = _sbs_tree(o_levels, W)
+    par_t, tok_t = torch.from_numpy(parent).cuda(), torch.from_numpy(token).cuda()
+    gv = _np(rsd.rsd_verify_tree(draft, target, par_t, tok_t, L, 21, 3, want_theta=True, draft_temperature=T,
+                                 target_temperature=T))
+    ov = oracle.verify_tree(host, workloads.as_oracle_rows(target), parent, token, L, 21, 3, draft_temperature=T,
+                            target_temperature=T)
+    t = Tally()
+    compare_verify(t, gv, ov, parent)
+    t.check()
+    # and with different temperatures for the two models
+    gv = _np(rsd.rsd_verify_tree(draft, target, par_t, tok_t, L, 21, 3, want_theta=True, draft_temperature=T,
+                                 target_temperature=1.0))
+    ov = oracle.verify_tree(host, workloads.as_oracle_rows(target), parent, token, L, 21, 3, draft_temperature=T)
+    t = Tally()
+    compare_verify(t, gv, ov, parent)
+    t.check()
+
+
+def test_temperature_arguments_are_checked(rsd):
+    rows = _rows((1, 1, 64), "f32", 1.0, 1)
+    for bad in (-0.5, float("nan"), float("inf")):
+        with pytest.raises(rsd.RsdError, match="temperature"):
+            rsd.rsd_gumbel_topk_draft(rows, [1], [0], seed=0, step=0, temperature=bad)
+    a = rsd.rsd_gumbel_topk_draft(rows, [4], [0], seed=0, step=0, temperature=0.0)     # 0 = none
+    b = rsd.rsd_gumbel_topk_draft(rows, [4], [0], seed=0, step=0)
+    assert torch.equal(a["token"], b["token"])
