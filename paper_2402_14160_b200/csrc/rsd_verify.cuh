@@ -82,19 +82,50 @@ __device__ __forceinline__ const char* row_ptr(const RowsDev& r, int b, int node
     return (const char*)r.data + ((int64_t)b * r.seq_stride + (int64_t)node * r.row_stride) * RowIO<T>::kBytes;
 }
 
+// Sum of 16 weights in a fixed order: four packed additions fold the eight (even, odd) pairs, the two halves last.
 __device__ __forceinline__ float tree_sum16(const float (&w)[16]) {
-    const float a0 = w[0] + w[1], a1 = w[2] + w[3], a2 = w[4] + w[5], a3 = w[6] + w[7];
-    const float a4 = w[8] + w[9], a5 = w[10] + w[11], a6 = w[12] + w[13], a7 = w[14] + w[15];
-    return ((a0 + a1) + (a2 + a3)) + ((a4 + a5) + (a6 + a7));
+    const unsigned long long x0 = add_f32x2(f32x2(w[0], w[1]), f32x2(w[2], w[3]));
+    const unsigned long long x1 = add_f32x2(f32x2(w[4], w[5]), f32x2(w[6], w[7]));
+    const unsigned long long x2 = add_f32x2(f32x2(w[8], w[9]), f32x2(w[10], w[11]));
+    const unsigned long long x3 = add_f32x2(f32x2(w[12], w[13]), f32x2(w[14], w[15]));
+    float lo, hi;
+    split_f32x2(add_f32x2(add_f32x2(x0, x1), add_f32x2(x2, x3)), lo, hi);
+    return lo + hi;
+}
+
+// exp2(v * k - c) of 16 values, two per fma
+__device__ __forceinline__ void exp16(const float (&v)[16], float k, float c, float (&e)[16]) {
+    const unsigned long long k2 = f32x2(k, k), c2 = f32x2(-c, -c);
+#pragma unroll
+    for (int j = 0; j < 16; j += 2) {
+        float a, b;
+        split_f32x2(fma_f32x2(f32x2(v[j], v[j + 1]), k2, c2), a, b);
+        e[j] = ex2_approx(a);
+        e[j + 1] = ex2_approx(b);
+    }
+}
+
+// (qh - a ph)+ for 16 pairs; a = a_hi + a_lo, applied as in residual_weight()
+__device__ __forceinline__ void residual16(const float (&qh)[16], const float (&ph)[16], float a_hi, float a_lo,
+                                           float (&w)[16]) {
+    const unsigned long long nh = f32x2(-a_hi, -a_hi), nl = f32x2(-a_lo, -a_lo);
+#pragma unroll
+    for (int j = 0; j < 16; j += 2) {
+        const unsigned long long p2 = f32x2(ph[j], ph[j + 1]);
+        float a, b;
+        split_f32x2(fma_f32x2(p2, nl, fma_f32x2(p2, nh, f32x2(qh[j], qh[j + 1]))), a, b);
+        w[j] = fmaxf(a, 0.0f);
+        w[j + 1] = fmaxf(b, 0.0f);
+    }
 }
 
 // load a group, turn NaN into -inf (reported), return the group's maximum
 template <typename T, bool ALIGNED>
 __device__ __forceinline__ float load_clean(const char* row, int g, int V, float (&v)[16], bool& saw_nan) {
-    load_group<T, ALIGNED>(row, g, V, v);
-    float m = kNegInf;
-#pragma unroll
-    for (int j = 0; j < 16; ++j) m = max_nan(m, v[j]);
+    Packed<T> pk;
+    pk.load(row, g, V, ALIGNED && (g + 1) * 16 <= V);
+    float m = group_max_nan(pk);   // packed maxima for bf16; NaN if any element is NaN
+    pk.unpack(v);
     if (m != m) {
         saw_nan = true;
         m = kNegInf;
@@ -142,15 +173,11 @@ __device__ double weight_pass(const char* rowq, const char* rowp, int V, float m
             if (WITH_DRAFT) {
                 float p[16];
                 tmp_ = fmaxf(tmp_, load_clean<T, ALIGNED>(rowp, g, V, p, saw_nan));
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float qh = ex2_approx(fmaf(q[j], kq, -cq));
-                    const float ph = ex2_approx(fmaf(p[j], kp, -cp));
-                    w[j] = residual_weight(qh, ph, a_hi, a_lo);
-                }
+                exp16(q, kq, cq, q);
+                exp16(p, kp, cp, p);
+                residual16(q, p, a_hi, a_lo, w);
             } else {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) w[j] = ex2_approx(fmaf(q[j], kq, -cq));
+                exp16(q, kq, cq, w);
             }
             gs = tree_sum16(w);
         }
@@ -188,11 +215,8 @@ __device__ void softmax_sums(const char* rowq, const char* rowp, int V, float mq
         float q[16], p[16];
         tmq = fmaxf(tmq, load_clean<T, ALIGNED>(rowq, g, V, q, saw_nan));
         tmp_ = fmaxf(tmp_, load_clean<T, ALIGNED>(rowp, g, V, p, saw_nan));
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            q[j] = ex2_approx(fmaf(q[j], kq, -cq));
-            p[j] = ex2_approx(fmaf(p[j], kp, -cp));
-        }
+        exp16(q, kq, cq, q);
+        exp16(p, kp, cp, p);
         accq += (double)tree_sum16(q);
         accp += (double)tree_sum16(p);
     }
@@ -240,12 +264,9 @@ __device__ int inverse_cdf_pick(const char* rowq, const char* rowp, int V, float
             if (WITH_DRAFT) {
                 float p[16];
                 load_clean<T, ALIGNED>(rowp, g, V, p, dummy);
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float qh = ex2_approx(fmaf(q[j], kq, -cq));
-                    const float ph = ex2_approx(fmaf(p[j], kp, -cp));
-                    w[j] = residual_weight(qh, ph, a_hi, a_lo);
-                }
+                exp16(q, kq, cq, q);
+                exp16(p, kp, cp, p);
+                residual16(q, p, a_hi, a_lo, w);
                 for (int i = 0; i < sm.n_removed; ++i) {
                     if ((sm.rem_x[i] >> 4) != g) continue;
 #pragma unroll
@@ -253,8 +274,7 @@ __device__ int inverse_cdf_pick(const char* rowq, const char* rowp, int V, float
                         if (j == (sm.rem_x[i] & 15)) w[j] = sm.rem_w[i];
                 }
             } else {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) w[j] = ex2_approx(fmaf(q[j], kq, -cq));
+                exp16(q, kq, cq, w);
             }
         }
         const double gs = (double)tree_sum16(w);
