@@ -123,7 +123,8 @@ __device__ __forceinline__ void residual16(const float (&qh)[16], const float (&
 template <typename T, bool ALIGNED>
 __device__ __forceinline__ float load_clean(const char* row, int g, int V, float (&v)[16], bool& saw_nan) {
     Packed<T> pk;
-    pk.load(row, g, V, ALIGNED && (g + 1) * 16 <= V);
+    // rows on 32-byte boundaries take 256-bit loads (a group is 32 or 64 bytes, so every group of the row is aligned)
+    pk.load(row, g, V, ALIGNED && (g + 1) * 16 <= V, ((uintptr_t)row & 31u) == 0);
     float m = group_max_nan(pk);   // packed maxima for bf16; NaN if any element is NaN
     pk.unpack(v);
     if (m != m) {
