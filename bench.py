@@ -29,7 +29,7 @@ import workloads  # noqa: E402
 # DRAM bytes moved per algorithmic byte by the scan kernel, from the ncu capture summarised in
 # profiles/scan_topk_kernel_workload5_256seq.md (dram__bytes_read + dram__bytes_write over rows x V x 2 bytes; the
 # traffic grows in proportion to the rows scanned).  Set to None whenever the kernel changes after a capture.
-SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.035
+SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.042
 
 METRIC = "verified tree nodes/sec"
 UNIT = "nodes/s"
