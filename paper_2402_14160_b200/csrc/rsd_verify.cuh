@@ -22,10 +22,21 @@
 
 namespace rsd {
 
-constexpr int kVerifyThreads = 256;
+#ifndef RSD_VERIFY_MIN_BLOCKS
+#define RSD_VERIFY_MIN_BLOCKS 3       // blocks per SM the walk is compiled for, 2-byte rows
+#endif
+#ifndef RSD_VERIFY_MIN_BLOCKS_F32
+#define RSD_VERIFY_MIN_BLOCKS_F32 2   // 4-byte rows: a group in flight is 16 registers per row
+#endif
+#ifndef RSD_VERIFY_THREADS
+#define RSD_VERIFY_THREADS 256
+#endif
+constexpr int kVerifyThreads = RSD_VERIFY_THREADS;
 constexpr int kVerifyWarps = kVerifyThreads / 32;
 constexpr int kMaxTiles = 512;        // tiles of 512 elements: V <= 262144
+constexpr int kMaxCachedNodes = 384;  // trees up to this size are copied to shared memory
 constexpr int kMaxRemoved = 32;      // removed tokens tracked per node (later ones carry no residual mass)
+constexpr int kPassUnroll = 4;        // turns of a pass whose warp-wide sums are taken together
 constexpr float kRefSlack = 60.0f;    // redo a pass if the row maximum exceeds its reference by more than this
 
 struct RowsDev {
@@ -62,12 +73,13 @@ struct ResampleArgs {
 
 struct VerifySmem {
     double tile_sum[kMaxTiles];
-    double red_d[kVerifyWarps];
-    float red_f[kVerifyWarps];
+    double red_d[kVerifyWarps], red_d2[kVerifyWarps];
+    float red_f[kVerifyWarps], red_f2[kVerifyWarps];
     int red_i[kVerifyWarps];
     int nan_flag;
     int pick;
     // tokens removed from the draft at the current node: index, the two exponentials, and the weight frozen at removal
+    int par[kMaxCachedNodes], tok[kMaxCachedNodes];   // the sequence's tree (small trees only)
     int n_removed;
     int rem_x[kMaxRemoved];
     float rem_qh[kMaxRemoved], rem_ph[kMaxRemoved], rem_w[kMaxRemoved];
@@ -119,12 +131,16 @@ __device__ __forceinline__ void residual16(const float (&qh)[16], const float (&
     }
 }
 
-// load a group, turn NaN into -inf (reported), return the group's maximum
+// raw load of group g; rows on 32-byte boundaries take 256-bit loads (a group is 32 or 64 bytes, so every group of
+// such a row is aligned)
 template <typename T, bool ALIGNED>
-__device__ __forceinline__ float load_clean(const char* row, int g, int V, float (&v)[16], bool& saw_nan) {
-    Packed<T> pk;
-    // rows on 32-byte boundaries take 256-bit loads (a group is 32 or 64 bytes, so every group of the row is aligned)
+__device__ __forceinline__ void load_raw(Packed<T>& pk, const char* row, int g, int V) {
     pk.load(row, g, V, ALIGNED && (g + 1) * 16 <= V, ((uintptr_t)row & 31u) == 0);
+}
+
+// unpack a loaded group, turn NaN into -inf (reported), return the group's maximum
+template <typename T>
+__device__ __forceinline__ float clean(const Packed<T>& pk, float (&v)[16], bool& saw_nan) {
     float m = group_max_nan(pk);   // packed maxima for bf16; NaN if any element is NaN
     pk.unpack(v);
     if (m != m) {
@@ -137,6 +153,14 @@ __device__ __forceinline__ float load_clean(const char* row, int g, int V, float
         }
     }
     return m;
+}
+
+// load a group, turn NaN into -inf (reported), return the group's maximum
+template <typename T, bool ALIGNED>
+__device__ __forceinline__ float load_clean(const char* row, int g, int V, float (&v)[16], bool& saw_nan) {
+    Packed<T> pk;
+    load_raw<T, ALIGNED>(pk, row, g, V);
+    return clean<T>(pk, v, saw_nan);
 }
 
 // Row maximum over the first block-wide sweep (cheap reference), or over the whole row when asked.
@@ -162,29 +186,51 @@ __device__ double weight_pass(const char* rowq, const char* rowp, int V, float m
     const int n_groups = (V + 15) >> 4;
     const int n_tiles = (n_groups + 31) >> 5;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float cq = mq * kq, cp = mp * kp;   // kq, kp = log2(e) / temperature of the row
+    const float cq_ = mq * kq, cp_ = mp * kp;   // kq, kp = log2(e) / temperature of the row
     float tmq = kNegInf, tmp_ = kNegInf;
     const int n_iter = (n_groups + kVerifyThreads - 1) / kVerifyThreads;
-    for (int it = 0; it < n_iter; ++it) {
-        const int g = it * kVerifyThreads + threadIdx.x;
-        float gs = 0.0f;
-        if (g < n_groups) {
-            float q[16], w[16];
-            tmq = fmaxf(tmq, load_clean<T, ALIGNED>(rowq, g, V, q, saw_nan));
-            if (WITH_DRAFT) {
-                float p[16];
-                tmp_ = fmaxf(tmp_, load_clean<T, ALIGNED>(rowp, g, V, p, saw_nan));
-                exp16(q, kq, cq, q);
-                exp16(p, kp, cp, p);
-                residual16(q, p, a_hi, a_lo, w);
-            } else {
-                exp16(q, kq, cq, w);
+    // The groups of the next turn are loaded before the current ones are worked on, and the warp-wide sums of
+    // kPassUnroll turns are taken together: a block that has an SM to itself (the long walks at the end of a launch)
+    // is otherwise idle for one load latency plus one chain of shuffles per turn.
+    Packed<T> nq, np;
+    if ((int)threadIdx.x < n_groups) {
+        load_raw<T, ALIGNED>(nq, rowq, threadIdx.x, V);
+        if (WITH_DRAFT) load_raw<T, ALIGNED>(np, rowp, threadIdx.x, V);
+    }
+    for (int it0 = 0; it0 < n_iter; it0 += kPassUnroll) {
+        float gs[kPassUnroll];
+#pragma unroll
+        for (int u = 0; u < kPassUnroll; ++u) {
+            const int g = (it0 + u) * kVerifyThreads + threadIdx.x;
+            gs[u] = 0.0f;
+            if (it0 + u < n_iter) {
+                const Packed<T> cq = nq, cp = np;
+                if (g + kVerifyThreads < n_groups) {
+                    load_raw<T, ALIGNED>(nq, rowq, g + kVerifyThreads, V);
+                    if (WITH_DRAFT) load_raw<T, ALIGNED>(np, rowp, g + kVerifyThreads, V);
+                }
+                if (g < n_groups) {
+                    float q[16], w[16];
+                    tmq = fmaxf(tmq, clean<T>(cq, q, saw_nan));
+                    if (WITH_DRAFT) {
+                        float p[16];
+                        tmp_ = fmaxf(tmp_, clean<T>(cp, p, saw_nan));
+                        exp16(q, kq, cq_, q);
+                        exp16(p, kp, cp_, p);
+                        residual16(q, p, a_hi, a_lo, w);
+                    } else {
+                        exp16(q, kq, cq_, w);
+                    }
+                    gs[u] = tree_sum16(w);
+                }
             }
-            gs = tree_sum16(w);
         }
-        const double ts = warp_sum((double)gs);
-        const int tile = it * kVerifyWarps + warp;
-        if (lane == 0 && tile < n_tiles) sm.tile_sum[tile] = ts;
+#pragma unroll
+        for (int u = 0; u < kPassUnroll; ++u) {
+            const double ts = warp_sum((double)gs[u]);
+            const int tile = (it0 + u) * kVerifyWarps + warp;
+            if (lane == 0 && tile < n_tiles) sm.tile_sum[tile] = ts;
+        }
     }
     if (true_max_q) *true_max_q = block_max<kVerifyThreads>(tmq, sm.red_f);
     if (true_max_p) *true_max_p = block_max<kVerifyThreads>(tmp_, sm.red_f);
@@ -198,9 +244,10 @@ __device__ double weight_pass(const char* rowq, const char* rowp, int V, float m
         }
         __syncthreads();
     }
-    double total = 0.0;
-    for (int t = 0; t < n_tiles; ++t) total += sm.tile_sum[t];
-    return total;
+    // total in a fixed order (strided partial sums, then warps), the same on every thread
+    double part = 0.0;
+    for (int t = threadIdx.x; t < n_tiles; t += kVerifyThreads) part += sm.tile_sum[t];
+    return block_sum<kVerifyThreads>(part, sm.red_d);
 }
 
 // Both normalisers of a node in one pass: S_q = sum exp(lt - m_q), S_p = sum exp(ld - m_p).
@@ -212,19 +259,52 @@ __device__ void softmax_sums(const char* rowq, const char* rowp, int V, float mq
     const float cq = mq * kq, cp = mp * kp;   // kq, kp = log2(e) / temperature of the row
     float tmq = kNegInf, tmp_ = kNegInf;
     double accq = 0.0, accp = 0.0;
+    Packed<T> nq, np;
+    if ((int)threadIdx.x < n_groups) {
+        load_raw<T, ALIGNED>(nq, rowq, threadIdx.x, V);
+        load_raw<T, ALIGNED>(np, rowp, threadIdx.x, V);
+    }
     for (int g = threadIdx.x; g < n_groups; g += kVerifyThreads) {
+        const Packed<T> cq_raw = nq, cp_raw = np;
+        if (g + kVerifyThreads < n_groups) {   // next turn's groups first
+            load_raw<T, ALIGNED>(nq, rowq, g + kVerifyThreads, V);
+            load_raw<T, ALIGNED>(np, rowp, g + kVerifyThreads, V);
+        }
         float q[16], p[16];
-        tmq = fmaxf(tmq, load_clean<T, ALIGNED>(rowq, g, V, q, saw_nan));
-        tmp_ = fmaxf(tmp_, load_clean<T, ALIGNED>(rowp, g, V, p, saw_nan));
+        tmq = fmaxf(tmq, clean<T>(cq_raw, q, saw_nan));
+        tmp_ = fmaxf(tmp_, clean<T>(cp_raw, p, saw_nan));
         exp16(q, kq, cq, q);
         exp16(p, kp, cp, p);
         accq += (double)tree_sum16(q);
         accp += (double)tree_sum16(p);
     }
-    *Sq = block_sum<kVerifyThreads>(accq, sm.red_d);
-    *Sp = block_sum<kVerifyThreads>(accp, sm.red_d);
-    *true_max_q = block_max<kVerifyThreads>(tmq, sm.red_f);
-    *true_max_p = block_max<kVerifyThreads>(tmp_, sm.red_f);
+    // the four block-wide results behind one pair of barriers
+    accq = warp_sum(accq);
+    accp = warp_sum(accp);
+    tmq = warp_max(tmq);
+    tmp_ = warp_max(tmp_);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) {
+        const int w = threadIdx.x >> 5;
+        sm.red_d[w] = accq;
+        sm.red_d2[w] = accp;
+        sm.red_f[w] = tmq;
+        sm.red_f2[w] = tmp_;
+    }
+    __syncthreads();
+    double sq = 0.0, sp = 0.0;
+    float xq = sm.red_f[0], xp = sm.red_f2[0];
+#pragma unroll
+    for (int w = 0; w < kVerifyWarps; ++w) {   // fixed order: the same on every thread
+        sq += sm.red_d[w];
+        sp += sm.red_d2[w];
+        xq = fmaxf(xq, sm.red_f[w]);
+        xp = fmaxf(xp, sm.red_f2[w]);
+    }
+    *Sq = sq;
+    *Sp = sp;
+    *true_max_q = xq;
+    *true_max_p = xp;
 }
 
 // Inverse CDF over the weights of the last weight_pass: the smallest y whose running sum exceeds u * total; if
@@ -337,8 +417,25 @@ struct NodeChain {
         __syncthreads();
         if (threadIdx.x == 0) sm.n_removed = 0;
         __syncthreads();
-        mq = row_reference<T, ALIGNED>(rowq, V, false, sm, saw_nan);
-        mp = row_reference<T, ALIGNED>(rowp, V, false, sm, saw_nan);
+        {   // first sweep of both rows, both loads in flight together, one pair of barriers
+            float a = kNegInf, c = kNegInf;
+            if ((int)threadIdx.x < ((V + 15) >> 4)) {
+                Packed<T> pq, pp;
+                load_raw<T, ALIGNED>(pq, rowq, threadIdx.x, V);
+                load_raw<T, ALIGNED>(pp, rowp, threadIdx.x, V);
+                float v[16];
+                a = clean<T>(pq, v, saw_nan);
+                c = clean<T>(pp, v, saw_nan);
+            }
+            a = warp_max(a);
+            c = warp_max(c);
+            if ((threadIdx.x & 31) == 0) { sm.red_f[threadIdx.x >> 5] = a; sm.red_f2[threadIdx.x >> 5] = c; }
+            __syncthreads();
+            mq = sm.red_f[0];
+            mp = sm.red_f2[0];
+#pragma unroll
+            for (int w = 1; w < kVerifyWarps; ++w) { mq = fmaxf(mq, sm.red_f[w]); mp = fmaxf(mp, sm.red_f2[w]); }
+        }
         if (!(mq > kNegInf)) mq = row_reference<T, ALIGNED>(rowq, V, true, sm, saw_nan);
         if (!(mp > kNegInf)) mp = row_reference<T, ALIGNED>(rowp, V, true, sm, saw_nan);
         for (int attempt = 0; attempt < 2; ++attempt) {
@@ -368,27 +465,26 @@ struct NodeChain {
         Sq = total;
     }
 
-    __device__ double prob_q(int x) const {
-        const float l = RowIO<T>::scalar(rowq, x);
+    // probabilities of a token from its two row values (loaded by the caller, usually one pass early)
+    __device__ double prob_q(float l) const {
         return (l == l) ? (double)ex2_approx(fmaf(l, kq, -mq * kq)) / Sq : 0.0;
     }
-    __device__ double prob_p(int x) const {
-        const float l = RowIO<T>::scalar(rowp, x);
+    __device__ double prob_p(float l) const {
         return (l == l) ? (double)ex2_approx(fmaf(l, kp, -mp * kp)) / Sp : 0.0;
     }
 
-    // Eq. 3 for the next child x
-    __device__ double threshold(int x, int& st) const {
-        const double qx = prob_q(x), px = prob_p(x);
+    // Eq. 3 for the next child, given its target and draft row values
+    __device__ double threshold(float lq, float lp, int& st) const {
+        const double qx = prob_q(lq), px = prob_p(lp);
         const double r = fmax(qx - A * px, 0.0);
         if (px > 0.0) return fmin(1.0, r * (1.0 - P) / (Z * px));
         st |= 8;  // RSD_ST_ZERO_DRAFT_PROB
         return r > 0.0 ? 1.0 : 0.0;
     }
 
-    // Eqs. 1-2 after rejecting x.  Returns false if the draft has no mass left.
-    __device__ bool reject(int x, VerifySmem& sm, bool& saw_nan, int& st) {
-        const double px = prob_p(x);
+    // Eqs. 1-2 after rejecting x (row values lq, lp).  Returns false if the draft has no mass left.
+    __device__ bool reject(int x, float lq, float lp, VerifySmem& sm, bool& saw_nan, int& st) {
+        const double px = prob_p(lp);
         const double A_new = A + Z / (1.0 - P);
         const double A_old = A;
         A = A_new;
@@ -409,7 +505,6 @@ struct NodeChain {
         __syncthreads();
         if (threadIdx.x == 0 && sm.n_removed < kMaxRemoved) {
             const int i = sm.n_removed++;
-            const float lq = RowIO<T>::scalar(rowq, x), lp = RowIO<T>::scalar(rowp, x);
             sm.rem_x[i] = x;
             sm.rem_qh[i] = (lq == lq) ? ex2_approx(fmaf(lq, kq, -mq * kq)) : 0.0f;
             sm.rem_ph[i] = (lp == lp) ? ex2_approx(fmaf(lp, kp, -mp * kp)) : 0.0f;
@@ -435,8 +530,20 @@ struct NodeChain {
     }
 };
 
-// smallest node c > after with parent[c] == cur and a token in [0, V), or -1
+// smallest node c > after with parent[c] == cur and a token in [0, V), or -1.  Trees of up to kMaxCachedNodes nodes
+// sit in shared memory and every warp searches them by itself (no barrier); larger trees are searched in global
+// memory by the whole block.
 __device__ int next_child(const int32_t* par, const int32_t* tok, int num_nodes, int V, int cur, int after, VerifySmem& sm) {
+    if (num_nodes <= kMaxCachedNodes) {
+        const int lane = threadIdx.x & 31;
+        for (int c0 = after + 1; c0 < num_nodes; c0 += 32) {
+            const int c = c0 + lane;
+            const bool ok = c < num_nodes && sm.par[c] == cur && sm.tok[c] >= 0 && sm.tok[c] < V;
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, ok);
+            if (m) return c0 + __ffs(m) - 1;
+        }
+        return -1;
+    }
     int best = 0x7FFFFFFF;
     for (int c = after + 1 + (int)threadIdx.x; c < num_nodes; c += kVerifyThreads) {
         if (par[c] == cur && tok[c] >= 0 && tok[c] < V) { best = c; break; }
@@ -453,7 +560,8 @@ __device__ int next_child(const int32_t* par, const int32_t* tok, int num_nodes,
 }
 
 template <typename T, bool ALIGNED>
-__global__ void __launch_bounds__(kVerifyThreads, 4) verify_tree_kernel(const VerifyArgs a) {
+__global__ void __launch_bounds__(kVerifyThreads, sizeof(T) == 2 ? RSD_VERIFY_MIN_BLOCKS : RSD_VERIFY_MIN_BLOCKS_F32)
+verify_tree_kernel(const VerifyArgs a) {
     __shared__ VerifySmem sm;
     const int b = blockIdx.x, tid = threadIdx.x;
     const int32_t* par = a.parent + (a.shared_topology ? 0 : (int64_t)b * a.num_nodes);
@@ -468,6 +576,9 @@ __global__ void __launch_bounds__(kVerifyThreads, 4) verify_tree_kernel(const Ve
     }
     if (a.dbg_theta)
         for (int n = tid; n < a.num_nodes; n += kVerifyThreads) a.dbg_theta[(int64_t)b * a.num_nodes + n] = __int_as_float(0x7FC00000);
+    const bool cached = a.num_nodes <= kMaxCachedNodes;
+    if (cached)
+        for (int n = tid; n < a.num_nodes; n += kVerifyThreads) { sm.par[n] = par[n]; sm.tok[n] = tok[n]; }
     __syncthreads();
 
     NodeChain<T, ALIGNED> chain;
@@ -479,24 +590,26 @@ __global__ void __launch_bounds__(kVerifyThreads, 4) verify_tree_kernel(const Ve
             chain.open_target_only(row_ptr<T>(a.target, b, cur), a.V, kLog2e * a.target.inv_temp, sm, saw_nan);
             break;
         }
-        chain.open_both(row_ptr<T>(a.target, b, cur), row_ptr<T>(a.draft, b, cur), a.V, kLog2e * a.target.inv_temp,
-                        kLog2e * a.draft.inv_temp, sm, saw_nan);
+        const char* rowq = row_ptr<T>(a.target, b, cur);
+        const char* rowp = row_ptr<T>(a.draft, b, cur);
+        chain.open_both(rowq, rowp, a.V, kLog2e * a.target.inv_temp, kLog2e * a.draft.inv_temp, sm, saw_nan);
         int accepted = -1, j = 0;
         while (c >= 0) {
-            const int x = tok[c];
-            const double theta = chain.threshold(x, st);
+            const int x = cached ? sm.tok[c] : tok[c];
+            const float lq = RowIO<T>::scalar(rowq, x), lp = RowIO<T>::scalar(rowp, x);
+            const double theta = chain.threshold(lq, lp, st);
             const uint4 rw = rng_draw(key, (uint32_t)cur, kTagAccept, (uint32_t)j);
             const double U = (double)(rw.x >> 8) * (1.0 / 16777216.0);
             if (a.dbg_theta && tid == 0) a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)theta;
             if (U < theta) { accepted = c; break; }
-            if (!chain.reject(x, sm, saw_nan, st)) break;
+            if (!chain.reject(x, lq, lp, sm, saw_nan, st)) break;
             ++j;
             c = next_child(par, tok, a.num_nodes, a.V, cur, c, sm);
         }
         if (accepted < 0) { reason = 0; break; }  // RSD_STOP_ALL_REJECTED
         if (tid == 0) {
             a.accepted_node[(int64_t)b * a.L + len] = accepted;
-            a.accepted_token[(int64_t)b * a.L + len] = tok[accepted];
+            a.accepted_token[(int64_t)b * a.L + len] = cached ? sm.tok[accepted] : tok[accepted];
         }
         ++len;
         cur = accepted;
@@ -535,7 +648,7 @@ __global__ void __launch_bounds__(kVerifyThreads) resample_residual_kernel(const
         for (int i = 0; i < a.max_k; ++i) {
             const int x = a.rejected[(int64_t)b * a.max_k + i];
             if (x < 0 || x >= a.V) continue;
-            if (!chain.reject(x, sm, saw_nan, st)) break;
+            if (!chain.reject(x, RowIO<T>::scalar(rowq, x), RowIO<T>::scalar(chain.rowp, x), sm, saw_nan, st)) break;
         }
     }
     const uint4 rw = rng_draw(key, (uint32_t)a.rng_node[b], kTagResample, 0u);
