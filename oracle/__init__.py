@@ -135,6 +135,19 @@ def rrs_chain(p, q, tokens):
     return theta, res, st
 
 
+def baseline_chain(rule, p, q, tokens, gamma=1.0):
+    """theta[k] and the all-rejected residual of a baseline verifier (RULE_MULTIROUND or RULE_KSEQ) for an
+    ordered tuple of independent drafts (Section 2)."""
+    p = np.ascontiguousarray(p, dtype=np.float64)
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    t = _i32(tokens)
+    theta = np.zeros(len(t), dtype=np.float64)
+    res = np.zeros(p.shape[0], dtype=np.float64)
+    st = lib().rsd_oracle_baseline_chain(C.c_int(int(rule)), C.c_double(float(gamma)), _ptr(p), _ptr(q),
+                                         C.c_int(p.shape[0]), _ptr(t), C.c_int(len(t)), _ptr(theta), _ptr(res))
+    return theta, res, st
+
+
 def gumbel_topk(rows, k_per_row, rng_node, seed, step, *, is_logprob=False, seq_base=0, max_k=None,
                 temperature=1.0):
     """rows [B,R,V]; returns dict(token[B,R,max_k], perturbed, logprob, margin[B,R], status[B])."""
@@ -180,9 +193,14 @@ def sbs_step(rows, W, first_parent_node, sum_logprob_in, trunc_gumbel_in, seed, 
     return dict(token=tok, parent=par, sum_logprob=so, trunc_gumbel=go, count=cnt, margin=margin, status=status)
 
 
+RULE_RRS, RULE_MULTIROUND, RULE_KSEQ = 0, 1, 2
+
+
 def verify_tree(draft, target, parent, token, num_levels, seed, step, *, seq_base=0, want_weights=False,
-                draft_temperature=1.0, target_temperature=1.0):
-    """draft [B,P,V], target [B,N+1,V], parent [N+1] or [B,N+1] (flat, root -1), token [B,N+1]."""
+                draft_temperature=1.0, target_temperature=1.0, rule=RULE_RRS, gamma=1.0):
+    """draft [B,P,V], target [B,N+1,V], parent [N+1] or [B,N+1] (flat, root -1), token [B,N+1].
+    rule: recursive rejection sampling (the paper's), or one of the two baselines of Section 2 on the same tree:
+    multi-round rejection sampling with one draft model, K-SEQ with parameter gamma."""
     d, ddt = _rows(draft)
     t, tdt = _rows(target)
     B, _, V = t.shape
@@ -201,7 +219,8 @@ def verify_tree(draft, target, parent, token, num_levels, seed, step, *, seq_bas
     fmargin = np.zeros(B, np.float64)
     weights = np.zeros((B, V), np.float64) if want_weights else None
     status = np.zeros(B, np.int32)
-    lib().rsd_oracle_verify_tree(_ptr(d), C.c_int(ddt), C.c_int64(d.strides[0] // d.itemsize),
+    lib().rsd_oracle_verify_tree_rule(C.c_int(int(rule)), C.c_double(float(gamma)),
+                                 _ptr(d), C.c_int(ddt), C.c_int64(d.strides[0] // d.itemsize),
                                  C.c_int64(d.strides[1] // d.itemsize), C.c_double(draft_temperature),
                                  _ptr(t), C.c_int(tdt), C.c_int64(t.strides[0] // t.itemsize),
                                  C.c_int64(t.strides[1] // t.itemsize), C.c_double(target_temperature),

@@ -420,6 +420,93 @@ static int rrs_reject(double* q, double* p, int V, int x, int* st) {
 }
 
 /*
+ * Multi-round rejection sampling (Section 2, the SpecInfer paragraph) with one
+ * draft model, p^(k) = p for every k: the children are independent draws from
+ * p (repeats allowed), the threshold is min{1, q^(k)(x)/p(x)} and the residual
+ * q^(k+1) = Norm[(q^(k) - p)+].  The draft is never changed.
+ */
+static void multiround_reject(double* q, const double* p, int V, int* st) {
+    double s = 0.0;
+    for (int y = 0; y < V; ++y) {
+        double r = q[y] - p[y];
+        s += (r > 0.0 ? r : 0.0);
+    }
+    if (s > 0.0 && isfinite(s)) {
+        for (int y = 0; y < V; ++y) {
+            double r = q[y] - p[y];
+            q[y] = (r > 0.0 ? r : 0.0) / s;
+        }
+    } else {
+        *st |= ORC_ST_ZERO_RESIDUAL;
+    }
+}
+
+/*
+ * K-sequential draft selection (Section 2, the SpecTr paragraph): each of the
+ * K independent drafts x ~ p is accepted with probability
+ * min{1, q(x) / (gamma p(x))}; if all K are rejected the token comes from
+ * Norm[q - min{p, q/gamma} (1 - (1 - beta)^K) / beta],  beta = sum_x min{p(x), q(x)/gamma}.
+ * Negative entries (a gamma too small for these p, q, K) are clamped to 0.
+ */
+static double kseq_threshold(const double* q, const double* p, double gamma, int x, int* st) {
+    if (p[x] > 0.0) {
+        double r = q[x] / (gamma * p[x]);
+        return r < 1.0 ? r : 1.0;
+    }
+    *st |= ORC_ST_ZERO_DRAFT_PROB;
+    return q[x] > 0.0 ? 1.0 : 0.0;
+}
+
+static void kseq_residual(double* q, const double* p, int V, double gamma, int K, int* st) {
+    double beta = 0.0;
+    for (int y = 0; y < V; ++y) {
+        double a = p[y], b = q[y] / gamma;
+        beta += (a < b ? a : b);
+    }
+    double c = beta > 0.0 ? (1.0 - pow(1.0 - beta, (double)K)) / beta : (double)K;
+    double s = 0.0;
+    for (int y = 0; y < V; ++y) {
+        double a = p[y], b = q[y] / gamma;
+        double r = q[y] - (a < b ? a : b) * c;
+        s += (r > 0.0 ? r : 0.0);
+    }
+    if (s > 0.0 && isfinite(s)) {
+        for (int y = 0; y < V; ++y) {
+            double a = p[y], b = q[y] / gamma;
+            double r = q[y] - (a < b ? a : b) * c;
+            q[y] = (r > 0.0 ? r : 0.0) / s;
+        }
+    } else {
+        *st |= ORC_ST_ZERO_RESIDUAL;
+    }
+}
+
+/*
+ * Deterministic part of the two baseline verifiers for given distributions and
+ * an ordered tuple of K drafts: theta[k] assuming all earlier drafts were
+ * rejected, residual = the distribution of the token drawn when all K are
+ * rejected.  rule 1 = multi-round, rule 2 = K-SEQ.
+ */
+int rsd_oracle_baseline_chain(int rule, double gamma, const double* p_in, const double* q_in, int V,
+                              const int32_t* tokens, int K, double* theta, double* residual) {
+    double* q = (double*)malloc(sizeof(double) * (size_t)V);
+    memcpy(q, q_in, sizeof(double) * (size_t)V);
+    int st = 0;
+    for (int k = 0; k < K; ++k) {
+        if (rule == 1) {
+            theta[k] = rrs_threshold(q, p_in, tokens[k], &st);
+            multiround_reject(q, p_in, V, &st);
+        } else {
+            theta[k] = kseq_threshold(q, p_in, gamma, tokens[k], &st);
+        }
+    }
+    if (rule != 1) kseq_residual(q, p_in, V, gamma, K, &st);
+    memcpy(residual, q, sizeof(double) * (size_t)V);
+    free(q);
+    return st;
+}
+
+/*
  * Deterministic part of Algorithm 1 for given distributions and an ordered
  * draft tuple: theta[k] = Theta^(k+1) assuming all earlier drafts were
  * rejected, residual = q^(K+1).  Used by the exact-enumeration pins.
@@ -461,7 +548,8 @@ int rsd_oracle_rrs_chain(const double* p_in, const double* q_in, int V, const in
  * out_final_weights: optional [B][V], the normalised distribution the last
  * token was drawn from.
  */
-int rsd_oracle_verify_tree(const void* draft, int draft_dtype, int64_t draft_seq_stride, int64_t draft_row_stride,
+int rsd_oracle_verify_tree_rule(int rule, double gamma,
+                           const void* draft, int draft_dtype, int64_t draft_seq_stride, int64_t draft_row_stride,
                            double draft_temperature,
                            const void* target, int target_dtype, int64_t target_seq_stride, int64_t target_row_stride,
                            double target_temperature,
@@ -504,15 +592,20 @@ int rsd_oracle_verify_tree(const void* draft, int draft_dtype, int64_t draft_seq
             for (int c = 1; c < n_nodes && alive; ++c) {
                 if (par[c] != cur || tok[c] < 0) continue;
                 int x = tok[c];
-                double theta = rrs_threshold(q, p, x, &st);
+                double theta = (rule == 2) ? kseq_threshold(q, p, gamma, x, &st) : rrs_threshold(q, p, x, &st);
                 double U = rsd_oracle_accept_uniform(seed, step, seq, (uint32_t)cur, (uint32_t)j);
                 if (dbg_theta) dbg_theta[(int64_t)b * n_nodes + c] = theta;
                 if (dbg_margin) dbg_margin[(int64_t)b * n_nodes + c] = fabs(U - theta);
                 if (U < theta) { accepted_child = c; break; }
-                alive = rrs_reject(q, p, V, x, &st);
+                if (rule == 0) alive = rrs_reject(q, p, V, x, &st);
+                else if (rule == 1) multiround_reject(q, p, V, &st);
                 ++j;
             }
-            if (accepted_child < 0) { reason = ORC_STOP_ALL_REJECTED; break; }
+            if (accepted_child < 0) {
+                if (rule == 2) kseq_residual(q, p, V, gamma, n_children, &st);
+                reason = ORC_STOP_ALL_REJECTED;
+                break;
+            }
             accepted_node[(int64_t)b * num_levels + len] = accepted_child;
             accepted_token[(int64_t)b * num_levels + len] = tok[accepted_child];
             ++len;
@@ -529,6 +622,25 @@ int rsd_oracle_verify_tree(const void* draft, int draft_dtype, int64_t draft_seq
         free(lt); free(ld); free(q); free(p);
     }
     return 0;
+}
+
+/* recursive rejection sampling (rule 0): the paper's method */
+int rsd_oracle_verify_tree(const void* draft, int draft_dtype, int64_t draft_seq_stride, int64_t draft_row_stride,
+                           double draft_temperature,
+                           const void* target, int target_dtype, int64_t target_seq_stride, int64_t target_row_stride,
+                           double target_temperature,
+                           int B, int V, int n_nodes, int num_levels,
+                           const int32_t* parent, int topology_is_shared, const int32_t* token,
+                           uint64_t seed, uint32_t step, uint32_t seq_base,
+                           int32_t* accepted_len, int32_t* accepted_node, int32_t* accepted_token,
+                           int32_t* last_token, int32_t* stop_reason,
+                           double* dbg_theta, double* dbg_margin, double* final_margin, double* out_final_weights,
+                           int32_t* status) {
+    return rsd_oracle_verify_tree_rule(0, 1.0, draft, draft_dtype, draft_seq_stride, draft_row_stride, draft_temperature,
+                                       target, target_dtype, target_seq_stride, target_row_stride, target_temperature,
+                                       B, V, n_nodes, num_levels, parent, topology_is_shared, token, seed, step,
+                                       seq_base, accepted_len, accepted_node, accepted_token, last_token, stop_reason,
+                                       dbg_theta, dbg_margin, final_margin, out_final_weights, status);
 }
 
 /* ------------------------------------------------------------------------ */
