@@ -195,6 +195,29 @@ int rsd_verify_tree(const rsd_rows* draft, const rsd_rows* target, const rsd_tre
                     int32_t* status, rsd_stream_t stream);
 
 /*
+ * rsd_verify_tree with the verification rule as an argument: recursive rejection sampling, or one of the two
+ * earlier tree verifiers that Section 2 describes, run over the same tree layout, rows and random streams, so that
+ * acceptance rates can be compared on equal inputs (Figure 1 does this for Bernoulli distributions).
+ *   RSD_RULE_RRS         recursive rejection sampling (Section 3.1): exactly rsd_verify_tree
+ *   RSD_RULE_MULTIROUND  multi-round rejection sampling with one draft model, p^(k) = p (Section 2, SpecInfer): the
+ *                        children of a node are independent draws from p (repeats allowed); child j is accepted
+ *                        with probability min(1, q^(j)(x_j) / p(x_j)), q^(j+1) = Norm[(q^(j) - p)+]; the draft is
+ *                        never changed
+ *   RSD_RULE_KSEQ        K-sequential selection (Section 2, SpecTr), K = the number of children of the node: child j
+ *                        is accepted with probability min(1, q(x_j) / (gamma p(x_j))); if all K are rejected the
+ *                        token is drawn from Norm[(q - min{p, q/gamma} (1 - (1 - beta)^K) / beta)+] with
+ *                        beta = sum_x min{p(x), q(x)/gamma}.  gamma in [1, K]; gamma = K is always admissible
+ *                        (smaller values need (1 - (1 - beta)^K) / beta <= gamma, else the clamp at 0 applies)
+ * gamma is read only by RSD_RULE_KSEQ (finite, >= 1).  All other arguments, outputs and status bits as in
+ * rsd_verify_tree; RSD_ST_ZERO_RESIDUAL under K-SEQ means the token was drawn from the target row itself.
+ */
+enum { RSD_RULE_RRS = 0, RSD_RULE_MULTIROUND = 1, RSD_RULE_KSEQ = 2 };
+int rsd_verify_tree_rule(const rsd_rows* draft, const rsd_rows* target, const rsd_tree* tree, int B, int V,
+                         int rule, float gamma, uint64_t seed, uint32_t step, uint32_t seq_base,
+                         int32_t* accepted_len, int32_t* accepted_node, int32_t* accepted_token, int32_t* last_token,
+                         int32_t* stop_reason, float* dbg_theta, int32_t* status, rsd_stream_t stream);
+
+/*
  * One draw from a residual distribution (Eq. 2 applied along a list of rejected drafts; Section 2's
  * Norm[(q - p)+] is the one-token case).  Per sequence: p = softmax(draft row), q = softmax(target row); for each
  * token of rejected[b][0..max_k) in order (-1 = none) the chain step of Eqs. 1-2 is applied; then one token is

@@ -18,10 +18,11 @@ LIB_PATH = os.environ.get("RSD_LIB_PATH") or os.path.join(_HERE, "librsd.so")  #
 RSD_F32, RSD_BF16 = 0, 1
 ST_NAN_INPUT, ST_FEWER_THAN_K, ST_ZERO_RESIDUAL, ST_ZERO_DRAFT_PROB, ST_DRAFT_EXHAUSTED = 1, 2, 4, 8, 16
 STOP_ALL_REJECTED, STOP_NO_CHILDREN, STOP_LEAF = 0, 1, 2
+RULE_RRS, RULE_MULTIROUND, RULE_KSEQ = 0, 1, 2
 MAX_K = 32
 
 EXPORTS = ["rsd_version", "rsd_rng_layout", "rsd_last_error", "rsd_profile_next_scan", "rsd_gumbel_topk_draft", "rsd_sbs_workspace_bytes",
-           "rsd_sbs_step", "rsd_sbs_step_static", "rsd_verify_tree", "rsd_resample_residual"]
+           "rsd_sbs_step", "rsd_sbs_step_static", "rsd_verify_tree", "rsd_verify_tree_rule", "rsd_resample_residual"]
 
 
 class RsdRows(C.Structure):
@@ -67,6 +68,10 @@ def lib():
         l.rsd_verify_tree.argtypes = [C.POINTER(RsdRows), C.POINTER(RsdRows), C.POINTER(RsdTree), C.c_int, C.c_int,
                                       C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        l.rsd_verify_tree_rule.argtypes = [C.POINTER(RsdRows), C.POINTER(RsdRows), C.POINTER(RsdTree), C.c_int, C.c_int,
+                                           C.c_int, C.c_float, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_void_p]
         l.rsd_resample_residual.argtypes = [C.POINTER(RsdRows), C.POINTER(RsdRows), C.c_int, C.c_int, C.c_void_p,
                                             C.c_int, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
                                             C.c_void_p, C.c_void_p, C.c_void_p]
@@ -207,8 +212,10 @@ def rsd_sbs_step_static(draft_level: torch.Tensor, W: int, first_parent_node: in
 
 def rsd_verify_tree(draft: torch.Tensor, target: torch.Tensor, parent: torch.Tensor, token: torch.Tensor,
                     num_levels: int, seed: int, step: int, *, seq_base: int = 0, want_theta: bool = False,
-                    out: Optional[dict] = None, draft_temperature: float = 1.0, target_temperature: float = 1.0):
-    """draft [B, P, V], target [B, N+1, V], parent [N+1] or [B, N+1] int32, token [B, N+1] int32."""
+                    out: Optional[dict] = None, draft_temperature: float = 1.0, target_temperature: float = 1.0,
+                    rule: int = 0, gamma: float = 1.0):
+    """draft [B, P, V], target [B, N+1, V], parent [N+1] or [B, N+1] int32, token [B, N+1] int32.
+    rule = RULE_RRS calls rsd_verify_tree; RULE_MULTIROUND / RULE_KSEQ call rsd_verify_tree_rule."""
     B, _, V = target.shape
     dev = target.device
     n_nodes = token.shape[1]
@@ -227,11 +234,20 @@ def rsd_verify_tree(draft: torch.Tensor, target: torch.Tensor, parent: torch.Ten
         out["theta"] = torch.empty((B, n_nodes), dtype=torch.float32, device=dev) if want_theta else None
     tree = RsdTree(L, n_nodes, parent.data_ptr(), token.data_ptr(), 1 if parent.dim() == 1 else 0)
     d, t = rows_of(draft, False, draft_temperature), rows_of(target, False, target_temperature)
-    _check(lib().rsd_verify_tree(C.byref(d), C.byref(t), C.byref(tree), B, V, seed, step, seq_base,
-                                 _ptr(out["accepted_len"]), _ptr(out["accepted_node"]), _ptr(out["accepted_token"]),
-                                 _ptr(out["last_token"]), _ptr(out["stop_reason"]), _ptr(out.get("theta")),
-                                 _ptr(out["status"]), _stream()))
+    outs = (_ptr(out["accepted_len"]), _ptr(out["accepted_node"]), _ptr(out["accepted_token"]),
+            _ptr(out["last_token"]), _ptr(out["stop_reason"]), _ptr(out.get("theta")), _ptr(out["status"]), _stream())
+    if rule == RULE_RRS:
+        _check(lib().rsd_verify_tree(C.byref(d), C.byref(t), C.byref(tree), B, V, seed, step, seq_base, *outs))
+    else:
+        _check(lib().rsd_verify_tree_rule(C.byref(d), C.byref(t), C.byref(tree), B, V, int(rule), float(gamma),
+                                          seed, step, seq_base, *outs))
     return out
+
+
+def rsd_verify_tree_rule(draft: torch.Tensor, target: torch.Tensor, parent: torch.Tensor, token: torch.Tensor,
+                         num_levels: int, rule: int, gamma: float, seed: int, step: int, **kw):
+    """rsd_verify_tree with a verification rule (RULE_RRS, RULE_MULTIROUND, RULE_KSEQ with its gamma)."""
+    return rsd_verify_tree(draft, target, parent, token, num_levels, seed, step, rule=rule, gamma=gamma, **kw)
 
 
 def rsd_resample_residual(draft_row: Optional[torch.Tensor], target_row: torch.Tensor,

@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librsd.so")
-SOURCES = ["rsd_api.cu"]
-HEADERS = ["rsd_device.cuh", "rsd_scan.cuh", "rsd_verify.cuh", os.path.join("..", "..", "include", "rsd.h")]
+SOURCES = ["rsd_api.cu", "rsd_api_verify.cu"]
+HEADERS = ["rsd_api_common.h", "rsd_device.cuh", "rsd_scan.cuh", "rsd_verify.cuh", os.path.join("..", "..", "include", "rsd.h")]
 
 
 def _stale() -> bool:
@@ -26,13 +26,22 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB, defines=()
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = out + ".%d.tmp" % os.getpid()
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
-           "-Xcompiler", "-fPIC", "--use_fast_math" if False else "-DRSD_BUILD", "-o", tmp]
-    cmd += ["-D" + d for d in defines]
+    flags = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
+             "-DRSD_BUILD"] + ["-D" + d for d in defines]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, f) for f in SOURCES]
-    subprocess.check_call(cmd)
+        flags += ["-Xptxas", "-v"]
+    # one object per translation unit, compiled side by side, then one link
+    objs = [tmp + "." + os.path.splitext(f)[0] + ".o" for f in SOURCES]
+    procs = [subprocess.Popen([nvcc] + flags + ["-c", os.path.join(CSRC, f), "-o", o]) for f, o in zip(SOURCES, objs)]
+    codes = [p.wait() for p in procs]
+    try:
+        if any(codes):
+            raise subprocess.CalledProcessError(max(codes), [nvcc] + flags + SOURCES)
+        subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", tmp] + objs)
+    finally:
+        for o in objs:
+            if os.path.exists(o):
+                os.remove(o)
     os.replace(tmp, out)
     return out
 

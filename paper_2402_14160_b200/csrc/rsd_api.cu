@@ -1,56 +1,21 @@
-// C ABI of librsd (declared in include/rsd.h): argument checks and kernel launches, nothing else.
+// C ABI of librsd (declared in include/rsd.h), drafting half: argument checks and kernel launches, nothing else.
+// The verification entry points are in rsd_api_verify.cu (two translation units keep each compile small).
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
 
-#include "../../include/rsd.h"
+#include "rsd_api_common.h"
 #include "rsd_scan.cuh"
-#include "rsd_verify.cuh"
+
+namespace rsd_host {
+thread_local char g_err[512] = "";
+}
+using namespace rsd_host;
 
 namespace {
 
-thread_local char g_err[512] = "";
 thread_local cudaEvent_t g_scan_before = nullptr, g_scan_after = nullptr;  // one-shot, see rsd_profile_next_scan
-
-int fail(int code, const char* fmt, ...) {
-    va_list ap;
-    va_start(ap, fmt);
-    vsnprintf(g_err, sizeof(g_err), fmt, ap);
-    va_end(ap);
-    return code;
-}
-
-int check_launch(const char* what) {
-    const cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return fail(RSD_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
-    return RSD_OK;
-}
-
-int check_rows(const char* name, const rsd_rows* r, int V, bool need_row_stride) {
-    if (!r || !r->data) return fail(RSD_ERR_INVALID_ARG, "%s: null rows", name);
-    if (r->dtype != RSD_F32 && r->dtype != RSD_BF16) return fail(RSD_ERR_UNSUPPORTED, "%s: unknown dtype %d", name, r->dtype);
-    if (need_row_stride && r->row_stride < V) return fail(RSD_ERR_INVALID_ARG, "%s: row_stride %lld < V %d", name, (long long)r->row_stride, V);
-    if (r->seq_stride < 0 || r->row_stride < 0) return fail(RSD_ERR_INVALID_ARG, "%s: negative stride", name);
-    if (!(r->temperature >= 0.0f) || r->temperature > 3.0e38f)
-        return fail(RSD_ERR_INVALID_ARG, "%s: temperature %g must be a finite number >= 0 (0 or 1: none)", name, (double)r->temperature);
-    return RSD_OK;
-}
-
-// temperature that applies (1 when the rows ask for none)
-float temperature_of(const rsd_rows* r) { return (r->temperature > 0.0f && r->temperature != 1.0f) ? r->temperature : 1.0f; }
-// rows usable as log-probabilities as they are: flagged so and not re-scored by a temperature
-bool rows_are_logprob(const rsd_rows* r) { return r->is_logprob && temperature_of(r) == 1.0f; }
-
-bool rows_aligned(const rsd_rows* r, int bytes = 16) {
-    const int64_t eb = r->dtype == RSD_F32 ? 4 : 2;
-    return ((uintptr_t)r->data % bytes == 0) && ((r->seq_stride * eb) % bytes == 0) && ((r->row_stride * eb) % bytes == 0);
-}
-
-int check_vocab(int V) {
-    if (V < 1 || V > RSD_MAX_VOCAB) return fail(RSD_ERR_UNSUPPORTED, "V = %d outside [1, %d]", V, (int)RSD_MAX_VOCAB);
-    return RSD_OK;
-}
 
 template <typename T, bool ALIGNED, bool WIDE, bool NEED_LSE, bool TEMP>
 void launch_scan_temp(int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
@@ -216,75 +181,6 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     const size_t smem = (size_t)n_par * W * (8 + 8 + 4) + (size_t)n_par * 4;
     rsd::sbs_epilogue_kernel<<<B, rsd::kEpilogueThreads, smem, s>>>(e);
     return check_launch("rsd_sbs_step(epilogue)");
-}
-
-int rsd_verify_tree(const rsd_rows* draft, const rsd_rows* target, const rsd_tree* tree, int B, int V, uint64_t seed,
-                    uint32_t step, uint32_t seq_base, int32_t* accepted_len, int32_t* accepted_node,
-                    int32_t* accepted_token, int32_t* last_token, int32_t* stop_reason, float* dbg_theta,
-                    int32_t* status, rsd_stream_t stream) {
-    g_err[0] = 0;
-    if (int e = check_vocab(V)) return e;
-    if (int e = check_rows("draft", draft, V, true)) return e;
-    if (int e = check_rows("target", target, V, true)) return e;
-    if (draft->dtype != target->dtype) return fail(RSD_ERR_UNSUPPORTED, "draft and target rows must have the same dtype");
-    if (!tree || !tree->parent || !tree->token) return fail(RSD_ERR_INVALID_ARG, "null tree");
-    if (tree->num_levels < 0 || tree->num_nodes < 1 || tree->num_nodes > RSD_MAX_TREE_NODES)
-        return fail(RSD_ERR_UNSUPPORTED, "num_levels = %d, num_nodes = %d", tree->num_levels, tree->num_nodes);
-    if (B < 0) return fail(RSD_ERR_INVALID_ARG, "B = %d", B);
-    if (!accepted_len || !accepted_node || !accepted_token || !last_token || !stop_reason || !status) return fail(RSD_ERR_INVALID_ARG, "null output");
-    if (B == 0) return RSD_OK;
-    rsd::VerifyArgs a;
-    a.draft = {draft->data, draft->seq_stride, draft->row_stride, 1.0f / temperature_of(draft)};
-    a.target = {target->data, target->seq_stride, target->row_stride, 1.0f / temperature_of(target)};
-    a.V = V; a.L = tree->num_levels; a.num_nodes = tree->num_nodes; a.shared_topology = tree->topology_is_shared;
-    a.parent = tree->parent; a.token = tree->token;
-    a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
-    a.accepted_len = accepted_len; a.accepted_node = accepted_node; a.accepted_token = accepted_token;
-    a.last_token = last_token; a.stop_reason = stop_reason; a.dbg_theta = dbg_theta; a.status = status;
-    cudaStream_t s = (cudaStream_t)stream;
-    const bool aligned = rows_aligned(draft) && rows_aligned(target);
-    using namespace rsd;
-    if (draft->dtype == RSD_F32) {
-        if (aligned) verify_tree_kernel<float, true><<<B, kVerifyThreads, 0, s>>>(a);
-        else verify_tree_kernel<float, false><<<B, kVerifyThreads, 0, s>>>(a);
-    } else {
-        if (aligned) verify_tree_kernel<__nv_bfloat16, true><<<B, kVerifyThreads, 0, s>>>(a);
-        else verify_tree_kernel<__nv_bfloat16, false><<<B, kVerifyThreads, 0, s>>>(a);
-    }
-    return check_launch("rsd_verify_tree");
-}
-
-int rsd_resample_residual(const rsd_rows* draft_row, const rsd_rows* target_row, int B, int V, const int32_t* rejected,
-                          int max_k, const int32_t* rng_node, uint64_t seed, uint32_t step, uint32_t seq_base,
-                          int32_t* out_token, float* out_residual, int32_t* status, rsd_stream_t stream) {
-    g_err[0] = 0;
-    if (int e = check_vocab(V)) return e;
-    if (int e = check_rows("target_row", target_row, V, false)) return e;
-    if (rejected) {
-        if (int e = check_rows("draft_row", draft_row, V, false)) return e;
-        if (draft_row->dtype != target_row->dtype) return fail(RSD_ERR_UNSUPPORTED, "draft and target rows must have the same dtype");
-        if (max_k < 1 || max_k > RSD_MAX_K) return fail(RSD_ERR_UNSUPPORTED, "max_k = %d outside [1, %d]", max_k, (int)RSD_MAX_K);
-    }
-    if (B < 0) return fail(RSD_ERR_INVALID_ARG, "B = %d", B);
-    if (!rng_node || !out_token || !status) return fail(RSD_ERR_INVALID_ARG, "null argument");
-    if (B == 0) return RSD_OK;
-    rsd::ResampleArgs a;
-    a.target = {target_row->data, target_row->seq_stride, 0, 1.0f / temperature_of(target_row)};
-    a.draft = rejected ? rsd::RowsDev{draft_row->data, draft_row->seq_stride, 0, 1.0f / temperature_of(draft_row)} : a.target;
-    a.V = V; a.max_k = rejected ? max_k : 0; a.rejected = rejected; a.rng_node = rng_node;
-    a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
-    a.out_token = out_token; a.out_residual = out_residual; a.status = status;
-    cudaStream_t s = (cudaStream_t)stream;
-    const bool aligned = rows_aligned(target_row) && (!rejected || rows_aligned(draft_row));
-    using namespace rsd;
-    if (target_row->dtype == RSD_F32) {
-        if (aligned) resample_residual_kernel<float, true><<<B, kVerifyThreads, 0, s>>>(a);
-        else resample_residual_kernel<float, false><<<B, kVerifyThreads, 0, s>>>(a);
-    } else {
-        if (aligned) resample_residual_kernel<__nv_bfloat16, true><<<B, kVerifyThreads, 0, s>>>(a);
-        else resample_residual_kernel<__nv_bfloat16, false><<<B, kVerifyThreads, 0, s>>>(a);
-    }
-    return check_launch("rsd_resample_residual");
 }
 
 }  // extern "C"

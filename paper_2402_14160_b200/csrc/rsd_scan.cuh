@@ -796,7 +796,7 @@ struct SbsEpilogueArgs {
 
 constexpr int kEpilogueThreads = 128;
 
-__global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const SbsEpilogueArgs a) {
+static __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const SbsEpilogueArgs a) {
     extern __shared__ double sm_d[];  // [F] phi~ then psi, [F] phi
     const int F = a.n_par * a.W;
     double* s_val = sm_d;

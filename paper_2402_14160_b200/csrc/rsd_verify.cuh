@@ -48,6 +48,8 @@ struct RowsDev {
 struct VerifyArgs {
     RowsDev draft, target;
     int V, L, num_nodes, shared_topology;
+    int rule;      // 0 recursive rejection sampling, 1 multi-round rejection sampling, 2 K-SEQ
+    float gamma;   // K-SEQ's parameter
     const int32_t* parent;
     const int32_t* token;
     uint32_t seed_lo, seed_hi, step, seq_base;
@@ -155,6 +157,33 @@ __device__ __forceinline__ float clean(const Packed<T>& pk, float (&v)[16], bool
     return m;
 }
 
+// Weight modes of a pass over the two rows (qh, ph = exponentials of the target and draft values):
+//   kTargetOnly  qh                               plain target distribution
+//   kResidual    (qh - a ph)+                     Eq. 2 in closed form, a = a_hi + a_lo
+//   kSeqOverlap  min(a_hi ph, a_lo qh)            K-SEQ: min{p, q / gamma} in units of qh
+//   kSeqResidual (qh - c min(a_hi ph, a_lo qh))+  K-SEQ: the all-rejected residual
+enum { kTargetOnly = 0, kResidual = 1, kSeqOverlap = 2, kSeqResidual = 3 };
+
+template <int MODE>
+__device__ __forceinline__ float weight1(float qh, float ph, float a_hi, float a_lo, float c) {
+    if (MODE == kResidual) return residual_weight(qh, ph, a_hi, a_lo);
+    const float m = fminf(a_hi * ph, a_lo * qh);
+    if (MODE == kSeqOverlap) return m;
+    if (MODE == kSeqResidual) return fmaxf(fmaf(-c, m, qh), 0.0f);
+    return qh;
+}
+
+template <int MODE>
+__device__ __forceinline__ void weights16(const float (&qh)[16], const float (&ph)[16], float a_hi, float a_lo, float c,
+                                          float (&w)[16]) {
+    if (MODE == kResidual) {
+        residual16(qh, ph, a_hi, a_lo, w);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) w[j] = weight1<MODE>(qh[j], ph[j], a_hi, a_lo, c);
+    }
+}
+
 // load a group, turn NaN into -inf (reported), return the group's maximum
 template <typename T, bool ALIGNED>
 __device__ __forceinline__ float load_clean(const char* row, int g, int V, float (&v)[16], bool& saw_nan) {
@@ -165,7 +194,7 @@ __device__ __forceinline__ float load_clean(const char* row, int g, int V, float
 
 // Row maximum over the first block-wide sweep (cheap reference), or over the whole row when asked.
 template <typename T, bool ALIGNED>
-__device__ float row_reference(const char* row, int V, bool whole_row, VerifySmem& sm, bool& saw_nan) {
+__device__ __forceinline__ float row_reference(const char* row, int V, bool whole_row, VerifySmem& sm, bool& saw_nan) {
     const int n_groups = (V + 15) >> 4;
     float m = kNegInf;
     float v[16];
@@ -179,10 +208,11 @@ __device__ float row_reference(const char* row, int V, bool whole_row, VerifySme
 // One pass over the row(s): weights w(y) = (qhat(y) - a phat(y))+ with qhat = exp(lt - m_q), phat = exp(ld - m_p)
 // (a = 0, no draft row: plain exponentials of the target).  Leaves the sum of every 512-element tile in
 // sm.tile_sum, returns their total (summed in tile order, identically on all threads) and the true row maxima.
-template <typename T, bool ALIGNED, bool WITH_DRAFT>
-__device__ double weight_pass(const char* rowq, const char* rowp, int V, float mq, float mp, float kq, float kp,
+template <typename T, bool ALIGNED, int MODE>
+__device__ __forceinline__ double weight_pass(const char* rowq, const char* rowp, int V, float mq, float mp, float kq, float kp,
                               float a_hi, float a_lo,
-                              VerifySmem& sm, bool& saw_nan, float* true_max_q, float* true_max_p) {
+                              VerifySmem& sm, bool& saw_nan, float* true_max_q, float* true_max_p, float c_seq = 0.0f) {
+    constexpr bool WITH_DRAFT = MODE != kTargetOnly;
     const int n_groups = (V + 15) >> 4;
     const int n_tiles = (n_groups + 31) >> 5;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -217,7 +247,7 @@ __device__ double weight_pass(const char* rowq, const char* rowp, int V, float m
                         tmp_ = fmaxf(tmp_, clean<T>(cp, p, saw_nan));
                         exp16(q, kq, cq_, q);
                         exp16(p, kp, cp_, p);
-                        residual16(q, p, a_hi, a_lo, w);
+                        weights16<MODE>(q, p, a_hi, a_lo, c_seq, w);
                     } else {
                         exp16(q, kq, cq_, w);
                     }
@@ -235,7 +265,7 @@ __device__ double weight_pass(const char* rowq, const char* rowp, int V, float m
     if (true_max_q) *true_max_q = block_max<kVerifyThreads>(tmq, sm.red_f);
     if (true_max_p) *true_max_p = block_max<kVerifyThreads>(tmp_, sm.red_f);
     __syncthreads();
-    if (WITH_DRAFT && sm.n_removed > 0) {  // removed tokens weigh what they weighed at removal
+    if (MODE == kResidual && sm.n_removed > 0) {  // removed tokens weigh what they weighed at removal
         if (threadIdx.x == 0) {
             for (int i = 0; i < sm.n_removed; ++i) {
                 const float generic = residual_weight(sm.rem_qh[i], sm.rem_ph[i], a_hi, a_lo);
@@ -252,7 +282,7 @@ __device__ double weight_pass(const char* rowq, const char* rowp, int V, float m
 
 // Both normalisers of a node in one pass: S_q = sum exp(lt - m_q), S_p = sum exp(ld - m_p).
 template <typename T, bool ALIGNED>
-__device__ void softmax_sums(const char* rowq, const char* rowp, int V, float mq, float mp, float kq, float kp,
+__device__ __forceinline__ void softmax_sums(const char* rowq, const char* rowp, int V, float mq, float mp, float kq, float kp,
                              VerifySmem& sm,
                              bool& saw_nan, double* Sq, double* Sp, float* true_max_q, float* true_max_p) {
     const int n_groups = (V + 15) >> 4;
@@ -309,10 +339,11 @@ __device__ void softmax_sums(const char* rowq, const char* rowp, int V, float mq
 
 // Inverse CDF over the weights of the last weight_pass: the smallest y whose running sum exceeds u * total; if
 // rounding leaves none, the largest y with positive weight; -1 if there is no weight at all.
-template <typename T, bool ALIGNED, bool WITH_DRAFT>
-__device__ int inverse_cdf_pick(const char* rowq, const char* rowp, int V, float mq, float mp, float kq, float kp,
+template <typename T, bool ALIGNED, int MODE>
+__device__ __forceinline__ int inverse_cdf_pick(const char* rowq, const char* rowp, int V, float mq, float mp, float kq, float kp,
                                 float a_hi, float a_lo,
-                                double total, double u, VerifySmem& sm) {
+                                double total, double u, VerifySmem& sm, float c_seq = 0.0f) {
+    constexpr bool WITH_DRAFT = MODE != kTargetOnly;
     const int n_groups = (V + 15) >> 4;
     const int n_tiles = (n_groups + 31) >> 5;
     if (!(total > 0.0) || total > 1.7e308) return -1;
@@ -347,8 +378,8 @@ __device__ int inverse_cdf_pick(const char* rowq, const char* rowp, int V, float
                 load_clean<T, ALIGNED>(rowp, g, V, p, dummy);
                 exp16(q, kq, cq, q);
                 exp16(p, kp, cp, p);
-                residual16(q, p, a_hi, a_lo, w);
-                for (int i = 0; i < sm.n_removed; ++i) {
+                weights16<MODE>(q, p, a_hi, a_lo, c_seq, w);
+                for (int i = 0; MODE == kResidual && i < sm.n_removed; ++i) {
                     if ((sm.rem_x[i] >> 4) != g) continue;
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
@@ -391,7 +422,8 @@ __device__ int inverse_cdf_pick(const char* rowq, const char* rowp, int V, float
 }
 
 // State of one sibling chain at a node; all threads hold identical copies.
-template <typename T, bool ALIGNED>
+// BASELINES: the chain also knows the two baseline rules; the plain instantiation carries none of their code.
+template <typename T, bool ALIGNED, bool BASELINES = false>
 struct NodeChain {
     const char* rowq;
     const char* rowp;
@@ -402,7 +434,10 @@ struct NodeChain {
     double A, P, Z;     // closed-form chain state
     double total;       // sum of the weights of the last weight_pass (valid if tiles_current)
     float a_hi, a_lo;
-    bool with_draft, tiles_current;
+    float c_seq;        // K-SEQ: the factor of its residual, set by seq_finish()
+    int rule;           // 0 recursive, 1 multi-round (the draft is never changed), 2 K-SEQ
+    double gamma;       // K-SEQ's parameter
+    bool with_draft, tiles_current, seq_residual;
 
     __device__ void split_a() {
         const double a = A * Sq / Sp;
@@ -413,7 +448,7 @@ struct NodeChain {
     // reference maxima and normalisers of the node (both rows)
     __device__ void open_both(const char* q, const char* p, int V_, float kq_, float kp_, VerifySmem& sm, bool& saw_nan) {
         rowq = q; rowp = p; V = V_; kq = kq_; kp = kp_; with_draft = true; tiles_current = false;
-        A = 0.0; P = 0.0; Z = 1.0; a_hi = a_lo = 0.0f;
+        A = 0.0; P = 0.0; Z = 1.0; a_hi = a_lo = 0.0f; c_seq = 0.0f; seq_residual = false;
         __syncthreads();
         if (threadIdx.x == 0) sm.n_removed = 0;
         __syncthreads();
@@ -450,7 +485,7 @@ struct NodeChain {
     // plain target row: weights exp(lt - m_q), total = S_q, tile sums ready for the draw
     __device__ void open_target_only(const char* q, int V_, float kq_, VerifySmem& sm, bool& saw_nan) {
         rowq = q; rowp = q; V = V_; kq = kq_; kp = kq_; with_draft = false; tiles_current = true;
-        A = 0.0; P = 0.0; Z = 1.0; a_hi = a_lo = 0.0f; Sp = 1.0; mp = 0.0f;
+        A = 0.0; P = 0.0; Z = 1.0; a_hi = a_lo = 0.0f; Sp = 1.0; mp = 0.0f; c_seq = 0.0f; seq_residual = false;
         __syncthreads();
         if (threadIdx.x == 0) sm.n_removed = 0;
         __syncthreads();
@@ -458,7 +493,7 @@ struct NodeChain {
         if (!(mq > kNegInf)) mq = row_reference<T, ALIGNED>(rowq, V, true, sm, saw_nan);
         for (int attempt = 0; attempt < 2; ++attempt) {
             float tq;
-            total = weight_pass<T, ALIGNED, false>(rowq, rowq, V, mq, 0.0f, kq, kq, 0.0f, 0.0f, sm, saw_nan, &tq, nullptr);
+            total = weight_pass<T, ALIGNED, kTargetOnly>(rowq, rowq, V, mq, 0.0f, kq, kq, 0.0f, 0.0f, sm, saw_nan, &tq, nullptr);
             if (!((tq - mq) * kq > kRefSlack * kLog2e)) break;
             mq = tq;
         }
@@ -473,9 +508,14 @@ struct NodeChain {
         return (l == l) ? (double)ex2_approx(fmaf(l, kp, -mp * kp)) / Sp : 0.0;
     }
 
-    // Eq. 3 for the next child, given its target and draft row values
+    // Eq. 3 for the next child, given its target and draft row values (K-SEQ: min{1, q(x) / (gamma p(x))})
     __device__ double threshold(float lq, float lp, int& st) const {
         const double qx = prob_q(lq), px = prob_p(lp);
+        if (BASELINES && rule == 2) {
+            if (px > 0.0) return fmin(1.0, qx / (gamma * px));
+            st |= 8;
+            return qx > 0.0 ? 1.0 : 0.0;
+        }
         const double r = fmax(qx - A * px, 0.0);
         if (px > 0.0) return fmin(1.0, r * (1.0 - P) / (Z * px));
         st |= 8;  // RSD_ST_ZERO_DRAFT_PROB
@@ -489,7 +529,7 @@ struct NodeChain {
         const double A_old = A;
         A = A_new;
         split_a();
-        const double zhat = weight_pass<T, ALIGNED, true>(rowq, rowp, V, mq, mp, kq, kp, a_hi, a_lo, sm, saw_nan, nullptr, nullptr);
+        const double zhat = weight_pass<T, ALIGNED, kResidual>(rowq, rowp, V, mq, mp, kq, kp, a_hi, a_lo, sm, saw_nan, nullptr, nullptr);
         const double Z_new = zhat / Sq;
         if (Z_new > 0.0 && Z_new < 1.7e308) {
             Z = Z_new;
@@ -501,6 +541,7 @@ struct NodeChain {
             split_a();
             tiles_current = false;
         }
+        if (BASELINES && rule == 1) return true;   // multi-round rejection sampling: the draft stays as it is
         P += px;
         __syncthreads();
         if (threadIdx.x == 0 && sm.n_removed < kMaxRemoved) {
@@ -515,25 +556,48 @@ struct NodeChain {
         return true;
     }
 
+    // K-SEQ after all K children were rejected: beta = sum min{p, q / gamma}, then the residual
+    // (q - min{p, q / gamma} (1 - (1 - beta)^K) / beta)+ with its tile sums ready for the draw
+    __device__ void seq_finish(int K, VerifySmem& sm, bool& saw_nan, int& st) {
+        const float a = (float)(Sq / Sp), g = (float)(1.0 / gamma);
+        const double overlap = weight_pass<T, ALIGNED, kSeqOverlap>(rowq, rowp, V, mq, mp, kq, kp, a, g, sm, saw_nan, nullptr, nullptr);
+        const double beta = overlap / Sq;
+        double miss = 1.0;   // (1 - beta)^K, K = the node's number of children
+        for (int i = 0; i < K; ++i) miss *= 1.0 - beta;
+        const double c = beta > 0.0 ? (1.0 - miss) / beta : (double)K;
+        const double t = weight_pass<T, ALIGNED, kSeqResidual>(rowq, rowp, V, mq, mp, kq, kp, a, g, sm, saw_nan, nullptr, nullptr, (float)c);
+        if (t > 0.0 && t < 1.7e308) {
+            a_hi = a; a_lo = g; c_seq = (float)c;
+            total = t;
+            tiles_current = true;
+            seq_residual = true;
+        } else {
+            st |= 4;  // RSD_ST_ZERO_RESIDUAL: draw from the target row itself
+            tiles_current = false;
+        }
+    }
+
     // draw from the current residual
     __device__ int draw(double u, VerifySmem& sm, bool& saw_nan) {
+        if (BASELINES && seq_residual)
+            return inverse_cdf_pick<T, ALIGNED, kSeqResidual>(rowq, rowp, V, mq, mp, kq, kp, a_hi, a_lo, total, u, sm, c_seq);
         if (!with_draft || A == 0.0) {
             if (!tiles_current || with_draft) {
                 float tq;
-                total = weight_pass<T, ALIGNED, false>(rowq, rowq, V, mq, 0.0f, kq, kq, 0.0f, 0.0f, sm, saw_nan, &tq, nullptr);
+                total = weight_pass<T, ALIGNED, kTargetOnly>(rowq, rowq, V, mq, 0.0f, kq, kq, 0.0f, 0.0f, sm, saw_nan, &tq, nullptr);
             }
-            return inverse_cdf_pick<T, ALIGNED, false>(rowq, rowq, V, mq, 0.0f, kq, kq, 0.0f, 0.0f, total, u, sm);
+            return inverse_cdf_pick<T, ALIGNED, kTargetOnly>(rowq, rowq, V, mq, 0.0f, kq, kq, 0.0f, 0.0f, total, u, sm);
         }
         if (!tiles_current)
-            total = weight_pass<T, ALIGNED, true>(rowq, rowp, V, mq, mp, kq, kp, a_hi, a_lo, sm, saw_nan, nullptr, nullptr);
-        return inverse_cdf_pick<T, ALIGNED, true>(rowq, rowp, V, mq, mp, kq, kp, a_hi, a_lo, total, u, sm);
+            total = weight_pass<T, ALIGNED, kResidual>(rowq, rowp, V, mq, mp, kq, kp, a_hi, a_lo, sm, saw_nan, nullptr, nullptr);
+        return inverse_cdf_pick<T, ALIGNED, kResidual>(rowq, rowp, V, mq, mp, kq, kp, a_hi, a_lo, total, u, sm);
     }
 };
 
 // smallest node c > after with parent[c] == cur and a token in [0, V), or -1.  Trees of up to kMaxCachedNodes nodes
 // sit in shared memory and every warp searches them by itself (no barrier); larger trees are searched in global
 // memory by the whole block.
-__device__ int next_child(const int32_t* par, const int32_t* tok, int num_nodes, int V, int cur, int after, VerifySmem& sm) {
+__device__ __forceinline__ int next_child(const int32_t* par, const int32_t* tok, int num_nodes, int V, int cur, int after, VerifySmem& sm) {
     if (num_nodes <= kMaxCachedNodes) {
         const int lane = threadIdx.x & 31;
         for (int c0 = after + 1; c0 < num_nodes; c0 += 32) {
@@ -559,7 +623,7 @@ __device__ int next_child(const int32_t* par, const int32_t* tok, int num_nodes,
     return r == 0x7FFFFFFF ? -1 : r;
 }
 
-template <typename T, bool ALIGNED>
+template <typename T, bool ALIGNED, bool BASELINES>
 __global__ void __launch_bounds__(kVerifyThreads, sizeof(T) == 2 ? RSD_VERIFY_MIN_BLOCKS : RSD_VERIFY_MIN_BLOCKS_F32)
 verify_tree_kernel(const VerifyArgs a) {
     __shared__ VerifySmem sm;
@@ -581,7 +645,10 @@ verify_tree_kernel(const VerifyArgs a) {
         for (int n = tid; n < a.num_nodes; n += kVerifyThreads) { sm.par[n] = par[n]; sm.tok[n] = tok[n]; }
     __syncthreads();
 
-    NodeChain<T, ALIGNED> chain;
+    NodeChain<T, ALIGNED, BASELINES> chain;
+    chain.rule = BASELINES ? a.rule : 0;
+    chain.gamma = (double)a.gamma;
+    const int rule = chain.rule;
     int cur = 0, len = 0, reason;
     for (;;) {
         int c = next_child(par, tok, a.num_nodes, a.V, cur, 0, sm);
@@ -602,11 +669,15 @@ verify_tree_kernel(const VerifyArgs a) {
             const double U = (double)(rw.x >> 8) * (1.0 / 16777216.0);
             if (a.dbg_theta && tid == 0) a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)theta;
             if (U < theta) { accepted = c; break; }
-            if (!chain.reject(x, lq, lp, sm, saw_nan, st)) break;
             ++j;
+            if (!(BASELINES && rule == 2) && !chain.reject(x, lq, lp, sm, saw_nan, st)) break;
             c = next_child(par, tok, a.num_nodes, a.V, cur, c, sm);
         }
-        if (accepted < 0) { reason = 0; break; }  // RSD_STOP_ALL_REJECTED
+        if (accepted < 0) {  // RSD_STOP_ALL_REJECTED
+            if (BASELINES && rule == 2) chain.seq_finish(j, sm, saw_nan, st);
+            reason = 0;
+            break;
+        }
         if (tid == 0) {
             a.accepted_node[(int64_t)b * a.L + len] = accepted;
             a.accepted_token[(int64_t)b * a.L + len] = cached ? sm.tok[accepted] : tok[accepted];
@@ -640,6 +711,8 @@ __global__ void __launch_bounds__(kVerifyThreads) resample_residual_kernel(const
     if (a.rejected)
         for (int i = 0; i < a.max_k; ++i) { const int x = a.rejected[(int64_t)b * a.max_k + i]; n_rej += (x >= 0 && x < a.V) ? 1 : 0; }
     NodeChain<T, ALIGNED> chain;
+    chain.rule = 0;
+    chain.gamma = 1.0;
     const char* rowq = row_ptr<T>(a.target, b, 0);
     if (n_rej == 0) {
         chain.open_target_only(rowq, a.V, kLog2e * a.target.inv_temp, sm, saw_nan);

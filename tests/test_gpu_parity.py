@@ -382,3 +382,65 @@ def test_temperature_arguments_are_checked(rsd):
     a = rsd.rsd_gumbel_topk_draft(rows, [4], [0], seed=0, step=0, temperature=0.0)     # 0 = none
     b = rsd.rsd_gumbel_topk_draft(rows, [4], [0], seed=0, step=0)
     assert torch.equal(a["token"], b["token"])
+
+
+# ---------------------------------------------------------------------------------------------------------
+# baseline verifiers on the same kernel: multi-round rejection sampling and K-SEQ (Section 2)
+# ---------------------------------------------------------------------------------------------------------
+def _iid_tree(draft_h, branching, seed):
+    """Tree with constant branching factors whose children are independent draws (repeats allowed) from the softmax of
+    the parent's draft row, as the two baseline verifiers assume."""
+    parent = workloads.rsdc_parent_array(branching)
+    B, P, V = draft_h.shape
+    rng = np.random.default_rng(seed)
+    token = np.full((B, len(parent)), -1, np.int32)
+    for b in range(B):
+        for n in range(1, len(parent)):
+            row = draft_h[b, parent[n]].astype(np.float64)
+            p = np.exp(row - row.max())
+            token[b, n] = rng.choice(V, p=p / p.sum())
+    return parent, token
+
+
+@pytest.mark.parametrize("rule,gamma", [(1, 1.0), (2, 3.0), (2, 1.5)])
+@pytest.mark.parametrize("dtype,V,branching", [("f32", 97, (3, 3)), ("bf16", 4099, (3, 2, 2)), ("bf16", 32000, (4, 2))])
+def test_verify_tree_baseline_rules_match_oracle(rsd, rule, gamma, dtype, V, branching):
+    B = 40 if V <= 5000 else 12
+    L = len(branching)
+    n_nodes = len(workloads.rsdc_parent_array(branching))
+    P = n_nodes - int(np.prod(branching))
+    # peaked drafts (sigma 3) so that repeated children occur; a target close enough for walks of several lengths
+    base = _rows((B, n_nodes, V), "f32", 3.0, 700 + V)
+    draft = base[:, :P].to(torch.bfloat16 if dtype == "bf16" else torch.float32).contiguous()
+    target = (base + _rows((B, n_nodes, V), "f32", 1.0, 701 + V)).to(draft.dtype).contiguous()
+    draft_h = workloads.as_oracle_rows(draft)
+    parent, token = _iid_tree(draft_h, branching, 5 + rule)
+    par_t, tok_t = torch.from_numpy(parent).cuda(), torch.from_numpy(token).cuda()
+    g = _np(rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, L, rule, gamma, 31, 2, seq_base=7, want_theta=True))
+    o = oracle.verify_tree(draft_h, workloads.as_oracle_rows(target), parent, token, L, 31, 2, seq_base=7,
+                           rule=rule, gamma=gamma)
+    t = Tally()
+    compare_verify(t, g, o, parent)
+    t.check()
+    assert t.final_mismatch <= max(1, 0.02 * B)
+    assert np.array_equal(g["status"], o["status"])
+    assert len(set(o["accepted_len"].tolist())) > 1
+    assert (o["stop_reason"] == 0).any()                       # some walks end in the rule's residual
+
+
+def test_verify_tree_rule_rrs_is_verify_tree_and_bad_rules_are_refused(rsd):
+    B, V, branching = 8, 515, (3, 2)
+    parent = workloads.rsdc_parent_array(branching)
+    base = _rows((B, len(parent), V), "f32", 2.0, 900)
+    draft = base[:, :4].contiguous()
+    target = (base + _rows((B, len(parent), V), "f32", 1.0, 901)).contiguous()
+    _, token = _iid_tree(workloads.as_oracle_rows(draft), branching, 3)
+    par_t, tok_t = torch.from_numpy(parent).cuda(), torch.from_numpy(token).cuda()
+    a = _np(rsd.rsd_verify_tree(draft, target, par_t, tok_t, 2, 5, 0, want_theta=True))
+    b = _np(rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, rsd.RULE_RRS, 1.0, 5, 0, want_theta=True))
+    for k in a:
+        assert np.array_equal(a[k], b[k], equal_nan=True), k
+    with pytest.raises(rsd.RsdError):
+        rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, 7, 1.0, 5, 0)
+    with pytest.raises(rsd.RsdError):
+        rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, rsd.RULE_KSEQ, 0.5, 5, 0)
