@@ -167,7 +167,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-sequences", type=int, default=16)
-    ap.add_argument("--cpu-baseline-sequences", type=int, default=32)
+    ap.add_argument("--cpu-baseline-sequences", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--sequences", type=int, default=0, help="sequences per GPU (default: the workload's batch)")

@@ -5,6 +5,20 @@
 
 using namespace rsd_host;
 
+namespace {
+// SMs of the current device (asked once per device; 148 if the query fails)
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        cached[dev] = (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0) ? n : 148;
+    }
+    return cached[dev];
+}
+}  // namespace
+
 extern "C" {
 
 int rsd_verify_tree(const rsd_rows* draft, const rsd_rows* target, const rsd_tree* tree, int B, int V, uint64_t seed,
@@ -45,19 +59,25 @@ int rsd_verify_tree_rule(const rsd_rows* draft, const rsd_rows* target, const rs
     a.last_token = last_token; a.stop_reason = stop_reason; a.dbg_theta = dbg_theta; a.status = status;
     cudaStream_t s = (cudaStream_t)stream;
     const bool aligned = rows_aligned(draft) && rows_aligned(target);
-    using namespace rsd;
-#define RSD_LAUNCH_WALK(BASELINES)                                                                                  \
-    do {                                                                                                            \
-        if (draft->dtype == RSD_F32) {                                                                              \
-            if (aligned) verify_tree_kernel<float, true, BASELINES><<<B, kVerifyThreads, 0, s>>>(a);                \
-            else verify_tree_kernel<float, false, BASELINES><<<B, kVerifyThreads, 0, s>>>(a);                       \
-        } else {                                                                                                    \
-            if (aligned) verify_tree_kernel<__nv_bfloat16, true, BASELINES><<<B, kVerifyThreads, 0, s>>>(a);        \
-            else verify_tree_kernel<__nv_bfloat16, false, BASELINES><<<B, kVerifyThreads, 0, s>>>(a);               \
-        }                                                                                                           \
+    // at most one sequence per SM: blocks of 512 threads; otherwise blocks of 256
+#define RSD_LAUNCH_WALK(NS, BASELINES)                                                                                   \
+    do {                                                                                                                 \
+        using namespace rsd::NS;                                                                                         \
+        if (draft->dtype == RSD_F32) {                                                                                   \
+            if (aligned) verify_tree_kernel<float, true, BASELINES><<<B, kVerifyThreads, 0, s>>>(a);                     \
+            else verify_tree_kernel<float, false, BASELINES><<<B, kVerifyThreads, 0, s>>>(a);                            \
+        } else {                                                                                                         \
+            if (aligned) verify_tree_kernel<__nv_bfloat16, true, BASELINES><<<B, kVerifyThreads, 0, s>>>(a);             \
+            else verify_tree_kernel<__nv_bfloat16, false, BASELINES><<<B, kVerifyThreads, 0, s>>>(a);                    \
+        }                                                                                                                \
     } while (0)
-    if (rule == RSD_RULE_RRS) RSD_LAUNCH_WALK(false);
-    else RSD_LAUNCH_WALK(true);
+    const bool wide_blocks = B <= sm_count();
+    if (rule == RSD_RULE_RRS) {
+        if (wide_blocks) RSD_LAUNCH_WALK(walk_wide, false);
+        else RSD_LAUNCH_WALK(walk_narrow, false);
+    } else {
+        RSD_LAUNCH_WALK(walk_narrow, true);
+    }
 #undef RSD_LAUNCH_WALK
     return check_launch("rsd_verify_tree_rule");
 }
@@ -84,7 +104,7 @@ int rsd_resample_residual(const rsd_rows* draft_row, const rsd_rows* target_row,
     a.out_token = out_token; a.out_residual = out_residual; a.status = status;
     cudaStream_t s = (cudaStream_t)stream;
     const bool aligned = rows_aligned(target_row) && (!rejected || rows_aligned(draft_row));
-    using namespace rsd;
+    using namespace rsd::walk_narrow;
     if (target_row->dtype == RSD_F32) {
         if (aligned) resample_residual_kernel<float, true><<<B, kVerifyThreads, 0, s>>>(a);
         else resample_residual_kernel<float, false><<<B, kVerifyThreads, 0, s>>>(a);

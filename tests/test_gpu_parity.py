@@ -444,3 +444,25 @@ def test_verify_tree_rule_rrs_is_verify_tree_and_bad_rules_are_refused(rsd):
         rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, 7, 1.0, 5, 0)
     with pytest.raises(rsd.RsdError):
         rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, rsd.RULE_KSEQ, 0.5, 5, 0)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_verify_tree_more_sequences_than_sms(rsd, dtype):
+    # batches above one sequence per SM run the walk in blocks of 256 threads, smaller ones in blocks of 512: the
+    # other verification tests here are small batches, this one is not
+    B, V, branching = 200, 1030, (3, 2, 2)
+    L = len(branching)
+    parent = workloads.rsdc_parent_array(branching)
+    n_nodes = len(parent)
+    k, nodes = workloads.rsdc_rows(branching)
+    base = _rows((B, n_nodes, V), "f32", 2.0, 1500)
+    draft = base[:, :len(k)].to(torch.bfloat16 if dtype == "bf16" else torch.float32).contiguous()
+    target = (base + _rows((B, n_nodes, V), "f32", 1.0, 1501)).to(draft.dtype).contiguous()
+    o_draft = oracle.gumbel_topk(workloads.as_oracle_rows(draft), k, nodes, 29, 0)
+    token = workloads.rsdc_tokens_from_rows(branching, o_draft["token"])
+    g, o = _verify_both(rsd, draft, target, parent, token, L, 29, 0)
+    t = Tally()
+    compare_verify(t, g, o, parent)
+    t.check()
+    assert t.final_mismatch <= 0.02 * B
+    assert np.array_equal(g["status"], o["status"])
