@@ -293,8 +293,14 @@ def main():
                 "launch_ms_by_level": [sum(scan_ev[s][l][0].elapsed_time(scan_ev[s][l][1]) for s in range(K)) / K
                                        for l in range(n_scan)],
                 "share_of_step": scan_ms / elapsed_ms,
-                "verify_walk": {"achieved": ver_gbs, "frac": ver_gbs / peak, "algorithmic_bytes_last_step": ver_bytes,
+                "frac_of_nominal_8000_gbs": scan_gbs / 8000.0,
+                "verify_walk": {"achieved": ver_gbs, "frac": ver_gbs / peak, "frac_of_nominal_8000_gbs": ver_gbs / 8000.0,
+                                "algorithmic_bytes_last_step": ver_bytes,
                                 "avg_launch_ms": ver_ms / K, "share_of_step": ver_ms / elapsed_ms}}
+    # the same nodes counted against the drafting launches alone (scans; SBS epilogues excluded) and the walk alone,
+    # timed on this rank
+    phases = {"draft_scan_only_nodes_per_s": nodes_per_step * K / (scan_ms * 1e-3),
+              "verify_only_nodes_per_s": nodes_per_step * K / (ver_ms * 1e-3)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
             "ms_per_step": elapsed_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -306,7 +312,8 @@ def main():
                        "l2": "inputs larger than L2 (%.2f GB resident per GPU)" % (resident_bytes / 1e9)
                        if resident_bytes > 256e6 else "inputs smaller than L2: timings are cache-assisted",
                        "mean_accepted_len": float(acc.mean())},
-            "clocks": clocks.summary(), "gpu_launches": stepper.kernel_launches * K, "roofline": roofline}
+            "clocks": clocks.summary(), "gpu_launches": stepper.kernel_launches * K, "roofline": roofline,
+            "phases": phases}
 
     # ---- end to end: pinned host logits -> device -> step -> results on the host ---------------------------
     if not args.no_e2e:

@@ -195,7 +195,8 @@ int rsd_verify_tree(const rsd_rows* draft, const rsd_rows* target, const rsd_tre
                     int32_t* status, rsd_stream_t stream);
 
 /*
- * rsd_verify_tree with the verification rule as an argument: recursive rejection sampling, or one of the two
+ * rsd_verify_tree with the verification rule and the sampler of the last token as arguments: recursive rejection
+ * sampling, or one of the two
  * earlier tree verifiers that Section 2 describes, run over the same tree layout, rows and random streams, so that
  * acceptance rates can be compared on equal inputs (Figure 1 does this for Bernoulli distributions).
  *   RSD_RULE_RRS         recursive rejection sampling (Section 3.1): exactly rsd_verify_tree
@@ -208,12 +209,18 @@ int rsd_verify_tree(const rsd_rows* draft, const rsd_rows* target, const rsd_tre
  *                        token is drawn from Norm[(q - min{p, q/gamma} (1 - (1 - beta)^K) / beta)+] with
  *                        beta = sum_x min{p(x), q(x)/gamma}.  gamma in [1, K]; gamma = K is always admissible
  *                        (smaller values need (1 - (1 - beta)^K) / beta <= gamma, else the clamp at 0 applies)
- * gamma is read only by RSD_RULE_KSEQ (finite, >= 1).  All other arguments, outputs and status bits as in
- * rsd_verify_tree; RSD_ST_ZERO_RESIDUAL under K-SEQ means the token was drawn from the target row itself.
+ * gamma is read only by RSD_RULE_KSEQ (finite, >= 1).
+ * final_sampler chooses how the last token is drawn from its distribution w (a residual or a target row):
+ *   RSD_FINAL_INVERSE_CDF  one uniform, smallest y whose running sum of w exceeds u * sum(w): rsd_verify_tree's way
+ *   RSD_FINAL_GUMBEL_TOP1  arg max over y of log w(y) + G(y) with fresh standard Gumbel noise G (Algorithm 6's last
+ *                          step; the same law), drawn group-wise like the drafting noise from streams of its own
+ * All other arguments, outputs and status bits as in rsd_verify_tree; RSD_ST_ZERO_RESIDUAL under K-SEQ means the
+ * token was drawn from the target row itself.
  */
 enum { RSD_RULE_RRS = 0, RSD_RULE_MULTIROUND = 1, RSD_RULE_KSEQ = 2 };
+enum { RSD_FINAL_INVERSE_CDF = 0, RSD_FINAL_GUMBEL_TOP1 = 1 };
 int rsd_verify_tree_rule(const rsd_rows* draft, const rsd_rows* target, const rsd_tree* tree, int B, int V,
-                         int rule, float gamma, uint64_t seed, uint32_t step, uint32_t seq_base,
+                         int rule, float gamma, int final_sampler, uint64_t seed, uint32_t step, uint32_t seq_base,
                          int32_t* accepted_len, int32_t* accepted_node, int32_t* accepted_token, int32_t* last_token,
                          int32_t* stop_reason, float* dbg_theta, int32_t* status, rsd_stream_t stream);
 

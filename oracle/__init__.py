@@ -197,10 +197,11 @@ RULE_RRS, RULE_MULTIROUND, RULE_KSEQ = 0, 1, 2
 
 
 def verify_tree(draft, target, parent, token, num_levels, seed, step, *, seq_base=0, want_weights=False,
-                draft_temperature=1.0, target_temperature=1.0, rule=RULE_RRS, gamma=1.0):
+                draft_temperature=1.0, target_temperature=1.0, rule=RULE_RRS, gamma=1.0, final_sampler=0):
     """draft [B,P,V], target [B,N+1,V], parent [N+1] or [B,N+1] (flat, root -1), token [B,N+1].
     rule: recursive rejection sampling (the paper's), or one of the two baselines of Section 2 on the same tree:
-    multi-round rejection sampling with one draft model, K-SEQ with parameter gamma."""
+    multi-round rejection sampling with one draft model, K-SEQ with parameter gamma.
+    final_sampler: 0 = inverse CDF with one uniform, 1 = Gumbel-Top-1 (Algorithm 6's last step)."""
     d, ddt = _rows(draft)
     t, tdt = _rows(target)
     B, _, V = t.shape
@@ -219,7 +220,7 @@ def verify_tree(draft, target, parent, token, num_levels, seed, step, *, seq_bas
     fmargin = np.zeros(B, np.float64)
     weights = np.zeros((B, V), np.float64) if want_weights else None
     status = np.zeros(B, np.int32)
-    lib().rsd_oracle_verify_tree_rule(C.c_int(int(rule)), C.c_double(float(gamma)),
+    lib().rsd_oracle_verify_tree_rule(C.c_int(int(rule)), C.c_double(float(gamma)), C.c_int(int(final_sampler)),
                                  _ptr(d), C.c_int(ddt), C.c_int64(d.strides[0] // d.itemsize),
                                  C.c_int64(d.strides[1] // d.itemsize), C.c_double(draft_temperature),
                                  _ptr(t), C.c_int(tdt), C.c_int64(t.strides[0] // t.itemsize),

@@ -53,6 +53,8 @@
 #define TAG_GUMBEL_FINE 1u
 #define TAG_ACCEPT 2u
 #define TAG_RESAMPLE 3u
+#define TAG_FINAL_GUMBEL_COARSE 4u /* Gumbel-Top-1 draw of the last token: same group-wise layout, own streams */
+#define TAG_FINAL_GUMBEL_FINE 5u
 
 /* ------------------------------------------------------------------------ */
 /* Philox4x32-10, written from the published definition: ten rounds of      */
@@ -129,6 +131,37 @@ double rsd_oracle_gumbel(uint64_t seed, uint32_t step, uint32_t seq, uint32_t no
     int32_t a;
     rsd_oracle_gumbel_parts(seed, step, seq, node, e, &tg, &a, &te);
     return -log(tg / 16.0 + ((int32_t)(e & 15u) != a ? te : 0.0));
+}
+
+/* Gumbel noise of element e for the Gumbel-Top-1 draw of the last token at `node` (same law and layout as above) */
+static double final_gumbel(uint64_t seed, uint32_t step, uint32_t seq, uint32_t node, uint32_t e) {
+    uint32_t w[4];
+    const uint32_t g = e >> 4;
+    draw(seed, step, seq, node, TAG_FINAL_GUMBEL_COARSE, ((g >> 7) << 5) | (g & 31u), w);
+    const uint32_t word = w[(g >> 5) & 3u];
+    const double tg = -log(((double)(word >> 4) + 0.5) * (1.0 / 268435456.0));
+    const int32_t a = (int32_t)(word & 15u);
+    draw(seed, step, seq, node, TAG_FINAL_GUMBEL_FINE, e >> 2, w);
+    const double te = neg_log_uniform(w[e & 3u]);
+    return -log(tg / 16.0 + ((int32_t)(e & 15u) != a ? te : 0.0));
+}
+
+/*
+ * Last token by Gumbel-Top-1 (Algorithm 6's final step): arg max over y of log w(y) + G(y), entries with
+ * w(y) = 0 left out; equal values go to the smaller token.  margin = gap to the runner-up.  -1 if w has no mass.
+ */
+static int gumbel_top1(const double* w, int V, uint64_t seed, uint32_t step, uint32_t seq, uint32_t node,
+                       double* margin) {
+    int best = -1;
+    double vb = -INFINITY, v2 = -INFINITY;
+    for (int y = 0; y < V; ++y) {
+        if (!(w[y] > 0.0)) continue;
+        double v = log(w[y]) + final_gumbel(seed, step, seq, node, (uint32_t)y);
+        if (v > vb) { v2 = vb; vb = v; best = y; }
+        else if (v > v2) v2 = v;
+    }
+    if (margin) *margin = (best >= 0) ? vb - v2 : 0.0;
+    return best;
 }
 
 /* U for the acceptance test of the j-th child (stored order) of `node`: 24 bits, in [0,1) */
@@ -548,7 +581,7 @@ int rsd_oracle_rrs_chain(const double* p_in, const double* q_in, int V, const in
  * out_final_weights: optional [B][V], the normalised distribution the last
  * token was drawn from.
  */
-int rsd_oracle_verify_tree_rule(int rule, double gamma,
+int rsd_oracle_verify_tree_rule(int rule, double gamma, int final_sampler /* 0 inverse CDF, 1 Gumbel-Top-1 */,
                            const void* draft, int draft_dtype, int64_t draft_seq_stride, int64_t draft_row_stride,
                            double draft_temperature,
                            const void* target, int target_dtype, int64_t target_seq_stride, int64_t target_row_stride,
@@ -611,9 +644,13 @@ int rsd_oracle_verify_tree_rule(int rule, double gamma,
             ++len;
             cur = accepted_child;
         }
-        double u = rsd_oracle_resample_uniform(seed, step, seq, (uint32_t)cur);
         double fm = 0.0;
-        last_token[b] = rsd_oracle_inverse_cdf(q, V, u, &fm);
+        if (final_sampler == 1) {
+            last_token[b] = gumbel_top1(q, V, seed, step, seq, (uint32_t)cur, &fm);
+        } else {
+            double u = rsd_oracle_resample_uniform(seed, step, seq, (uint32_t)cur);
+            last_token[b] = rsd_oracle_inverse_cdf(q, V, u, &fm);
+        }
         if (final_margin) final_margin[b] = fm;
         if (out_final_weights) memcpy(out_final_weights + (int64_t)b * V, q, sizeof(double) * (size_t)V);
         accepted_len[b] = len;
@@ -636,7 +673,7 @@ int rsd_oracle_verify_tree(const void* draft, int draft_dtype, int64_t draft_seq
                            int32_t* last_token, int32_t* stop_reason,
                            double* dbg_theta, double* dbg_margin, double* final_margin, double* out_final_weights,
                            int32_t* status) {
-    return rsd_oracle_verify_tree_rule(0, 1.0, draft, draft_dtype, draft_seq_stride, draft_row_stride, draft_temperature,
+    return rsd_oracle_verify_tree_rule(0, 1.0, 0, draft, draft_dtype, draft_seq_stride, draft_row_stride, draft_temperature,
                                        target, target_dtype, target_seq_stride, target_row_stride, target_temperature,
                                        B, V, n_nodes, num_levels, parent, topology_is_shared, token, seed, step,
                                        seq_base, accepted_len, accepted_node, accepted_token, last_token, stop_reason,

@@ -19,6 +19,7 @@ RSD_F32, RSD_BF16 = 0, 1
 ST_NAN_INPUT, ST_FEWER_THAN_K, ST_ZERO_RESIDUAL, ST_ZERO_DRAFT_PROB, ST_DRAFT_EXHAUSTED = 1, 2, 4, 8, 16
 STOP_ALL_REJECTED, STOP_NO_CHILDREN, STOP_LEAF = 0, 1, 2
 RULE_RRS, RULE_MULTIROUND, RULE_KSEQ = 0, 1, 2
+FINAL_INVERSE_CDF, FINAL_GUMBEL_TOP1 = 0, 1
 MAX_K = 32
 
 EXPORTS = ["rsd_version", "rsd_rng_layout", "rsd_last_error", "rsd_profile_next_scan", "rsd_gumbel_topk_draft", "rsd_sbs_workspace_bytes",
@@ -69,7 +70,7 @@ def lib():
                                       C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         l.rsd_verify_tree_rule.argtypes = [C.POINTER(RsdRows), C.POINTER(RsdRows), C.POINTER(RsdTree), C.c_int, C.c_int,
-                                           C.c_int, C.c_float, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
+                                           C.c_int, C.c_float, C.c_int, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                            C.c_void_p]
         l.rsd_resample_residual.argtypes = [C.POINTER(RsdRows), C.POINTER(RsdRows), C.c_int, C.c_int, C.c_void_p,
@@ -213,9 +214,10 @@ def rsd_sbs_step_static(draft_level: torch.Tensor, W: int, first_parent_node: in
 def rsd_verify_tree(draft: torch.Tensor, target: torch.Tensor, parent: torch.Tensor, token: torch.Tensor,
                     num_levels: int, seed: int, step: int, *, seq_base: int = 0, want_theta: bool = False,
                     out: Optional[dict] = None, draft_temperature: float = 1.0, target_temperature: float = 1.0,
-                    rule: int = 0, gamma: float = 1.0):
+                    rule: int = 0, gamma: float = 1.0, final_sampler: int = 0, _force_rule_entry: bool = False):
     """draft [B, P, V], target [B, N+1, V], parent [N+1] or [B, N+1] int32, token [B, N+1] int32.
-    rule = RULE_RRS calls rsd_verify_tree; RULE_MULTIROUND / RULE_KSEQ call rsd_verify_tree_rule."""
+    rule = RULE_RRS with final_sampler = FINAL_INVERSE_CDF calls rsd_verify_tree; anything else calls
+    rsd_verify_tree_rule."""
     B, _, V = target.shape
     dev = target.device
     n_nodes = token.shape[1]
@@ -236,18 +238,20 @@ def rsd_verify_tree(draft: torch.Tensor, target: torch.Tensor, parent: torch.Ten
     d, t = rows_of(draft, False, draft_temperature), rows_of(target, False, target_temperature)
     outs = (_ptr(out["accepted_len"]), _ptr(out["accepted_node"]), _ptr(out["accepted_token"]),
             _ptr(out["last_token"]), _ptr(out["stop_reason"]), _ptr(out.get("theta")), _ptr(out["status"]), _stream())
-    if rule == RULE_RRS:
+    if rule == RULE_RRS and final_sampler == FINAL_INVERSE_CDF and not _force_rule_entry:
         _check(lib().rsd_verify_tree(C.byref(d), C.byref(t), C.byref(tree), B, V, seed, step, seq_base, *outs))
     else:
         _check(lib().rsd_verify_tree_rule(C.byref(d), C.byref(t), C.byref(tree), B, V, int(rule), float(gamma),
-                                          seed, step, seq_base, *outs))
+                                          int(final_sampler), seed, step, seq_base, *outs))
     return out
 
 
 def rsd_verify_tree_rule(draft: torch.Tensor, target: torch.Tensor, parent: torch.Tensor, token: torch.Tensor,
-                         num_levels: int, rule: int, gamma: float, seed: int, step: int, **kw):
-    """rsd_verify_tree with a verification rule (RULE_RRS, RULE_MULTIROUND, RULE_KSEQ with its gamma)."""
-    return rsd_verify_tree(draft, target, parent, token, num_levels, seed, step, rule=rule, gamma=gamma, **kw)
+                         num_levels: int, rule: int, gamma: float, final_sampler: int, seed: int, step: int, **kw):
+    """rsd_verify_tree with a verification rule (RULE_RRS, RULE_MULTIROUND, RULE_KSEQ with its gamma) and a sampler
+    of the last token (FINAL_INVERSE_CDF, FINAL_GUMBEL_TOP1)."""
+    return rsd_verify_tree(draft, target, parent, token, num_levels, seed, step, rule=rule, gamma=gamma,
+                           final_sampler=final_sampler, _force_rule_entry=True, **kw)
 
 
 def rsd_resample_residual(draft_row: Optional[torch.Tensor], target_row: torch.Tensor,

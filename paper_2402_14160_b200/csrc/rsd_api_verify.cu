@@ -25,17 +25,19 @@ int rsd_verify_tree(const rsd_rows* draft, const rsd_rows* target, const rsd_tre
                     uint32_t step, uint32_t seq_base, int32_t* accepted_len, int32_t* accepted_node,
                     int32_t* accepted_token, int32_t* last_token, int32_t* stop_reason, float* dbg_theta,
                     int32_t* status, rsd_stream_t stream) {
-    return rsd_verify_tree_rule(draft, target, tree, B, V, RSD_RULE_RRS, 1.0f, seed, step, seq_base, accepted_len,
+    return rsd_verify_tree_rule(draft, target, tree, B, V, RSD_RULE_RRS, 1.0f, RSD_FINAL_INVERSE_CDF, seed, step, seq_base, accepted_len,
                                 accepted_node, accepted_token, last_token, stop_reason, dbg_theta, status, stream);
 }
 
 int rsd_verify_tree_rule(const rsd_rows* draft, const rsd_rows* target, const rsd_tree* tree, int B, int V, int rule,
-                         float gamma, uint64_t seed, uint32_t step, uint32_t seq_base, int32_t* accepted_len,
+                         float gamma, int final_sampler, uint64_t seed, uint32_t step, uint32_t seq_base, int32_t* accepted_len,
                          int32_t* accepted_node, int32_t* accepted_token, int32_t* last_token, int32_t* stop_reason,
                          float* dbg_theta, int32_t* status, rsd_stream_t stream) {
     g_err[0] = 0;
     if (rule != RSD_RULE_RRS && rule != RSD_RULE_MULTIROUND && rule != RSD_RULE_KSEQ)
         return fail(RSD_ERR_INVALID_ARG, "unknown verification rule %d", rule);
+    if (final_sampler != RSD_FINAL_INVERSE_CDF && final_sampler != RSD_FINAL_GUMBEL_TOP1)
+        return fail(RSD_ERR_INVALID_ARG, "unknown sampler of the last token %d", final_sampler);
     if (rule == RSD_RULE_KSEQ && !(gamma >= 1.0f && gamma < 3.0e38f))
         return fail(RSD_ERR_INVALID_ARG, "K-SEQ: gamma = %g must be a finite number >= 1", (double)gamma);
     if (int e = check_vocab(V)) return e;
@@ -52,7 +54,7 @@ int rsd_verify_tree_rule(const rsd_rows* draft, const rsd_rows* target, const rs
     a.draft = {draft->data, draft->seq_stride, draft->row_stride, 1.0f / temperature_of(draft)};
     a.target = {target->data, target->seq_stride, target->row_stride, 1.0f / temperature_of(target)};
     a.V = V; a.L = tree->num_levels; a.num_nodes = tree->num_nodes; a.shared_topology = tree->topology_is_shared;
-    a.rule = rule; a.gamma = rule == RSD_RULE_KSEQ ? gamma : 1.0f;
+    a.rule = rule; a.gamma = rule == RSD_RULE_KSEQ ? gamma : 1.0f; a.final_sampler = final_sampler;
     a.parent = tree->parent; a.token = tree->token;
     a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
     a.accepted_len = accepted_len; a.accepted_node = accepted_node; a.accepted_token = accepted_token;
@@ -72,7 +74,7 @@ int rsd_verify_tree_rule(const rsd_rows* draft, const rsd_rows* target, const rs
         }                                                                                                                \
     } while (0)
     const bool wide_blocks = B <= sm_count();
-    if (rule == RSD_RULE_RRS) {
+    if (rule == RSD_RULE_RRS && final_sampler == RSD_FINAL_INVERSE_CDF) {
         if (wide_blocks) RSD_LAUNCH_WALK(walk_wide, false);
         else RSD_LAUNCH_WALK(walk_narrow, false);
     } else {

@@ -8,6 +8,7 @@
 namespace rsd {
 
 constexpr uint32_t kTagGumbelCoarse = 0u, kTagGumbelFine = 1u, kTagAccept = 2u, kTagResample = 3u;
+constexpr uint32_t kTagFinalGumbelCoarse = 4u, kTagFinalGumbelFine = 5u;   // Gumbel-Top-1 draw of the last token
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kNegInf = -__builtin_huge_valf();
 

@@ -39,6 +39,7 @@ struct VerifyArgs {
     int V, L, num_nodes, shared_topology;
     int rule;      // 0 recursive rejection sampling, 1 multi-round rejection sampling, 2 K-SEQ
     float gamma;   // K-SEQ's parameter
+    int final_sampler;   // 0 inverse CDF with one uniform, 1 Gumbel-Top-1
     const int32_t* parent;
     const int32_t* token;
     uint32_t seed_lo, seed_hi, step, seq_base;

@@ -402,9 +402,9 @@ def _iid_tree(draft_h, branching, seed):
     return parent, token
 
 
-@pytest.mark.parametrize("rule,gamma", [(1, 1.0), (2, 3.0), (2, 1.5)])
+@pytest.mark.parametrize("rule,gamma,sampler", [(1, 1.0, 0), (2, 3.0, 0), (2, 1.5, 0), (0, 1.0, 1), (1, 1.0, 1), (2, 2.0, 1)])
 @pytest.mark.parametrize("dtype,V,branching", [("f32", 97, (3, 3)), ("bf16", 4099, (3, 2, 2)), ("bf16", 32000, (4, 2))])
-def test_verify_tree_baseline_rules_match_oracle(rsd, rule, gamma, dtype, V, branching):
+def test_verify_tree_baseline_rules_match_oracle(rsd, rule, gamma, sampler, dtype, V, branching):
     B = 40 if V <= 5000 else 12
     L = len(branching)
     n_nodes = len(workloads.rsdc_parent_array(branching))
@@ -414,11 +414,16 @@ def test_verify_tree_baseline_rules_match_oracle(rsd, rule, gamma, dtype, V, bra
     draft = base[:, :P].to(torch.bfloat16 if dtype == "bf16" else torch.float32).contiguous()
     target = (base + _rows((B, n_nodes, V), "f32", 1.0, 701 + V)).to(draft.dtype).contiguous()
     draft_h = workloads.as_oracle_rows(draft)
-    parent, token = _iid_tree(draft_h, branching, 5 + rule)
+    if rule == 0:   # recursive rejection sampling verifies drafts without replacement
+        k, nodes = workloads.rsdc_rows(branching)
+        parent = workloads.rsdc_parent_array(branching)
+        token = workloads.rsdc_tokens_from_rows(branching, oracle.gumbel_topk(draft_h, k, nodes, 31, 2, seq_base=7)["token"])
+    else:
+        parent, token = _iid_tree(draft_h, branching, 5 + rule)
     par_t, tok_t = torch.from_numpy(parent).cuda(), torch.from_numpy(token).cuda()
-    g = _np(rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, L, rule, gamma, 31, 2, seq_base=7, want_theta=True))
+    g = _np(rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, L, rule, gamma, sampler, 31, 2, seq_base=7, want_theta=True))
     o = oracle.verify_tree(draft_h, workloads.as_oracle_rows(target), parent, token, L, 31, 2, seq_base=7,
-                           rule=rule, gamma=gamma)
+                           rule=rule, gamma=gamma, final_sampler=sampler)
     t = Tally()
     compare_verify(t, g, o, parent)
     t.check()
@@ -437,13 +442,15 @@ def test_verify_tree_rule_rrs_is_verify_tree_and_bad_rules_are_refused(rsd):
     _, token = _iid_tree(workloads.as_oracle_rows(draft), branching, 3)
     par_t, tok_t = torch.from_numpy(parent).cuda(), torch.from_numpy(token).cuda()
     a = _np(rsd.rsd_verify_tree(draft, target, par_t, tok_t, 2, 5, 0, want_theta=True))
-    b = _np(rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, rsd.RULE_RRS, 1.0, 5, 0, want_theta=True))
+    b = _np(rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, rsd.RULE_RRS, 1.0, rsd.FINAL_INVERSE_CDF, 5, 0, want_theta=True))
     for k in a:
         assert np.array_equal(a[k], b[k], equal_nan=True), k
     with pytest.raises(rsd.RsdError):
-        rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, 7, 1.0, 5, 0)
+        rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, 7, 1.0, 0, 5, 0)
     with pytest.raises(rsd.RsdError):
-        rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, rsd.RULE_KSEQ, 0.5, 5, 0)
+        rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, rsd.RULE_KSEQ, 0.5, 0, 5, 0)
+    with pytest.raises(rsd.RsdError):
+        rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, rsd.RULE_RRS, 1.0, 3, 5, 0)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])

@@ -177,3 +177,28 @@ def test_resample_residual_entry():
     for b in range(B):
         _, expect, _ = oracle.rrs_chain(_softmax(d[b]), _softmax(t[b]), [3, 8])
         assert np.allclose(res["residual"][b], expect, atol=1e-15)
+
+
+def test_gumbel_top1_final_token_follows_the_residual():
+    # Algorithm 6 draws the last token by Gumbel-Top-1: over many independent sequences its law must be the
+    # distribution it is drawn from (here: the target row of a root without children), like the inverse-CDF draw
+    rng = np.random.default_rng(41)
+    V, B = 50, 40000
+    row = rng.normal(0, 1.5, V).astype(np.float32)
+    row[7] = -np.inf                                           # a token without mass is never drawn
+    target = np.broadcast_to(row, (B, 1, V)).copy()
+    draft = np.zeros((B, 1, V), np.float32)
+    parent = np.array([-1], np.int32)
+    token = np.full((B, 1), -1, np.int32)
+    q = np.exp(row.astype(np.float64) - row[np.isfinite(row)].max())
+    q /= q.sum()
+    laws = {}
+    for sampler in (0, 1):
+        out = oracle.verify_tree(draft, target, parent, token, 0, seed=5, step=1, final_sampler=sampler)
+        counts = np.bincount(out["last_token"], minlength=V).astype(np.float64)
+        assert counts[7] == 0
+        keep = q > 0
+        chi2 = (((counts - B * q) ** 2)[keep] / (B * q[keep])).sum()
+        assert chi2 < 100.0, (sampler, chi2)                  # 48 degrees of freedom: 100 is far in the tail
+        laws[sampler] = out["last_token"]
+    assert (laws[0] != laws[1]).mean() > 0.5                    # two different samplers, one law
