@@ -25,7 +25,10 @@ namespace rsd {
 constexpr int kMaxTiles = 512;        // tiles of 512 elements: V <= 262144
 constexpr int kMaxCachedNodes = 384;  // trees up to this size are copied to shared memory
 constexpr int kMaxRemoved = 32;      // removed tokens tracked per node (later ones carry no residual mass)
-constexpr int kPassUnroll = 4;        // turns of a pass whose warp-wide sums are taken together
+#ifndef RSD_PASS_UNROLL
+#define RSD_PASS_UNROLL 4
+#endif
+constexpr int kPassUnroll = RSD_PASS_UNROLL;        // turns of a pass whose warp-wide sums are taken together
 constexpr float kRefSlack = 60.0f;    // redo a pass if the row maximum exceeds its reference by more than this
 
 struct RowsDev {
