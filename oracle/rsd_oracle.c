@@ -17,7 +17,7 @@
  * Random numbers.  The paper only says "standard Gumbel" and "Uniform[0,1]".
  * Both sides of the parity check draw them from the counter-based generator
  * Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) with the counter layout
- * documented at rsd_oracle_gumbel() below (RNG layout version 2).
+ * documented at draw() and rsd_oracle_gumbel() below (RNG layout version 3).
  *
  * Pins (see tests, "-m 'not gpu'"): Philox known answers and bijectivity,
  * Gumbel moments/CDF, Plackett-Luce law of Gumbel-Top-k, exact enumeration of
@@ -80,7 +80,7 @@ void rsd_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint
 }
 
 /*
- * RNG layout version 1.  key = (seed low word, seed high word).
+ * Counter and key of every stream (RNG layout version 3).  key = (seed low word, seed high word).
  * counter = (index, node | tag << 28, sequence, step) where
  *   node     = flat node id inside the sequence's tree (< 2^28),
  *   sequence = global sequence index of the batch,

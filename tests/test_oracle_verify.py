@@ -202,3 +202,34 @@ def test_gumbel_top1_final_token_follows_the_residual():
         assert chi2 < 100.0, (sampler, chi2)                  # 48 degrees of freedom: 100 is far in the tail
         laws[sampler] = out["last_token"]
     assert (laws[0] != laws[1]).mean() > 0.5                    # two different samplers, one law
+
+
+def test_first_emitted_token_is_target_distributed_with_gumbel_top1_last_draw():
+    # Theorem 3.1 with Algorithm 6's own last step: three children of the root drawn by Gumbel-Top-k, the walk, and
+    # the last token by Gumbel-Top-1 on the residual.  The noise of that last draw must be independent of the noise
+    # that drafted the children (it has streams of its own): were it the node's drafting noise again, the residual
+    # draw after three rejections would lean towards the fourth-best perturbed draft value and the first emitted
+    # token would no longer follow q(. | root).
+    rng = np.random.default_rng(44)
+    V, n, K = 50, 60000, 3
+    ld = rng.normal(0, 1.5, V).astype(np.float32)
+    lt = (ld + rng.normal(0, 1.5, V)).astype(np.float32)      # far apart: all three rejected fairly often
+    q = _softmax(lt)
+    draft = np.broadcast_to(ld[None, None, :], (n, 1, V))
+    target = np.broadcast_to(lt[None, None, :], (n, 1 + K, V))
+    parent = np.array([-1, 0, 0, 0], np.int32)
+    d = oracle.gumbel_topk(draft, [K], [0], seed=13, step=5)
+    token = np.concatenate([np.full((n, 1), -1, np.int32), d["token"][:, 0, :]], 1)
+    out = oracle.verify_tree(draft, target, parent, token, 1, seed=13, step=5, final_sampler=1)
+    rejected_all = out["accepted_len"] == 0
+    assert 0.1 < rejected_all.mean() < 0.9                    # both branches carry weight
+    first = np.where(out["accepted_len"] > 0, out["accepted_token"][:, 0], out["last_token"])
+    counts = np.bincount(first, minlength=V).astype(float)
+    keep = q * n > 5
+    obs = np.append(counts[keep], counts[~keep].sum())
+    exp = np.append(q[keep] * n, q[~keep].sum() * n)
+    assert stats.chisquare(obs, exp).pvalue > 1e-3
+    # the same law as with the inverse-CDF draw, from different random numbers
+    out0 = oracle.verify_tree(draft, target, parent, token, 1, seed=13, step=5, final_sampler=0)
+    assert np.array_equal(out0["accepted_len"], out["accepted_len"])
+    assert (out0["last_token"][rejected_all] != out["last_token"][rejected_all]).mean() > 0.3
