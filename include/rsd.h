@@ -140,7 +140,9 @@ int rsd_gumbel_topk_draft(const rsd_rows* draft, int B, int R, int V, const int3
  *                     parent_base + slot index within the level, so with out_token/out_parent pointing at a level's
  *                     first node inside [B][N+1] tree arrays and parent_base = first_parent_node the tree arrays
  *                     of rsd_verify_tree are filled in place; entries beyond out_count[b] are -1
- *   sum_logprob_out, trunc_gumbel_out  [B][W] fp32: phi and psi of each pick, the next level's inputs
+ *   sum_logprob_out, trunc_gumbel_out  [B][W] fp32: phi and psi of each pick, the next level's inputs; entries
+ *                     beyond out_count[b] are -inf.  On input, a parent slot whose sum_logprob_in or
+ *                     trunc_gumbel_in is -inf is such an empty slot: it contributes no children.
  *   out_count         [B]
  *   ws                scratch of at least rsd_sbs_workspace_bytes(B, n_par, W) bytes, 256-byte aligned; contents
  *                     are undefined afterwards; calls that overlap on the GPU need separate scratch
@@ -163,7 +165,8 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
  *   - Sizes: rsd_sbs_workspace_bytes(B, n_par, W) must not exceed RSD_SBS_STATIC_SCRATCH_BYTES (for example
  *     B = 1024, n_par = 8, W = 8 needs 851,968 bytes); larger calls return RSD_ERR_WORKSPACE with a message.
  *   - The first call on each device looks up the array's device address (with that device current) and keeps it;
- *     make that first call outside any stream capture.
+ *     make that first call outside any stream capture.  The kept address belongs to the device's current context:
+ *     after a cudaDeviceReset() in this process it is stale and this entry point must not be used any more.
  *   - All calls on a device share the one array.  Nothing in it has to start at zero (every entry is written before
  *     it is read) and its contents after a call are unspecified.  Two calls that overlap on the same GPU (different
  *     streams, or different host threads) race on it: order them, or use rsd_sbs_step with separate scratch.

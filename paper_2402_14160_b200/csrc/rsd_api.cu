@@ -20,11 +20,13 @@ thread_local cudaEvent_t g_scan_before = nullptr, g_scan_after = nullptr;  // on
 template <typename T, bool ALIGNED, bool WIDE, bool NEED_LSE, bool TEMP>
 void launch_scan_temp(int blocks, const rsd::ScanArgs& a, cudaStream_t s) {
     const size_t smem = sizeof(float) * (size_t)((((a.V + 15) / 16) + 3) / 4 * 4);  // one bound per group of 16 elements, padded to fours
-    static bool raised = false;  // per instantiation: allow the largest vocabulary's dynamic shared memory
-    if (!raised) {
-        cudaFuncSetAttribute(rsd::scan_topk_kernel<T, ALIGNED, WIDE, NEED_LSE, TEMP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)(sizeof(float) * (RSD_MAX_VOCAB / 16)));
-        raised = true;
+    if (smem > 48 * 1024) {
+        // The attribute belongs to the (function, device) pair; it is only needed beyond 48 KB (V > 196,608), so it
+        // is simply set on every such launch instead of being remembered per device.
+        if (cudaFuncSetAttribute(rsd::scan_topk_kernel<T, ALIGNED, WIDE, NEED_LSE, TEMP>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)(sizeof(float) * (RSD_MAX_VOCAB / 16))) != cudaSuccess)
+            return;   // the error stays pending: the caller's check_launch() reports it
     }
     rsd::scan_topk_kernel<T, ALIGNED, WIDE, NEED_LSE, TEMP><<<blocks, rsd::kScanThreads, smem, s>>>(a);
 }
@@ -221,7 +223,11 @@ extern "C" int rsd_sbs_step_static(const rsd_rows* draft_level, int B, int n_par
                                    int64_t out_stride, int32_t parent_base, float* sum_logprob_out,
                                    float* trunc_gumbel_out, int32_t* out_count, int32_t* status, rsd_stream_t stream) {
     g_err[0] = 0;
+    // the argument errors rsd_sbs_step would report come first, so that an oversized n_par or W is named as such
     if (B < 0 || n_par < 1 || W < 1) return fail(RSD_ERR_INVALID_ARG, "B = %d, n_par = %d, W = %d", B, n_par, W);
+    if (n_par > RSD_MAX_ROWS_PER_SEQ) return fail(RSD_ERR_UNSUPPORTED, "n_par = %d > %d", n_par, (int)RSD_MAX_ROWS_PER_SEQ);
+    if (W > RSD_MAX_K) return fail(RSD_ERR_UNSUPPORTED, "W = %d outside [1, %d]", W, (int)RSD_MAX_K);
+    if (n_par * W > 1024) return fail(RSD_ERR_UNSUPPORTED, "n_par * W = %d > 1024", n_par * W);
     const size_t need = rsd_sbs_workspace_bytes(B, n_par, W);
     if (need > (size_t)RSD_SBS_STATIC_SCRATCH_BYTES)
         return fail(RSD_ERR_WORKSPACE,

@@ -836,6 +836,9 @@ static __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(c
     for (int f = tid; f < F; f += kEpilogueThreads) {
         const int kpar = f / a.W;
         int x = a.fin_token[(int64_t)b * F + f];
+        // a parent slot that the level above left empty (its sum or truncated Gumbel is -inf) has no children
+        // (s_gam is -inf exactly for the slots that deliver nothing)
+        if (s_gam[kpar] == kNegInf) x = -1;
         if (x >= 0 && L > kNegInf && f != kpar * a.W) {
             // psi_f < L  <=>  exp(-phi~_f) - exp(-Z) > exp(-L) - exp(-Gamma_k), with Z - phi~_f = the gap d between
             // the parent's best and this finalist's fp32 perturbed values; margins cover the fp32 arithmetic

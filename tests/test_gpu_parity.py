@@ -203,6 +203,30 @@ def test_sbs_parent_with_a_fully_masked_row(rsd):
     assert np.all(g["count"] == W) and not np.any(g["parent"] == 2)
 
 
+def test_sbs_level_after_an_underfull_level(rsd):
+    # A level that finds fewer than W finite candidates pads its outputs with -1 / -inf.  Fed to the next level,
+    # those slots are empty parents: they must contribute no children (no NaN, no pick pointing at them), like the
+    # oracle, which drops every candidate whose sequence log-probability is -inf.
+    W, V = 4, 80
+    root = torch.full((2, 1, V), float("-inf"), device="cuda")
+    root[0, 0, [3, 17, 40]] = torch.tensor([0.5, -0.25, 1.0], device="cuda")      # W - 1 finite entries
+    root[1, 0, [5, 6]] = torch.tensor([0.0, 0.1], device="cuda")                  # W - 2
+    g0 = _np(rsd.rsd_sbs_step(root, W, 0, None, None, 8, 2))
+    o0 = oracle.sbs_step(workloads.as_oracle_rows(root), W, 0, None, None, 8, 2)
+    assert np.array_equal(g0["token"], o0["token"]) and list(g0["count"]) == [3, 2]
+    assert np.all(np.isneginf(g0["sum_logprob"][0, 3:])) and np.all(np.isneginf(g0["trunc_gumbel"][1, 2:]))
+    rows = _rows((2, W, V), "f32", 2.0, 4242)
+    g1 = _np(rsd.rsd_sbs_step(rows, W, 1, torch.from_numpy(g0["sum_logprob"]).cuda(),
+                              torch.from_numpy(g0["trunc_gumbel"]).cuda(), 8, 2, parent_base=1))
+    o1 = oracle.sbs_step(workloads.as_oracle_rows(rows), W, 1, o0["sum_logprob"], o0["trunc_gumbel"], 8, 2)
+    t = Tally()
+    g1_rel = dict(g1, parent=np.where(g1["parent"] >= 0, g1["parent"] - 1, -1))
+    compare_sbs_level(t, g1_rel, o1, W, set())
+    t.check()
+    assert np.all(g1["count"] == W) and not np.any(np.isnan(g1["trunc_gumbel"]))
+    assert np.all(g1_rel["parent"][0] < 3) and np.all(g1_rel["parent"][1] < 2)   # never an empty slot
+
+
 # ---------------------------------------------------------------------------------------------------------
 # verification
 # ---------------------------------------------------------------------------------------------------------

@@ -37,9 +37,17 @@ def test_static_scratch_entry_point_matches_the_caller_scratch_one_twice():
             sig = -torch.rand((B, W), generator=g).cuda() * 5.0
             gam = -torch.sort(torch.rand((B, W), generator=g), dim=1).values.cuda()
         ref = rsd.rsd_sbs_step(rows, W, first_node, sig, gam, 21, step, seq_base=3, parent_base=first_node)
-        got = rsd.rsd_sbs_step_static(rows, W, first_node, sig, gam, 21, step, _outputs(B, W), seq_base=3,
+        outs = _outputs(B, W)
+        torch.cuda.synchronize()
+        # the property the entry point exists for: the call takes no device memory, neither from torch's pool nor
+        # from the driver (the first call on a device only looks an address up)
+        torch_before, (free_before, _) = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()
+        got = rsd.rsd_sbs_step_static(rows, W, first_node, sig, gam, 21, step, outs, seq_base=3,
                                       parent_base=first_node)
         torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == torch_before
+        if done > 0:   # (the very first call on a device may still page the library's image in)
+            assert torch.cuda.mem_get_info()[0] >= free_before
         for key in ("token", "parent", "count", "status"):
             assert torch.equal(ref[key], got[key]), key
         for key in ("sum_logprob", "trunc_gumbel"):
@@ -58,3 +66,28 @@ def test_static_scratch_entry_point_rejects_oversized_calls():
     big = rows.expand(B, n_par, 64)
     with pytest.raises(rsd.RsdError, match="built-in scratch"):
         rsd.rsd_sbs_step_static(big, W, 1, None, None, 0, 0, _outputs(B, W))
+
+
+def test_static_scratch_entry_point_takes_the_largest_documented_batch():
+    # B = 1024, n_par = 8, W = 8 needs 851,968 bytes: the example the header gives as fitting
+    import paper_2402_14160_b200 as rsd
+    B, n_par, W, V = 1024, 8, 8, 256
+    assert rsd.rsd_sbs_workspace_bytes(B, n_par, W) == 851968 <= rsd.api.SBS_STATIC_SCRATCH_BYTES
+    g = torch.Generator(device="cpu").manual_seed(5)
+    rows = (torch.randn((B, n_par, V), generator=g) * 2.0).cuda()
+    sig = -torch.rand((B, n_par), generator=g).cuda() * 3.0
+    gam = -torch.sort(torch.rand((B, n_par), generator=g), dim=1).values.cuda()
+    ref = rsd.rsd_sbs_step(rows, W, 1, sig, gam, 2, 9, parent_base=1)
+    got = rsd.rsd_sbs_step_static(rows, W, 1, sig, gam, 2, 9, _outputs(B, W), parent_base=1)
+    torch.cuda.synchronize()
+    for key in ("token", "parent", "count", "status"):
+        assert torch.equal(ref[key], got[key]), key
+    for key in ("sum_logprob", "trunc_gumbel"):
+        assert torch.allclose(ref[key], got[key], rtol=1e-5, atol=1e-6), key
+
+
+def test_static_scratch_entry_point_names_argument_errors_before_the_size():
+    import paper_2402_14160_b200 as rsd
+    rows = torch.zeros((1, 1, 64), dtype=torch.float32, device="cuda").expand(2, 300, 64)
+    with pytest.raises(rsd.RsdError, match="n_par = 300"):
+        rsd.rsd_sbs_step_static(rows, 4, 1, None, None, 0, 0, _outputs(2, 4))
