@@ -42,10 +42,10 @@ def test_static_scratch_entry_point_matches_the_caller_scratch_one_twice():
         # the property the entry point exists for: the call takes no device memory, neither from torch's pool nor
         # from the driver (the first call on a device only looks an address up)
         torch_before, (free_before, _) = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()
-        got = rsd.rsd_sbs_step_static(rows, W, first_node, sig, gam, 21, step, outs, seq_base=3,
-                                      parent_base=first_node)
+        rsd.rsd_sbs_step_static(rows, W, first_node, sig, gam, 21, step, outs, seq_base=3, parent_base=first_node)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == torch_before
+        assert torch.cuda.memory_allocated() == torch_before   # (no name is rebound in between: nothing is freed either)
+        got = outs
         if done > 0:   # (the very first call on a device may still page the library's image in)
             assert torch.cuda.mem_get_info()[0] >= free_before
         for key in ("token", "parent", "count", "status"):
