@@ -4,7 +4,7 @@
 
 #include "rsd_api_common.h"
 #include "rsd_verify.cuh"
-#include "rsd_walk_resident.cuh"
+#include "rsd_walk_ring.cuh"
 
 using namespace rsd_host;
 
@@ -21,32 +21,20 @@ int sm_count() {
     return cached[dev];
 }
 
-// The walk with the node's rows resident in shared memory, if this call qualifies: returns false when it does not
-// (the caller then takes the streaming kernel), true after a launch or a launch error.
+// The walk fed by the copy engine (rsd_walk_ring.cuh); a launch error stays pending for check_launch().
 template <typename T>
-bool launch_resident_walk(const rsd::VerifyArgs& a, int B, cudaStream_t s) {
-    using namespace rsd::walk_res;
-    if (a.V > kMaxChunks * kChunkElems) return false;
-    ResidentLaunch rl;
-    rl.n_chunks = (a.V + kChunkElems - 1) / kChunkElems;
-    rl.n_tiles = (a.V + kTileElems - 1) / kTileElems;
-    rl.gsum_offset = (size_t)rl.n_chunks * 2 * kChunkElems * sizeof(T);
-    rl.dyn_bytes = rl.gsum_offset + (size_t)rl.n_tiles * 32 * sizeof(float);
-    constexpr size_t kSharedPerBlock = 227 * 1024;   // sm_100: opt-in limit per block, static part included
-    if (rl.dyn_bytes + sizeof(ResSmem) + 256 > kSharedPerBlock) return false;
-    // The attribute belongs to the (function, device) pair and setting it costs tens of microseconds of host time:
-    // raised once per device to the largest size this kernel can use (a failure stays pending for check_launch()).
+void launch_ring_walk(const rsd::VerifyArgs& a, int B, cudaStream_t s) {
+    using namespace rsd::walk_ring;
+    // The attribute belongs to the (function, device) pair and setting it costs host time: once per device.
     static std::atomic<bool> raised[64];
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return true;
+    if (cudaGetDevice(&dev) != cudaSuccess) return;
     if (dev < 0 || dev >= 64 || !raised[dev].load(std::memory_order_acquire)) {
-        if (cudaFuncSetAttribute(verify_tree_resident_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(kSharedPerBlock - sizeof(ResSmem) - 256)) != cudaSuccess)
-            return true;
+        if (cudaFuncSetAttribute(verify_tree_ring_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingBytes) != cudaSuccess)
+            return;
         if (dev >= 0 && dev < 64) raised[dev].store(true, std::memory_order_release);
     }
-    verify_tree_resident_kernel<T><<<B, kThreads, rl.dyn_bytes, s>>>(a, rl);
-    return true;
+    verify_tree_ring_kernel<T><<<B, kThreads, kRingBytes, s>>>(a);
 }
 }  // namespace
 
@@ -106,11 +94,11 @@ int rsd_verify_tree_rule(const rsd_rows* draft, const rsd_rows* target, const rs
     } while (0)
     const bool wide_blocks = B <= sm_count();
     if (rule == RSD_RULE_RRS && final_sampler == RSD_FINAL_INVERSE_CDF) {
-        // rows that fit in shared memory as a pair: the walk that reads each visited row from HBM once and runs
-        // every later pass on chip
-        const bool resident = aligned && (draft->dtype == RSD_F32 ? launch_resident_walk<float>(a, B, s)
-                                                                   : launch_resident_walk<__nv_bfloat16>(a, B, s));
-        if (resident) { /* launched */ }
+        // rows on 16-byte boundaries: the walk whose passes are fed by the copy engine
+        if (aligned) {
+            if (draft->dtype == RSD_F32) launch_ring_walk<float>(a, B, s);
+            else launch_ring_walk<__nv_bfloat16>(a, B, s);
+        }
         else if (wide_blocks) RSD_LAUNCH_WALK(walk_wide, false);
         else RSD_LAUNCH_WALK(walk_narrow, false);
     } else {

@@ -1,0 +1,628 @@
+// Recursive rejection sampling along the draft tree (Eqs. 1-4, Algorithm 1; Section 3.2.2, Algorithm 6): the walk
+// whose passes stream a node's rows through a ring of shared-memory slots filled by the copy engine.
+//
+// One block walks one sequence and reads only the rows of visited nodes.  The chain of residuals is carried in
+// closed form (see rsd_verify.cuh), so every pass is a read-only sweep over the node's target and draft rows: the
+// first pass gives both soft-max normalisers, each rejected child costs one more pass (served by L2, the rows were
+// just read), the last token is drawn from the tile sums of the last pass.
+//
+// A block has eight working warps and one copy warp.  The copy warp asks the copy engine for the rows in chunks of
+// 8 KB per row (cp.async.bulk into a ring of four slots, one mbarrier pair per slot: "full" counts the bytes that
+// landed, "empty" counts the working warps that are done with the slot), so a block keeps up to 64 KB in flight
+// without holding a single register for it, and three blocks share an SM: while one walk waits for a reduction, a
+// decision or its next node's rows, the other two keep the SM's special-function unit and its memory pipe busy.
+// Every wait on a barrier is bounded (about a second); a wait that runs out abandons the walk with RSD_ST_TIMEOUT.
+//
+// Used for rows whose base and strides are multiples of 16 bytes, recursive rejection sampling with the inverse-CDF
+// last draw; everything else takes the register-fed kernels of rsd_verify_walk.inc.
+#pragma once
+#include "rsd_verify.cuh"
+
+namespace rsd {
+namespace walk_ring {
+
+constexpr int kWorkWarps = 8;
+constexpr int kThreads = (kWorkWarps + 1) * 32;   // the last warp feeds the ring
+constexpr int kSlots = 4;                         // power of two
+constexpr int kRowChunkBytes = 8192;              // bytes of one row per slot (a slot holds a target and a draft chunk)
+constexpr int kTileElems = 512;                   // one warp-wide step: 16 elements per lane
+constexpr int kMaxChildren = 64;                  // children of a node whose row values are fetched ahead
+constexpr int kMaxRemovedRing = 64;               // rejected tokens remembered per node (to recognise a repeated sibling)
+constexpr long long kWaitCycles = 1ll << 31;      // about a second: a copy that has not landed by then never will
+constexpr int kRingBytes = kSlots * 2 * kRowChunkBytes;
+
+struct RingSmem {
+    unsigned long long full[kSlots], empty[kSlots];
+    float4 red[2][kWorkWarps];                    // per warp: two sums, two maxima; two copies used in turn
+    double tile_sum[kMaxTiles];
+    int par[kMaxCachedNodes], tok[kMaxCachedNodes];
+    float child_lq[kMaxChildren], child_lp[kMaxChildren];
+    int rem_x[kMaxRemovedRing];
+    int n_removed;
+    int pick;
+    int abort;                                    // a wait ran out: the walk is abandoned and reported
+};
+
+// ---- mbarrier / bulk copy (this GPU's own memory; no cluster, no multicast) -------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// global -> shared, `bytes` a multiple of 16, both addresses 16-byte aligned; completion counts on `bar`
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+// Wait for phase `parity` of `bar`, at most about a second.  A wait that runs out sets *abort and returns: the
+// caller goes on with whatever the slot holds and the walk is abandoned at the next block-wide decision point.
+__device__ __forceinline__ void wait_bar(unsigned long long* bar, uint32_t parity, int* abort) {
+    if (mbar_try_wait(bar, parity)) return;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kWaitCycles) {
+            *abort = 1;
+            return;
+        }
+    }
+}
+
+// A lane's 16 values of a 512-element tile in shared memory: the 16-byte pieces lane, lane + 32, ... of the tile
+// (conflict-free 128-bit loads).  Which elements a lane sums does not matter; the one place that needs token order
+// (the last draw) reads its tile from global memory.
+__device__ __forceinline__ void load_pieces(Packed<__nv_bfloat16>& pk, const unsigned char* tile, int lane) {
+    pk.w[0] = *(const uint4*)(tile + 16 * lane);
+    pk.w[1] = *(const uint4*)(tile + 512 + 16 * lane);
+}
+__device__ __forceinline__ void load_pieces(Packed<float>& pk, const unsigned char* tile, int lane) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) pk.w[i] = *(const uint4*)(tile + 512 * i + 16 * lane);
+}
+
+__device__ __forceinline__ float warp_sum_f32(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max_nan(float v) {   // NaN if any lane holds one
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max_nan(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+
+// unpack a loaded group; CLEAN: NaN -> -inf
+template <typename T, bool CLEAN>
+__device__ __forceinline__ void values16(const Packed<T>& pk, float (&v)[16]) {
+    pk.unpack(v);
+    if (CLEAN) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            if (v[j] != v[j]) v[j] = kNegInf;
+    }
+}
+
+// State of the walk at one node; all threads hold identical copies (the closed-form chain of rsd_verify.cuh).
+struct NodeState {
+    float mq, mp;       // reference values of the exponentials (raw units)
+    float kq, kp;       // log2(e) / temperature
+    double Sq, Sp;      // normalisers relative to the references
+    double A, P, Z;     // chain state
+    float a_hi, a_lo;   // A Sq / Sp as a two-float sum
+    bool with_draft;    // false: a node without children, only its target row is read
+    bool has_nan;       // a NaN was seen in the node's rows: the passes clean their inputs
+};
+
+enum { kPassFirst = 0, kPassTarget = 1, kPassResidual = 2 };
+
+template <typename T>
+struct Ring {
+    RingSmem& sm;
+    unsigned char* slots;      // [kSlots][2][kRowChunkBytes]: target chunk, then draft chunk
+    int V, n_chunks, n_tiles;
+    uint32_t g0;               // chunks asked for before the current pass (all passes of the block)
+    int red_turn;              // which copy of sm.red the next reduction uses
+
+    static constexpr int kElem = (int)sizeof(T);
+    static constexpr int kChunkElems = kRowChunkBytes / kElem;
+    static constexpr int kTPC = kChunkElems / kTileElems;   // tiles per chunk: 8 (2-byte elements) or 4
+
+    // ---- copy warp: all chunks of one pass, in order ------------------------------------------------------------
+    __device__ __forceinline__ void produce(const char* rowq, const char* rowp, bool with_draft) {
+        const int lane = threadIdx.x & 31;
+        const int row_bytes = V * kElem, row_bytes16 = row_bytes & ~15;
+        for (int c = 0; c < n_chunks; ++c) {
+            const uint32_t g = g0 + (uint32_t)c;
+            const int slot = (int)(g & (kSlots - 1));
+            if (g >= (uint32_t)kSlots) wait_bar(&sm.empty[slot], ((g / kSlots) - 1u) & 1u, &sm.abort);
+            const int off = c * kRowChunkBytes;
+            int bytes = row_bytes16 - off;
+            bytes = bytes > kRowChunkBytes ? kRowChunkBytes : (bytes < 0 ? 0 : bytes);
+            unsigned char* dq = slots + (size_t)slot * 2 * kRowChunkBytes;
+            unsigned char* dp = dq + kRowChunkBytes;
+            if (c == n_chunks - 1) {
+                // End of the row: the last V sizeof(T) mod 16 bytes cannot go through the copy engine and are copied
+                // by hand; what follows, up to the end of the tile, is filled with -inf so that the working warps
+                // never have to look at an index.  Published by the barrier arrival below.
+                const int first = row_bytes16 / kElem;                        // first element copied by hand
+                const int tile_end = ((V + kTileElems - 1) / kTileElems) * kTileElems;
+                for (int x = first + lane; x < tile_end; x += 32) {
+                    const int at = (x - c * kChunkElems) * kElem;
+                    if (kElem == 2) {
+                        *(uint16_t*)(dq + at) = x < V ? ((const uint16_t*)rowq)[x] : (uint16_t)0xFF80u;
+                        if (with_draft) *(uint16_t*)(dp + at) = x < V ? ((const uint16_t*)rowp)[x] : (uint16_t)0xFF80u;
+                    } else {
+                        *(uint32_t*)(dq + at) = x < V ? ((const uint32_t*)rowq)[x] : 0xFF800000u;
+                        if (with_draft) *(uint32_t*)(dp + at) = x < V ? ((const uint32_t*)rowp)[x] : 0xFF800000u;
+                    }
+                }
+                __syncwarp();
+            }
+            if (lane == 0) {
+                mbar_expect_tx(&sm.full[slot], with_draft ? 2u * (uint32_t)bytes : (uint32_t)bytes);
+                if (bytes > 0) {
+                    bulk_load(dq, rowq + off, (uint32_t)bytes, &sm.full[slot]);
+                    if (with_draft) bulk_load(dp, rowp + off, (uint32_t)bytes, &sm.full[slot]);
+                }
+            }
+        }
+    }
+
+    // ---- working warps: every chunk of the pass in order; fn(tile, q tile, p tile) for this warp's tile of it -------
+    template <typename F>
+    __device__ __forceinline__ void consume(F&& fn) {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        for (int c = 0; c < n_chunks; ++c) {
+            const uint32_t g = g0 + (uint32_t)c;
+            const int slot = (int)(g & (kSlots - 1));
+            const int i = (warp - c * kTPC) & (kWorkWarps - 1);   // tile of the chunk with (c kTPC + i) mod 8 == warp
+            const int tile = c * kTPC + i;
+            // every warp waits for every chunk, with or without a tile in it: a warp can then never be a whole turn
+            // of the ring ahead of another, so an "empty" phase counts each warp exactly once
+            wait_bar(&sm.full[slot], (g / kSlots) & 1u, &sm.abort);
+            if (i < kTPC && tile < n_tiles) {
+                const unsigned char* q = slots + (size_t)slot * 2 * kRowChunkBytes + (size_t)i * kTileElems * kElem;
+                fn(tile, q, q + kRowChunkBytes);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.empty[slot]);
+        }
+    }
+
+    // Block-wide: sums s0, s1 (returned in double) and maxima m0, m1 (NaN if any thread holds one) of the working
+    // warps' values, identical on all threads; one barrier.
+    __device__ __forceinline__ void reduce(float s0, float s1, float m0, float m1, double& S0, double& S1, float& M0, float& M1) {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        if (warp < kWorkWarps) {
+            s0 = warp_sum_f32(s0);
+            s1 = warp_sum_f32(s1);
+            m0 = warp_max_nan(m0);
+            m1 = warp_max_nan(m1);
+            if (lane == 0) sm.red[red_turn][warp] = make_float4(s0, s1, m0, m1);
+        }
+        __syncthreads();
+        S0 = 0.0;
+        S1 = 0.0;
+        M0 = kNegInf;
+        M1 = kNegInf;
+#pragma unroll
+        for (int w = 0; w < kWorkWarps; ++w) {   // fixed order: the same on every thread
+            const float4 r = sm.red[red_turn][w];
+            S0 += (double)r.x;
+            S1 += (double)r.y;
+            M0 = max_nan(M0, r.z);
+            M1 = max_nan(M1, r.w);
+        }
+        red_turn ^= 1;
+    }
+
+    // One pass over the node's rows.
+    //   kPassFirst     both rows: S0 = sum exp(lt - m_q), S1 = sum exp(ld - m_p), M0 / M1 the rows' maxima
+    //   kPassTarget    target row only: S0 = sum of the weights exp(lt - m_q), M0 its maximum; tile sums stored
+    //   kPassResidual  both rows: S0 = sum of the weights (qh - a ph)+; tile sums stored if STORE_TILES
+    template <int KIND, bool CLEAN, bool STORE_TILES>
+    __device__ __forceinline__ void pass(const char* rowq, const char* rowp, const NodeState& st, double& S0, double& S1,
+                                         float& M0, float& M1) {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        float s0 = 0.0f, s1 = 0.0f, m0 = kNegInf, m1 = kNegInf;
+        if (warp == kWorkWarps) {
+            produce(rowq, rowp, KIND != kPassTarget);
+        } else {
+            const float cq = st.mq * st.kq, cp = st.mp * st.kp;
+            consume([&](int tile, const unsigned char* qt, const unsigned char* pt) {
+                Packed<T> pq;
+                load_pieces(pq, qt, lane);
+                float q[16];
+                if (KIND != kPassResidual && !CLEAN) m0 = max_nan(m0, group_max_nan(pq));   // NaN if the group holds one
+                values16<T, CLEAN>(pq, q);
+                if (KIND != kPassResidual && CLEAN) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) m0 = fmaxf(m0, q[j]);
+                }
+                exp16(q, st.kq, cq, q);
+                float s;
+                if (KIND == kPassTarget) {
+                    s = tree_sum16(q);
+                    s0 += s;
+                } else {
+                    Packed<T> pp;
+                    load_pieces(pp, pt, lane);
+                    float p[16];
+                    if (KIND == kPassFirst && !CLEAN) m1 = max_nan(m1, group_max_nan(pp));
+                    values16<T, CLEAN>(pp, p);
+                    if (KIND == kPassFirst && CLEAN) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) m1 = fmaxf(m1, p[j]);
+                    }
+                    exp16(p, st.kp, cp, p);
+                    if (KIND == kPassFirst) {
+                        s0 += tree_sum16(q);
+                        s1 += tree_sum16(p);
+                        s = 0.0f;
+                    } else {
+                        float w[16];
+                        residual16(q, p, st.a_hi, st.a_lo, w);
+                        s = tree_sum16(w);
+                        s0 += s;
+                    }
+                }
+                if (KIND == kPassTarget || (KIND == kPassResidual && STORE_TILES)) {
+                    const float ts = warp_sum_f32(s);
+                    if (lane == 0) sm.tile_sum[tile] = (double)ts;
+                }
+            });
+        }
+        g0 += (uint32_t)n_chunks;
+        reduce(s0, s1, m0, m1, S0, S1, M0, M1);
+    }
+};
+
+// weights of 16 consecutive tokens of group g, read from global memory (the last draw's exact scan)
+template <typename T>
+__device__ __forceinline__ void group_weights(const char* rowq, const char* rowp, int g, int V, const NodeState& st, bool residual,
+                                              float (&w)[16]) {
+    const float cq = st.mq * st.kq, cp = st.mp * st.kp;
+    float q[16];
+    bool dummy = false;
+    load_clean<T, true>(rowq, g, V, q, dummy);
+    if (residual) {
+        float p[16];
+        load_clean<T, true>(rowp, g, V, p, dummy);
+        exp16(q, st.kq, cq, q);
+        exp16(p, st.kp, cp, p);
+        residual16(q, p, st.a_hi, st.a_lo, w);
+    } else {
+        exp16(q, st.kq, cq, w);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const VerifyArgs a) {
+    extern __shared__ __align__(128) unsigned char ring_mem[];
+    __shared__ RingSmem sm;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int32_t* par = a.parent + (a.shared_topology ? 0 : (int64_t)b * a.num_nodes);
+    const int32_t* tok = a.token + (int64_t)b * a.num_nodes;
+    const RngKey key = {a.seed_lo, a.seed_hi, a.step, a.seq_base + (uint32_t)b};
+    constexpr int kChunkElems = Ring<T>::kChunkElems;
+
+    Ring<T> ring = {sm, ring_mem, a.V, (a.V + kChunkElems - 1) / kChunkElems, (a.V + kTileElems - 1) / kTileElems, 0u, 0};
+    if (tid == 0) {
+        for (int s = 0; s < kSlots; ++s) {
+            mbar_init(&sm.full[s], 1);
+            mbar_init(&sm.empty[s], kWorkWarps);
+        }
+        sm.abort = 0;
+        sm.n_removed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i < a.L; i += kThreads) {
+        a.accepted_node[(int64_t)b * a.L + i] = -1;
+        a.accepted_token[(int64_t)b * a.L + i] = -1;
+    }
+    if (a.dbg_theta)
+        for (int n = tid; n < a.num_nodes; n += kThreads) a.dbg_theta[(int64_t)b * a.num_nodes + n] = __int_as_float(0x7FC00000);
+    const bool cached = a.num_nodes <= kMaxCachedNodes;
+    if (cached)
+        for (int n = tid; n < a.num_nodes; n += kThreads) { sm.par[n] = par[n]; sm.tok[n] = tok[n]; }
+    __syncthreads();
+
+    // smallest node c > after with parent cur_node and a token in [0, V), or -1; every warp searches by itself (the
+    // shared copy of the tree, or global memory for trees too large for it)
+    auto find_child = [&](int cur_node, int after) -> int {
+        for (int c0 = after + 1; c0 < a.num_nodes; c0 += 32) {
+            const int cc = c0 + lane;
+            bool ok = false;
+            if (cc < a.num_nodes) {
+                const int p = cached ? sm.par[cc] : par[cc];
+                const int t = cached ? sm.tok[cc] : tok[cc];
+                ok = p == cur_node && t >= 0 && t < a.V;
+            }
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, ok);
+            if (m) return c0 + __ffs(m) - 1;
+        }
+        return -1;
+    };
+
+    NodeState st;
+    st.kq = kLog2e * a.target.inv_temp;
+    st.kp = kLog2e * a.draft.inv_temp;
+    int status = 0, cur = 0, len = 0, reason = 0, last = -1;
+    bool tiles_valid = false;   // sm.tile_sum holds the tile sums of the distribution the last token is drawn from
+    const char* rowq = nullptr;
+    const char* rowp = nullptr;
+    for (;;) {
+        int c = find_child(cur, 0);
+        st.with_draft = !(c < 0 || len >= a.L);
+        rowq = row_ptr<T>(a.target, b, cur);
+        rowp = st.with_draft ? row_ptr<T>(a.draft, b, cur) : rowq;
+        st.A = 0.0; st.P = 0.0; st.Z = 1.0; st.a_hi = st.a_lo = 0.0f; st.has_nan = false;
+        st.mq = 0.0f; st.mp = 0.0f; st.Sp = 1.0;
+        tiles_valid = false;
+        // The copy warp fetches, ahead of time, the row values of the node's first children (the thresholds need
+        // them right after the first pass); the loads are in flight while it feeds the ring.
+        float ahead_q[kMaxChildren / 32], ahead_p[kMaxChildren / 32];
+        if (warp == kWorkWarps && st.with_draft) {
+            int cc = c, j = 0;
+#pragma unroll
+            for (int r = 0; r < kMaxChildren / 32; ++r) { ahead_q[r] = 0.0f; ahead_p[r] = 0.0f; }
+            while (cc >= 0 && j < kMaxChildren) {
+                if ((j & 31) == lane) {
+                    const int x = cached ? sm.tok[cc] : tok[cc];
+#pragma unroll
+                    for (int r = 0; r < kMaxChildren / 32; ++r)
+                        if (r == (j >> 5)) { ahead_q[r] = RowIO<T>::scalar(rowq, x); ahead_p[r] = RowIO<T>::scalar(rowp, x); }
+                }
+                ++j;
+                cc = find_child(cur, cc);
+            }
+        }
+        // First pass.  The exponentials are taken relative to a reference: 0 to begin with, the row maximum when that
+        // turns out to be too far from 0 (rare: logits beyond +-60 / temperature); a NaN in the rows switches the
+        // node's passes to their cleaning form.
+        for (int attempt = 0; attempt < 4; ++attempt) {
+            double S0, S1;
+            float M0, M1;
+            if (st.with_draft) {
+                if (st.has_nan) ring.template pass<kPassFirst, true, false>(rowq, rowp, st, S0, S1, M0, M1);
+                else ring.template pass<kPassFirst, false, false>(rowq, rowp, st, S0, S1, M0, M1);
+            } else {
+                if (st.has_nan) ring.template pass<kPassTarget, true, true>(rowq, rowp, st, S0, S1, M0, M1);
+                else ring.template pass<kPassTarget, false, true>(rowq, rowp, st, S0, S1, M0, M1);
+                M1 = 0.0f;
+                S1 = 1.0;
+            }
+            if (attempt == 0 && warp == kWorkWarps && st.with_draft) {
+#pragma unroll
+                for (int r = 0; r < kMaxChildren / 32; ++r) { sm.child_lq[r * 32 + lane] = ahead_q[r]; sm.child_lp[r * 32 + lane] = ahead_p[r]; }
+            }
+            if (sm.abort) break;
+            if (!st.has_nan && (M0 != M0 || M1 != M1)) {   // a NaN logit: counts as -inf, reported
+                st.has_nan = true;
+                status |= 1;                                // RSD_ST_NAN_INPUT
+                continue;
+            }
+            st.Sq = S0;
+            st.Sp = S1;
+            const bool redo_q = M0 > kNegInf && fabsf((M0 - st.mq) * st.kq) > kRefSlack * kLog2e;
+            const bool redo_p = st.with_draft && M1 > kNegInf && fabsf((M1 - st.mp) * st.kp) > kRefSlack * kLog2e;
+            if (!redo_q && !redo_p) { tiles_valid = !st.with_draft; break; }
+            if (redo_q) st.mq = M0;
+            if (redo_p) st.mp = M1;
+        }
+        if (tid == 0) sm.n_removed = 0;
+        __syncthreads();   // the children's values are in shared memory
+        if (sm.abort) break;
+        if (!st.with_draft) {
+            reason = (len >= a.L) ? 2 : 1;  // RSD_STOP_LEAF : RSD_STOP_NO_CHILDREN
+            break;
+        }
+        int accepted = -1, j = 0;
+        while (c >= 0) {
+            const int x = cached ? sm.tok[c] : tok[c];
+            float lq, lp;
+            if (j < kMaxChildren) { lq = sm.child_lq[j]; lp = sm.child_lp[j]; }
+            else { lq = RowIO<T>::scalar(rowq, x); lp = RowIO<T>::scalar(rowp, x); }
+            const float qh = (lq == lq) ? ex2_approx(fmaf(lq, st.kq, -st.mq * st.kq)) : 0.0f;
+            const float ph = (lp == lp) ? ex2_approx(fmaf(lp, st.kp, -st.mp * st.kp)) : 0.0f;
+            const double qx = (double)qh / st.Sq, px_row = (double)ph / st.Sp;
+            bool repeated = false;   // a sibling with the same token was rejected before: its draft mass is gone (Eq. 1)
+            for (int i = 0; i < sm.n_removed; ++i) repeated |= sm.rem_x[i] == x;
+            const double px = repeated ? 0.0 : px_row;
+            const double r = fmax(qx - st.A * px_row, 0.0);
+            double theta;
+            if (px > 0.0) theta = fmin(1.0, r * (1.0 - st.P) / (st.Z * px));
+            else { status |= 8; theta = r > 0.0 ? 1.0 : 0.0; }   // RSD_ST_ZERO_DRAFT_PROB
+            const uint4 rw = rng_draw(key, (uint32_t)cur, kTagAccept, (uint32_t)j);
+            const double U = (double)(rw.x >> 8) * (1.0 / 16777216.0);
+            if (a.dbg_theta && tid == 0) a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)theta;
+            if (U < theta) { accepted = c; break; }
+            ++j;
+            const int next = find_child(cur, c);
+            // Eqs. 1-2 in closed form: A_{j+1} = A_j + Z_j / (1 - P_j), Z_{j+1} = sum (q - A_{j+1} p)+
+            const double A_old = st.A;
+            st.A = st.A + st.Z / (1.0 - st.P);
+            {
+                const double aa = st.A * st.Sq / st.Sp;
+                st.a_hi = (float)aa;
+                st.a_lo = (float)(aa - (double)st.a_hi);
+            }
+            double zhat, none;
+            float f0, f1;
+            const bool maybe_last = next < 0;   // no sibling left: the last token is drawn from this residual
+            if (st.has_nan) {
+                if (maybe_last) ring.template pass<kPassResidual, true, true>(rowq, rowp, st, zhat, none, f0, f1);
+                else ring.template pass<kPassResidual, true, false>(rowq, rowp, st, zhat, none, f0, f1);
+            } else {
+                if (maybe_last) ring.template pass<kPassResidual, false, true>(rowq, rowp, st, zhat, none, f0, f1);
+                else ring.template pass<kPassResidual, false, false>(rowq, rowp, st, zhat, none, f0, f1);
+            }
+            if (sm.abort) break;
+            const double Z_new = zhat / st.Sq;
+            if (Z_new > 0.0 && Z_new < 1.7e308) {
+                st.Z = Z_new;
+                tiles_valid = maybe_last;
+            } else {
+                status |= 4;   // RSD_ST_ZERO_RESIDUAL: keep the previous residual
+                st.A = A_old;
+                const double aa = st.A * st.Sq / st.Sp;
+                st.a_hi = (float)aa;
+                st.a_lo = (float)(aa - (double)st.a_hi);
+                tiles_valid = false;
+            }
+            st.P += px;
+            if (tid == 0 && !repeated && sm.n_removed < kMaxRemovedRing) sm.rem_x[sm.n_removed++] = x;
+            __syncthreads();
+            if (!(1.0 - st.P > 0.0)) { status |= 16; tiles_valid = tiles_valid && maybe_last; break; }   // RSD_ST_DRAFT_EXHAUSTED
+            c = next;
+        }
+        if (sm.abort) break;
+        if (accepted < 0) {   // RSD_STOP_ALL_REJECTED: the last token comes from the residual in force
+            reason = 0;
+            break;
+        }
+        if (tid == 0) {
+            a.accepted_node[(int64_t)b * a.L + len] = accepted;
+            a.accepted_token[(int64_t)b * a.L + len] = cached ? sm.tok[accepted] : tok[accepted];
+        }
+        ++len;
+        cur = accepted;
+    }
+
+    if (!sm.abort) {
+        const bool residual = st.with_draft && st.A != 0.0;
+        if (!tiles_valid) {   // rare: the last pass was not kept, or it did not store its tile sums
+            double s, none;
+            float f0, f1;
+            if (residual) {
+                if (st.has_nan) ring.template pass<kPassResidual, true, true>(rowq, rowp, st, s, none, f0, f1);
+                else ring.template pass<kPassResidual, false, true>(rowq, rowp, st, s, none, f0, f1);
+            } else {
+                if (st.has_nan) ring.template pass<kPassTarget, true, true>(rowq, rowq, st, s, none, f0, f1);
+                else ring.template pass<kPassTarget, false, true>(rowq, rowq, st, s, none, f0, f1);
+            }
+        }
+    }
+    if (!sm.abort) {
+        // Inverse CDF over the tile sums of the last pass: the smallest y whose running sum exceeds u * total; if
+        // rounding leaves none, the largest y with positive weight; -1 if there is no weight at all.
+        const bool residual = st.with_draft && st.A != 0.0;
+        const uint4 rw = rng_draw(key, (uint32_t)cur, kTagResample, 0u);
+        const double u = ((double)rw.x + 0.5) * (1.0 / 4294967296.0);
+        __syncthreads();   // every tile sum is in place
+        if (warp == 0) {
+            const int n_tiles = ring.n_tiles;
+            // lanes take consecutive runs of tiles; running sums in tile order
+            const int per = (n_tiles + 31) / 32;
+            const int t_lo = lane * per, t_hi = min(n_tiles, t_lo + per);
+            double mine = 0.0;
+            for (int t = t_lo; t < t_hi; ++t) mine += sm.tile_sum[t];
+            double incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            const double total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            int y = -1;
+            if (total > 0.0 && total < 1.7e308) {   // (uniform over the warp)
+                const double target = u * total;
+                // the tile that holds the crossing, or failing that the last tile with weight
+                const unsigned crossing = __ballot_sync(0xFFFFFFFFu, incl > target);
+                const unsigned positive = __ballot_sync(0xFFFFFFFFu, mine > 0.0);
+                const bool take_last = crossing == 0u;
+                const int src = take_last ? 31 - __clz(positive) : __ffs(crossing) - 1;
+                int tile = -1;
+                double before = 0.0;
+                if (lane == src) {
+                    double cum = incl - mine;
+                    for (int t = t_lo; t < t_hi; ++t) {
+                        const double s = sm.tile_sum[t];
+                        if (take_last) { if (s > 0.0) { tile = t; before = cum; } }
+                        else if (cum + s > target) { tile = t; before = cum; break; }
+                        cum += s;
+                    }
+                    if (tile < 0) {   // rounding: the lane's total crossed, no tile did: its last tile with weight
+                        cum = incl - mine;
+                        for (int t = t_lo; t < t_hi; ++t) {
+                            const double s = sm.tile_sum[t];
+                            if (s > 0.0) { tile = t; before = cum; }
+                            cum += s;
+                        }
+                    }
+                }
+                tile = __shfl_sync(0xFFFFFFFFu, tile, src);
+                before = __shfl_sync(0xFFFFFFFFu, before, src);
+                // the tile's weights once more, in token order: lane owns tokens 16 lane .. 16 lane + 15 of the tile
+                float w[16];
+                const int g = tile * 32 + lane;
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) w[jj] = 0.0f;
+                if (tile >= 0 && g * 16 < a.V) group_weights<T>(rowq, rowp, g, a.V, st, residual, w);
+                double gs = 0.0;
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) gs += (double)w[jj];
+                double gincl = gs;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const double t = __shfl_up_sync(0xFFFFFFFFu, gincl, o);
+                    if (lane >= o) gincl += t;
+                }
+                const unsigned cross2 = __ballot_sync(0xFFFFFFFFu, !take_last && (before + gincl > target));
+                const unsigned pos2 = __ballot_sync(0xFFFFFFFFu, gs > 0.0);
+                const bool last_mode = cross2 == 0u;
+                const int src2 = last_mode ? (pos2 ? 31 - __clz(pos2) : 0) : __ffs(cross2) - 1;
+                if (lane == src2) {
+                    int last_pos = -1;
+                    double cacc = before + (gincl - gs);
+#pragma unroll
+                    for (int jj = 0; jj < 16; ++jj) {
+                        cacc += (double)w[jj];
+                        if (w[jj] > 0.0f) last_pos = g * 16 + jj;
+                        if (!last_mode && y < 0 && cacc > target) y = g * 16 + jj;
+                    }
+                    if (y < 0) y = last_pos;
+                }
+                y = __shfl_sync(0xFFFFFFFFu, y, src2);
+            }
+            if (lane == 0) sm.pick = y;
+        }
+        __syncthreads();
+        last = sm.pick;
+    } else {
+        // A wait ran out.  Before the block gives its shared memory back, wait once more (bounded) for the copies it
+        // may still have in flight: the last kSlots chunks it asked for.
+        if (warp == kWorkWarps) {
+            for (uint32_t g = ring.g0 > (uint32_t)kSlots ? ring.g0 - kSlots : 0u; g < ring.g0; ++g)
+                wait_bar(&sm.full[g & (kSlots - 1)], (g / kSlots) & 1u, &sm.abort);
+        }
+        status |= 32;   // RSD_ST_TIMEOUT
+        __syncthreads();
+    }
+    if (tid == 0) {
+        a.accepted_len[b] = len;
+        a.last_token[b] = last;
+        a.stop_reason[b] = reason;
+        a.status[b] = status;
+    }
+}
+
+}  // namespace walk_ring
+}  // namespace rsd
