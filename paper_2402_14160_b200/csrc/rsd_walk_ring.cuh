@@ -6,12 +6,15 @@
 // first pass gives both soft-max normalisers, each rejected child costs one more pass (served by L2, the rows were
 // just read), the last token is drawn from the tile sums of the last pass.
 //
-// A block has eight working warps and one copy warp.  The copy warp asks the copy engine for the rows in chunks of
-// 8 KB per row (cp.async.bulk into a ring of four slots, one mbarrier pair per slot: "full" counts the bytes that
-// landed, "empty" counts the working warps that are done with the slot), so a block keeps up to 64 KB in flight
-// without holding a single register for it, and three blocks share an SM: while one walk waits for a reduction, a
-// decision or its next node's rows, the other two keep the SM's special-function unit and its memory pipe busy.
-// Every wait on a barrier is bounded (about a second); a wait that runs out abandons the walk with RSD_ST_TIMEOUT.
+// A block has eight working warps and one control warp.  The control warp alone walks the tree: it takes every
+// decision (thresholds, acceptance tests, the chain's scalars, the last draw), tells the working warps which pass to
+// run next through a command word in shared memory, and asks the copy engine for the rows in chunks of 8 KB per row
+// (cp.async.bulk into a ring of four slots, one mbarrier pair per slot: "full" counts the bytes that landed, "empty"
+// counts the working warps that are done with the slot).  A block thus keeps up to 64 KB in flight without holding
+// a register for it, the scalar part of the walk is executed once instead of by every warp, and three blocks share an
+// SM: while one walk waits for a decision or for its next node's rows, the other two keep the SM's special-function
+// unit and its memory pipe busy.
+// Every wait on an mbarrier is bounded (about a second); a wait that runs out abandons the walk with RSD_ST_TIMEOUT.
 //
 // Used for rows whose base and strides are multiples of 16 bytes, recursive rejection sampling with the inverse-CDF
 // last draw; everything else takes the register-fed kernels of rsd_verify_walk.inc.
@@ -28,18 +31,27 @@ constexpr int kRowChunkBytes = 8192;              // bytes of one row per slot (
 constexpr int kTileElems = 512;                   // one warp-wide step: 16 elements per lane
 constexpr int kMaxChildren = 64;                  // children of a node whose row values are fetched ahead
 constexpr int kMaxRemovedRing = 64;               // rejected tokens remembered per node (to recognise a repeated sibling)
+constexpr float kSumFloor = 8.673617379884035e-19f;   // 2^-60: a normaliser below this has lost its small terms to underflow
 constexpr long long kWaitCycles = 1ll << 31;      // about a second: a copy that has not landed by then never will
 constexpr int kRingBytes = kSlots * 2 * kRowChunkBytes;
 
+// What the working warps do next (written by the control warp, read after a block barrier).
+struct PassCmd {
+    int kind;            // kPassEnd, or a pass kind below
+    int clean;           // 1: NaN inputs are turned into -inf (a NaN was seen in the node's rows)
+    int store_tiles;     // 1: the pass leaves the sum of every 512-element tile in tile_sum
+    float kq, kp;        // log2(e) / temperature of the target and draft rows
+    float cq, cp;        // reference * k: exponentials are 2^(value * k - c)
+    float a_hi, a_lo;    // coefficient of the residual pass, as a two-float sum
+};
+
 struct RingSmem {
     unsigned long long full[kSlots], empty[kSlots];
-    float4 red[2][kWorkWarps];                    // per warp: two sums, two maxima; two copies used in turn
+    PassCmd cmd;
+    float4 red[kWorkWarps];                       // per working warp: two sums, two maxima of its last pass
     double tile_sum[kMaxTiles];
     int par[kMaxCachedNodes], tok[kMaxCachedNodes];
-    float child_lq[kMaxChildren], child_lp[kMaxChildren];
-    int rem_x[kMaxRemovedRing];
-    int n_removed;
-    int pick;
+    int nan_seen;                                 // a cleaning pass met a NaN
     int abort;                                    // a wait ran out: the walk is abandoned and reported
 };
 
@@ -119,7 +131,9 @@ __device__ __forceinline__ void values16(const Packed<T>& pk, float (&v)[16]) {
     }
 }
 
-// State of the walk at one node; all threads hold identical copies (the closed-form chain of rsd_verify.cuh).
+enum { kPassEnd = -1, kPassFirst = 0, kPassTarget = 1, kPassResidual = 2 };
+
+// State of the walk at one node (control warp only): the closed-form chain of rsd_verify.cuh.
 struct NodeState {
     float mq, mp;       // reference values of the exponentials (raw units)
     float kq, kp;       // log2(e) / temperature
@@ -130,25 +144,22 @@ struct NodeState {
     bool has_nan;       // a NaN was seen in the node's rows: the passes clean their inputs
 };
 
-enum { kPassFirst = 0, kPassTarget = 1, kPassResidual = 2 };
-
 template <typename T>
 struct Ring {
     RingSmem& sm;
     unsigned char* slots;      // [kSlots][2][kRowChunkBytes]: target chunk, then draft chunk
     int V, n_chunks, n_tiles;
     uint32_t g0;               // chunks asked for before the current pass (all passes of the block)
-    int red_turn;              // which copy of sm.red the next reduction uses
 
     static constexpr int kElem = (int)sizeof(T);
     static constexpr int kChunkElems = kRowChunkBytes / kElem;
     static constexpr int kTPC = kChunkElems / kTileElems;   // tiles per chunk: 8 (2-byte elements) or 4
 
-    // ---- copy warp: all chunks of one pass, in order ------------------------------------------------------------
-    __device__ __forceinline__ void produce(const char* rowq, const char* rowp, bool with_draft) {
+    // ---- control warp: ask for chunks [c_begin, c_end) of the current pass, in order ----------------------------------
+    __device__ __forceinline__ void produce(const char* rowq, const char* rowp, bool with_draft, int c_begin, int c_end) {
         const int lane = threadIdx.x & 31;
         const int row_bytes = V * kElem, row_bytes16 = row_bytes & ~15;
-        for (int c = 0; c < n_chunks; ++c) {
+        for (int c = c_begin; c < c_end; ++c) {
             const uint32_t g = g0 + (uint32_t)c;
             const int slot = (int)(g & (kSlots - 1));
             if (g >= (uint32_t)kSlots) wait_bar(&sm.empty[slot], ((g / kSlots) - 1u) & 1u, &sm.abort);
@@ -206,91 +217,60 @@ struct Ring {
         }
     }
 
-    // Block-wide: sums s0, s1 (returned in double) and maxima m0, m1 (NaN if any thread holds one) of the working
-    // warps' values, identical on all threads; one barrier.
-    __device__ __forceinline__ void reduce(float s0, float s1, float m0, float m1, double& S0, double& S1, float& M0, float& M1) {
-        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-        if (warp < kWorkWarps) {
-            s0 = warp_sum_f32(s0);
-            s1 = warp_sum_f32(s1);
-            m0 = warp_max_nan(m0);
-            m1 = warp_max_nan(m1);
-            if (lane == 0) sm.red[red_turn][warp] = make_float4(s0, s1, m0, m1);
-        }
-        __syncthreads();
-        S0 = 0.0;
-        S1 = 0.0;
-        M0 = kNegInf;
-        M1 = kNegInf;
-#pragma unroll
-        for (int w = 0; w < kWorkWarps; ++w) {   // fixed order: the same on every thread
-            const float4 r = sm.red[red_turn][w];
-            S0 += (double)r.x;
-            S1 += (double)r.y;
-            M0 = max_nan(M0, r.z);
-            M1 = max_nan(M1, r.w);
-        }
-        red_turn ^= 1;
-    }
-
-    // One pass over the node's rows.
-    //   kPassFirst     both rows: S0 = sum exp(lt - m_q), S1 = sum exp(ld - m_p), M0 / M1 the rows' maxima
-    //   kPassTarget    target row only: S0 = sum of the weights exp(lt - m_q), M0 its maximum; tile sums stored
-    //   kPassResidual  both rows: S0 = sum of the weights (qh - a ph)+; tile sums stored if STORE_TILES
+    // One pass of a working warp over the node's rows; leaves the warp's sums and maxima in sm.red[warp].
+    //   kPassFirst     both rows: sums of exp(lt k_q - c_q) and exp(ld k_p - c_p)
+    //   kPassTarget    target row only: sum of the weights exp(lt k_q - c_q)
+    //   kPassResidual  both rows: sum of the weights (qh - a ph)+
+    // CLEAN passes turn NaN into -inf (reported through sm.nan_seen) and also return the rows' maxima; the plain ones
+    // carry no code for either.  STORE_TILES: the sum of every tile goes to sm.tile_sum.
     template <int KIND, bool CLEAN, bool STORE_TILES>
-    __device__ __forceinline__ void pass(const char* rowq, const char* rowp, const NodeState& st, double& S0, double& S1,
-                                         float& M0, float& M1) {
+    __device__ __forceinline__ void work(const PassCmd& cmd) {
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
         float s0 = 0.0f, s1 = 0.0f, m0 = kNegInf, m1 = kNegInf;
-        if (warp == kWorkWarps) {
-            produce(rowq, rowp, KIND != kPassTarget);
-        } else {
-            const float cq = st.mq * st.kq, cp = st.mp * st.kp;
-            consume([&](int tile, const unsigned char* qt, const unsigned char* pt) {
-                Packed<T> pq;
-                load_pieces(pq, qt, lane);
-                float q[16];
-                if (KIND != kPassResidual && !CLEAN) m0 = max_nan(m0, group_max_nan(pq));   // NaN if the group holds one
-                values16<T, CLEAN>(pq, q);
-                if (KIND != kPassResidual && CLEAN) {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) m0 = fmaxf(m0, q[j]);
-                }
-                exp16(q, st.kq, cq, q);
-                float s;
-                if (KIND == kPassTarget) {
-                    s = tree_sum16(q);
-                    s0 += s;
+        bool saw_nan = false;
+        consume([&](int tile, const unsigned char* qt, const unsigned char* pt) {
+            Packed<T> pq;
+            load_pieces(pq, qt, lane);
+            float q[16];
+            if (CLEAN) m0 = fmaxf(m0, clean<T>(pq, q, saw_nan));
+            else pq.unpack(q);
+            exp16(q, cmd.kq, cmd.cq, q);
+            float s;
+            if (KIND == kPassTarget) {
+                s = tree_sum16(q);
+                s0 += s;
+            } else {
+                Packed<T> pp;
+                load_pieces(pp, pt, lane);
+                float p[16];
+                if (CLEAN) m1 = fmaxf(m1, clean<T>(pp, p, saw_nan));
+                else pp.unpack(p);
+                exp16(p, cmd.kp, cmd.cp, p);
+                if (KIND == kPassFirst) {
+                    s0 += tree_sum16(q);
+                    s1 += tree_sum16(p);
+                    s = 0.0f;
                 } else {
-                    Packed<T> pp;
-                    load_pieces(pp, pt, lane);
-                    float p[16];
-                    if (KIND == kPassFirst && !CLEAN) m1 = max_nan(m1, group_max_nan(pp));
-                    values16<T, CLEAN>(pp, p);
-                    if (KIND == kPassFirst && CLEAN) {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) m1 = fmaxf(m1, p[j]);
-                    }
-                    exp16(p, st.kp, cp, p);
-                    if (KIND == kPassFirst) {
-                        s0 += tree_sum16(q);
-                        s1 += tree_sum16(p);
-                        s = 0.0f;
-                    } else {
-                        float w[16];
-                        residual16(q, p, st.a_hi, st.a_lo, w);
-                        s = tree_sum16(w);
-                        s0 += s;
-                    }
+                    float w[16];
+                    residual16(q, p, cmd.a_hi, cmd.a_lo, w);
+                    s = tree_sum16(w);
+                    s0 += s;
                 }
-                if (KIND == kPassTarget || (KIND == kPassResidual && STORE_TILES)) {
-                    const float ts = warp_sum_f32(s);
-                    if (lane == 0) sm.tile_sum[tile] = (double)ts;
-                }
-            });
-        }
+            }
+            if (STORE_TILES) {
+                const float ts = warp_sum_f32(s);
+                if (lane == 0) sm.tile_sum[tile] = (double)ts;
+            }
+        });
         g0 += (uint32_t)n_chunks;
-        reduce(s0, s1, m0, m1, S0, S1, M0, M1);
+        s0 = warp_sum_f32(s0);
+        s1 = warp_sum_f32(s1);
+        if (CLEAN) {
+            m0 = warp_max(m0);
+            m1 = warp_max(m1);
+            if (saw_nan) sm.nan_seen = 1;
+        }
+        if (lane == 0) sm.red[warp] = make_float4(s0, s1, m0, m1);
     }
 };
 
@@ -320,17 +300,16 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int32_t* par = a.parent + (a.shared_topology ? 0 : (int64_t)b * a.num_nodes);
     const int32_t* tok = a.token + (int64_t)b * a.num_nodes;
-    const RngKey key = {a.seed_lo, a.seed_hi, a.step, a.seq_base + (uint32_t)b};
     constexpr int kChunkElems = Ring<T>::kChunkElems;
 
-    Ring<T> ring = {sm, ring_mem, a.V, (a.V + kChunkElems - 1) / kChunkElems, (a.V + kTileElems - 1) / kTileElems, 0u, 0};
+    Ring<T> ring = {sm, ring_mem, a.V, (a.V + kChunkElems - 1) / kChunkElems, (a.V + kTileElems - 1) / kTileElems, 0u};
     if (tid == 0) {
         for (int s = 0; s < kSlots; ++s) {
             mbar_init(&sm.full[s], 1);
             mbar_init(&sm.empty[s], kWorkWarps);
         }
         sm.abort = 0;
-        sm.n_removed = 0;
+        sm.nan_seen = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = tid; i < a.L; i += kThreads) {
@@ -344,8 +323,34 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
         for (int n = tid; n < a.num_nodes; n += kThreads) { sm.par[n] = par[n]; sm.tok[n] = tok[n]; }
     __syncthreads();
 
-    // smallest node c > after with parent cur_node and a token in [0, V), or -1; every warp searches by itself (the
-    // shared copy of the tree, or global memory for trees too large for it)
+    // ================================ working warps: run the passes they are told to ===================================
+    if (warp < kWorkWarps) {
+        for (;;) {
+            __syncthreads();   // the command is in place
+            const PassCmd cmd = sm.cmd;
+            if (cmd.kind == kPassEnd) return;
+            if (cmd.kind == kPassFirst) {
+                if (cmd.clean) ring.template work<kPassFirst, true, false>(cmd);
+                else ring.template work<kPassFirst, false, false>(cmd);
+            } else if (cmd.kind == kPassTarget) {
+                if (cmd.clean) ring.template work<kPassTarget, true, true>(cmd);
+                else ring.template work<kPassTarget, false, true>(cmd);
+            } else {
+                if (cmd.clean) {
+                    if (cmd.store_tiles) ring.template work<kPassResidual, true, true>(cmd);
+                    else ring.template work<kPassResidual, true, false>(cmd);
+                } else {
+                    if (cmd.store_tiles) ring.template work<kPassResidual, false, true>(cmd);
+                    else ring.template work<kPassResidual, false, false>(cmd);
+                }
+            }
+            __syncthreads();   // the warps' sums are in place
+        }
+    }
+
+    // ================================ control warp: the walk itself =======================================================
+    const RngKey key = {a.seed_lo, a.seed_hi, a.step, a.seq_base + (uint32_t)b};
+    // smallest node c > after with parent cur_node and a token in [0, V), or -1
     auto find_child = [&](int cur_node, int after) -> int {
         for (int c0 = after + 1; c0 < a.num_nodes; c0 += 32) {
             const int cc = c0 + lane;
@@ -364,10 +369,40 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
     NodeState st;
     st.kq = kLog2e * a.target.inv_temp;
     st.kp = kLog2e * a.draft.inv_temp;
-    int status = 0, cur = 0, len = 0, reason = 0, last = -1;
-    bool tiles_valid = false;   // sm.tile_sum holds the tile sums of the distribution the last token is drawn from
     const char* rowq = nullptr;
     const char* rowp = nullptr;
+    // One pass: publish the command, ask for the rows, collect the working warps' results.  The first chunks are
+    // asked for before the command is published: their slots are free (every working warp has released every slot
+    // of the pass before), and the copies travel while the working warps wake up.
+    auto run_pass = [&](int kind, bool store_tiles, double& S0, double& S1, float& M0, float& M1) {
+        const bool with_draft = kind != kPassTarget;
+        if (lane == 0) {
+            PassCmd cmd;
+            cmd.kind = kind; cmd.clean = st.has_nan ? 1 : 0; cmd.store_tiles = store_tiles ? 1 : 0;
+            cmd.kq = st.kq; cmd.kp = st.kp; cmd.cq = st.mq * st.kq; cmd.cp = st.mp * st.kp;
+            cmd.a_hi = st.a_hi; cmd.a_lo = st.a_lo;
+            sm.cmd = cmd;
+        }
+        const int early = ring.n_chunks < kSlots ? ring.n_chunks : kSlots;
+        ring.produce(rowq, rowp, with_draft, 0, early);
+        __syncthreads();   // the command is in place
+        ring.produce(rowq, rowp, with_draft, early, ring.n_chunks);
+        ring.g0 += (uint32_t)ring.n_chunks;
+        __syncthreads();   // the warps' sums are in place
+        S0 = 0.0; S1 = 0.0; M0 = kNegInf; M1 = kNegInf;
+#pragma unroll
+        for (int w = 0; w < kWorkWarps; ++w) {   // fixed order
+            const float4 r = sm.red[w];
+            S0 += (double)r.x;
+            S1 += (double)r.y;
+            M0 = fmaxf(M0, r.z);
+            M1 = fmaxf(M1, r.w);
+        }
+    };
+
+    int status = 0, cur = 0, len = 0, reason = 0, last = -1;
+    bool tiles_valid = false;   // sm.tile_sum holds the tile sums of the distribution the last token is drawn from
+    bool aborted = false;
     for (;;) {
         int c = find_child(cur, 0);
         st.with_draft = !(c < 0 || len >= a.L);
@@ -376,75 +411,80 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
         st.A = 0.0; st.P = 0.0; st.Z = 1.0; st.a_hi = st.a_lo = 0.0f; st.has_nan = false;
         st.mq = 0.0f; st.mp = 0.0f; st.Sp = 1.0;
         tiles_valid = false;
-        // The copy warp fetches, ahead of time, the row values of the node's first children (the thresholds need
-        // them right after the first pass); the loads are in flight while it feeds the ring.
-        float ahead_q[kMaxChildren / 32], ahead_p[kMaxChildren / 32];
-        if (warp == kWorkWarps && st.with_draft) {
-            int cc = c, j = 0;
-#pragma unroll
-            for (int r = 0; r < kMaxChildren / 32; ++r) { ahead_q[r] = 0.0f; ahead_p[r] = 0.0f; }
-            while (cc >= 0 && j < kMaxChildren) {
-                if ((j & 31) == lane) {
-                    const int x = cached ? sm.tok[cc] : tok[cc];
-#pragma unroll
-                    for (int r = 0; r < kMaxChildren / 32; ++r)
-                        if (r == (j >> 5)) { ahead_q[r] = RowIO<T>::scalar(rowq, x); ahead_p[r] = RowIO<T>::scalar(rowp, x); }
+        // The row values of the node's first 32 children (the thresholds need them right after the first pass): lane j
+        // fetches those of child j; the loads are in flight while the rows stream.
+        int child_node = -1, child_x = -1;
+        float child_lq = 0.0f, child_lp = 0.0f;
+        if (st.with_draft) {
+            int cc = c;
+            for (int j = 0; j < 32 && cc >= 0; ++j) {
+                if (j == lane) {
+                    child_node = cc;
+                    child_x = cached ? sm.tok[cc] : tok[cc];
+                    child_lq = RowIO<T>::scalar(rowq, child_x);
+                    child_lp = RowIO<T>::scalar(rowp, child_x);
                 }
-                ++j;
                 cc = find_child(cur, cc);
             }
         }
-        // First pass.  The exponentials are taken relative to a reference: 0 to begin with, the row maximum when that
-        // turns out to be too far from 0 (rare: logits beyond +-60 / temperature); a NaN in the rows switches the
-        // node's passes to their cleaning form.
-        for (int attempt = 0; attempt < 4; ++attempt) {
+        // First pass.  Exponentials are taken relative to a reference, 0 to begin with: the plain pass has no code for
+        // maxima or NaN.  If its sums are not finite, or so small that underflow may have eaten them (logits beyond
+        // about +-40 / temperature), a cleaning pass finds the rows' maxima and the pass is run again relative to them.
+        {
             double S0, S1;
             float M0, M1;
-            if (st.with_draft) {
-                if (st.has_nan) ring.template pass<kPassFirst, true, false>(rowq, rowp, st, S0, S1, M0, M1);
-                else ring.template pass<kPassFirst, false, false>(rowq, rowp, st, S0, S1, M0, M1);
-            } else {
-                if (st.has_nan) ring.template pass<kPassTarget, true, true>(rowq, rowp, st, S0, S1, M0, M1);
-                else ring.template pass<kPassTarget, false, true>(rowq, rowp, st, S0, S1, M0, M1);
-                M1 = 0.0f;
-                S1 = 1.0;
+            const int kind = st.with_draft ? kPassFirst : kPassTarget;
+            for (int attempt = 0; attempt < 3; ++attempt) {
+                run_pass(kind, !st.with_draft, S0, S1, M0, M1);
+                if (sm.abort) { aborted = true; break; }
+                if (!st.with_draft) S1 = 1.0;
+                const bool good = S0 >= (double)kSumFloor && S0 < 1e300 && S1 >= (double)kSumFloor && S1 < 1e300;
+                if (attempt == 0) {
+                    if (good) break;
+                    st.has_nan = true;                 // next: the cleaning pass, which also returns the maxima
+                    if (lane == 0) sm.nan_seen = 0;    // (published with the next command)
+                } else if (attempt == 1) {
+                    if (sm.nan_seen) status |= 1;      // RSD_ST_NAN_INPUT: the node's passes keep cleaning
+                    else st.has_nan = false;
+                    if (good) break;                   // only a NaN was in the way
+                    if (M0 > kNegInf) st.mq = M0;      // under- or overflow: once more, relative to the maxima
+                    if (st.with_draft && M1 > kNegInf) st.mp = M1;
+                }
             }
-            if (attempt == 0 && warp == kWorkWarps && st.with_draft) {
-#pragma unroll
-                for (int r = 0; r < kMaxChildren / 32; ++r) { sm.child_lq[r * 32 + lane] = ahead_q[r]; sm.child_lp[r * 32 + lane] = ahead_p[r]; }
-            }
-            if (sm.abort) break;
-            if (!st.has_nan && (M0 != M0 || M1 != M1)) {   // a NaN logit: counts as -inf, reported
-                st.has_nan = true;
-                status |= 1;                                // RSD_ST_NAN_INPUT
-                continue;
-            }
+            if (aborted) break;
             st.Sq = S0;
             st.Sp = S1;
-            const bool redo_q = M0 > kNegInf && fabsf((M0 - st.mq) * st.kq) > kRefSlack * kLog2e;
-            const bool redo_p = st.with_draft && M1 > kNegInf && fabsf((M1 - st.mp) * st.kp) > kRefSlack * kLog2e;
-            if (!redo_q && !redo_p) { tiles_valid = !st.with_draft; break; }
-            if (redo_q) st.mq = M0;
-            if (redo_p) st.mp = M1;
+            tiles_valid = !st.with_draft;
         }
-        if (tid == 0) sm.n_removed = 0;
-        __syncthreads();   // the children's values are in shared memory
-        if (sm.abort) break;
         if (!st.with_draft) {
             reason = (len >= a.L) ? 2 : 1;  // RSD_STOP_LEAF : RSD_STOP_NO_CHILDREN
             break;
         }
         int accepted = -1, j = 0;
+        int rem_x[4];            // rejected tokens of this node, lanes hold them four at a time (lane i: entries 4 i ..)
+        int n_removed = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) rem_x[i] = -1;
         while (c >= 0) {
-            const int x = cached ? sm.tok[c] : tok[c];
+            int x;
             float lq, lp;
-            if (j < kMaxChildren) { lq = sm.child_lq[j]; lp = sm.child_lp[j]; }
-            else { lq = RowIO<T>::scalar(rowq, x); lp = RowIO<T>::scalar(rowp, x); }
+            if (j < 32) {
+                x = __shfl_sync(0xFFFFFFFFu, child_x, j);
+                lq = __shfl_sync(0xFFFFFFFFu, child_lq, j);
+                lp = __shfl_sync(0xFFFFFFFFu, child_lp, j);
+            } else {
+                x = cached ? sm.tok[c] : tok[c];
+                lq = RowIO<T>::scalar(rowq, x);
+                lp = RowIO<T>::scalar(rowp, x);
+            }
             const float qh = (lq == lq) ? ex2_approx(fmaf(lq, st.kq, -st.mq * st.kq)) : 0.0f;
             const float ph = (lp == lp) ? ex2_approx(fmaf(lp, st.kp, -st.mp * st.kp)) : 0.0f;
             const double qx = (double)qh / st.Sq, px_row = (double)ph / st.Sp;
-            bool repeated = false;   // a sibling with the same token was rejected before: its draft mass is gone (Eq. 1)
-            for (int i = 0; i < sm.n_removed; ++i) repeated |= sm.rem_x[i] == x;
+            // a sibling with the same token was rejected before: its draft mass is gone (Eq. 1)
+            bool mine = false;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) mine |= rem_x[i] == x;
+            const bool repeated = __any_sync(0xFFFFFFFFu, mine);
             const double px = repeated ? 0.0 : px_row;
             const double r = fmax(qx - st.A * px_row, 0.0);
             double theta;
@@ -452,10 +492,10 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             else { status |= 8; theta = r > 0.0 ? 1.0 : 0.0; }   // RSD_ST_ZERO_DRAFT_PROB
             const uint4 rw = rng_draw(key, (uint32_t)cur, kTagAccept, (uint32_t)j);
             const double U = (double)(rw.x >> 8) * (1.0 / 16777216.0);
-            if (a.dbg_theta && tid == 0) a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)theta;
+            if (a.dbg_theta && lane == 0) a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)theta;
             if (U < theta) { accepted = c; break; }
             ++j;
-            const int next = find_child(cur, c);
+            const int next = j < 32 ? __shfl_sync(0xFFFFFFFFu, child_node, j) : find_child(cur, c);
             // Eqs. 1-2 in closed form: A_{j+1} = A_j + Z_j / (1 - P_j), Z_{j+1} = sum (q - A_{j+1} p)+
             const double A_old = st.A;
             st.A = st.A + st.Z / (1.0 - st.P);
@@ -467,14 +507,8 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             double zhat, none;
             float f0, f1;
             const bool maybe_last = next < 0;   // no sibling left: the last token is drawn from this residual
-            if (st.has_nan) {
-                if (maybe_last) ring.template pass<kPassResidual, true, true>(rowq, rowp, st, zhat, none, f0, f1);
-                else ring.template pass<kPassResidual, true, false>(rowq, rowp, st, zhat, none, f0, f1);
-            } else {
-                if (maybe_last) ring.template pass<kPassResidual, false, true>(rowq, rowp, st, zhat, none, f0, f1);
-                else ring.template pass<kPassResidual, false, false>(rowq, rowp, st, zhat, none, f0, f1);
-            }
-            if (sm.abort) break;
+            run_pass(kPassResidual, maybe_last, zhat, none, f0, f1);
+            if (sm.abort) { aborted = true; break; }
             const double Z_new = zhat / st.Sq;
             if (Z_new > 0.0 && Z_new < 1.7e308) {
                 st.Z = Z_new;
@@ -488,17 +522,23 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
                 tiles_valid = false;
             }
             st.P += px;
-            if (tid == 0 && !repeated && sm.n_removed < kMaxRemovedRing) sm.rem_x[sm.n_removed++] = x;
-            __syncthreads();
-            if (!(1.0 - st.P > 0.0)) { status |= 16; tiles_valid = tiles_valid && maybe_last; break; }   // RSD_ST_DRAFT_EXHAUSTED
+            if (!repeated && n_removed < kMaxRemovedRing) {
+                if (lane == (n_removed >> 2)) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (i == (n_removed & 3)) rem_x[i] = x;
+                }
+                ++n_removed;
+            }
+            if (!(1.0 - st.P > 0.0)) { status |= 16; break; }   // RSD_ST_DRAFT_EXHAUSTED
             c = next;
         }
-        if (sm.abort) break;
+        if (aborted) break;
         if (accepted < 0) {   // RSD_STOP_ALL_REJECTED: the last token comes from the residual in force
             reason = 0;
             break;
         }
-        if (tid == 0) {
+        if (lane == 0) {
             a.accepted_node[(int64_t)b * a.L + len] = accepted;
             a.accepted_token[(int64_t)b * a.L + len] = cached ? sm.tok[accepted] : tok[accepted];
         }
@@ -506,117 +546,106 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
         cur = accepted;
     }
 
-    if (!sm.abort) {
-        const bool residual = st.with_draft && st.A != 0.0;
-        if (!tiles_valid) {   // rare: the last pass was not kept, or it did not store its tile sums
-            double s, none;
-            float f0, f1;
-            if (residual) {
-                if (st.has_nan) ring.template pass<kPassResidual, true, true>(rowq, rowp, st, s, none, f0, f1);
-                else ring.template pass<kPassResidual, false, true>(rowq, rowp, st, s, none, f0, f1);
-            } else {
-                if (st.has_nan) ring.template pass<kPassTarget, true, true>(rowq, rowq, st, s, none, f0, f1);
-                else ring.template pass<kPassTarget, false, true>(rowq, rowq, st, s, none, f0, f1);
-            }
-        }
+    const bool residual = st.with_draft && st.A != 0.0;
+    if (!aborted && !tiles_valid) {   // rare: the last pass was not kept, or it did not store its tile sums
+        double s, none;
+        float f0, f1;
+        if (!residual) rowp = rowq;
+        run_pass(residual ? kPassResidual : kPassTarget, true, s, none, f0, f1);
+        aborted = sm.abort != 0;
     }
-    if (!sm.abort) {
-        // Inverse CDF over the tile sums of the last pass: the smallest y whose running sum exceeds u * total; if
-        // rounding leaves none, the largest y with positive weight; -1 if there is no weight at all.
-        const bool residual = st.with_draft && st.A != 0.0;
-        const uint4 rw = rng_draw(key, (uint32_t)cur, kTagResample, 0u);
-        const double u = ((double)rw.x + 0.5) * (1.0 / 4294967296.0);
-        __syncthreads();   // every tile sum is in place
-        if (warp == 0) {
-            const int n_tiles = ring.n_tiles;
-            // lanes take consecutive runs of tiles; running sums in tile order
-            const int per = (n_tiles + 31) / 32;
-            const int t_lo = lane * per, t_hi = min(n_tiles, t_lo + per);
-            double mine = 0.0;
-            for (int t = t_lo; t < t_hi; ++t) mine += sm.tile_sum[t];
-            double incl = mine;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const double t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                if (lane >= o) incl += t;
-            }
-            const double total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-            int y = -1;
-            if (total > 0.0 && total < 1.7e308) {   // (uniform over the warp)
-                const double target = u * total;
-                // the tile that holds the crossing, or failing that the last tile with weight
-                const unsigned crossing = __ballot_sync(0xFFFFFFFFu, incl > target);
-                const unsigned positive = __ballot_sync(0xFFFFFFFFu, mine > 0.0);
-                const bool take_last = crossing == 0u;
-                const int src = take_last ? 31 - __clz(positive) : __ffs(crossing) - 1;
-                int tile = -1;
-                double before = 0.0;
-                if (lane == src) {
-                    double cum = incl - mine;
-                    for (int t = t_lo; t < t_hi; ++t) {
-                        const double s = sm.tile_sum[t];
-                        if (take_last) { if (s > 0.0) { tile = t; before = cum; } }
-                        else if (cum + s > target) { tile = t; before = cum; break; }
-                        cum += s;
-                    }
-                    if (tile < 0) {   // rounding: the lane's total crossed, no tile did: its last tile with weight
-                        cum = incl - mine;
-                        for (int t = t_lo; t < t_hi; ++t) {
-                            const double s = sm.tile_sum[t];
-                            if (s > 0.0) { tile = t; before = cum; }
-                            cum += s;
-                        }
-                    }
-                }
-                tile = __shfl_sync(0xFFFFFFFFu, tile, src);
-                before = __shfl_sync(0xFFFFFFFFu, before, src);
-                // the tile's weights once more, in token order: lane owns tokens 16 lane .. 16 lane + 15 of the tile
-                float w[16];
-                const int g = tile * 32 + lane;
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj) w[jj] = 0.0f;
-                if (tile >= 0 && g * 16 < a.V) group_weights<T>(rowq, rowp, g, a.V, st, residual, w);
-                double gs = 0.0;
-#pragma unroll
-                for (int jj = 0; jj < 16; ++jj) gs += (double)w[jj];
-                double gincl = gs;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const double t = __shfl_up_sync(0xFFFFFFFFu, gincl, o);
-                    if (lane >= o) gincl += t;
-                }
-                const unsigned cross2 = __ballot_sync(0xFFFFFFFFu, !take_last && (before + gincl > target));
-                const unsigned pos2 = __ballot_sync(0xFFFFFFFFu, gs > 0.0);
-                const bool last_mode = cross2 == 0u;
-                const int src2 = last_mode ? (pos2 ? 31 - __clz(pos2) : 0) : __ffs(cross2) - 1;
-                if (lane == src2) {
-                    int last_pos = -1;
-                    double cacc = before + (gincl - gs);
-#pragma unroll
-                    for (int jj = 0; jj < 16; ++jj) {
-                        cacc += (double)w[jj];
-                        if (w[jj] > 0.0f) last_pos = g * 16 + jj;
-                        if (!last_mode && y < 0 && cacc > target) y = g * 16 + jj;
-                    }
-                    if (y < 0) y = last_pos;
-                }
-                y = __shfl_sync(0xFFFFFFFFu, y, src2);
-            }
-            if (lane == 0) sm.pick = y;
-        }
-        __syncthreads();
-        last = sm.pick;
-    } else {
+    // the working warps are done: let them go, then finish alone
+    if (lane == 0) sm.cmd.kind = kPassEnd;
+    if (aborted) {
         // A wait ran out.  Before the block gives its shared memory back, wait once more (bounded) for the copies it
         // may still have in flight: the last kSlots chunks it asked for.
-        if (warp == kWorkWarps) {
-            for (uint32_t g = ring.g0 > (uint32_t)kSlots ? ring.g0 - kSlots : 0u; g < ring.g0; ++g)
-                wait_bar(&sm.full[g & (kSlots - 1)], (g / kSlots) & 1u, &sm.abort);
-        }
+        for (uint32_t g = ring.g0 > (uint32_t)kSlots ? ring.g0 - kSlots : 0u; g < ring.g0; ++g)
+            wait_bar(&sm.full[g & (kSlots - 1)], (g / kSlots) & 1u, &sm.abort);
         status |= 32;   // RSD_ST_TIMEOUT
-        __syncthreads();
     }
-    if (tid == 0) {
+    __syncthreads();
+    if (!aborted) {
+        // Inverse CDF over the tile sums of the last pass: the smallest y whose running sum exceeds u * total; if
+        // rounding leaves none, the largest y with positive weight; -1 if there is no weight at all.
+        const uint4 rw = rng_draw(key, (uint32_t)cur, kTagResample, 0u);
+        const double u = ((double)rw.x + 0.5) * (1.0 / 4294967296.0);
+        const int n_tiles = ring.n_tiles;
+        // lanes take consecutive runs of tiles; running sums in tile order
+        const int per = (n_tiles + 31) / 32;
+        const int t_lo = lane * per, t_hi = min(n_tiles, t_lo + per);
+        double mine = 0.0;
+        for (int t = t_lo; t < t_hi; ++t) mine += sm.tile_sum[t];
+        double incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        const double total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        int y = -1;
+        if (total > 0.0 && total < 1.7e308) {   // (uniform over the warp)
+            const double target = u * total;
+            // the tile that holds the crossing, or failing that the last tile with weight
+            const unsigned crossing = __ballot_sync(0xFFFFFFFFu, incl > target);
+            const unsigned positive = __ballot_sync(0xFFFFFFFFu, mine > 0.0);
+            const bool take_last = crossing == 0u;
+            const int src = take_last ? 31 - __clz(positive) : __ffs(crossing) - 1;
+            int tile = -1;
+            double before = 0.0;
+            if (lane == src) {
+                double cum = incl - mine;
+                for (int t = t_lo; t < t_hi; ++t) {
+                    const double s = sm.tile_sum[t];
+                    if (take_last) { if (s > 0.0) { tile = t; before = cum; } }
+                    else if (cum + s > target) { tile = t; before = cum; break; }
+                    cum += s;
+                }
+                if (tile < 0) {   // rounding: the lane's total crossed, no tile did: its last tile with weight
+                    cum = incl - mine;
+                    for (int t = t_lo; t < t_hi; ++t) {
+                        const double s = sm.tile_sum[t];
+                        if (s > 0.0) { tile = t; before = cum; }
+                        cum += s;
+                    }
+                }
+            }
+            tile = __shfl_sync(0xFFFFFFFFu, tile, src);
+            before = __shfl_sync(0xFFFFFFFFu, before, src);
+            // the tile's weights once more, in token order: lane owns tokens 16 lane .. 16 lane + 15 of the tile
+            float w[16];
+            const int g = tile * 32 + lane;
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) w[jj] = 0.0f;
+            if (tile >= 0 && g * 16 < a.V) group_weights<T>(rowq, rowp, g, a.V, st, residual, w);
+            double gs = 0.0;
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) gs += (double)w[jj];
+            double gincl = gs;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double t = __shfl_up_sync(0xFFFFFFFFu, gincl, o);
+                if (lane >= o) gincl += t;
+            }
+            const unsigned cross2 = __ballot_sync(0xFFFFFFFFu, !take_last && (before + gincl > target));
+            const unsigned pos2 = __ballot_sync(0xFFFFFFFFu, gs > 0.0);
+            const bool last_mode = cross2 == 0u;
+            const int src2 = last_mode ? (pos2 ? 31 - __clz(pos2) : 0) : __ffs(cross2) - 1;
+            if (lane == src2) {
+                int last_pos = -1;
+                double cacc = before + (gincl - gs);
+#pragma unroll
+                for (int jj = 0; jj < 16; ++jj) {
+                    cacc += (double)w[jj];
+                    if (w[jj] > 0.0f) last_pos = g * 16 + jj;
+                    if (!last_mode && y < 0 && cacc > target) y = g * 16 + jj;
+                }
+                if (y < 0) y = last_pos;
+            }
+            y = __shfl_sync(0xFFFFFFFFu, y, src2);
+        }
+        last = y;
+    }
+    if (lane == 0) {
         a.accepted_len[b] = len;
         a.last_token[b] = last;
         a.stop_reason[b] = reason;
