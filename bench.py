@@ -26,10 +26,22 @@ if ROOT not in sys.path:
 
 import workloads  # noqa: E402
 
-# DRAM bytes moved per algorithmic byte by the scan kernel, from the ncu capture summarised in
-# profiles/scan_topk_kernel_workload5_256seq.md (dram__bytes_read + dram__bytes_write over rows x V x 2 bytes; the
-# traffic grows in proportion to the rows scanned).  Set to None whenever the kernel changes after a capture.
+# DRAM bytes moved per algorithmic byte by the scan kernel, from the committed ncu summary of the scan kernel
+# (dram__bytes_read + dram__bytes_write over rows x V x 2 bytes; the traffic grows in proportion to the rows scanned),
+# together with the SHA-256 of the kernel sources it was measured on: when the sources differ, `traffic` is null.
 SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.042
+SCAN_TRAFFIC_SOURCES = ("paper_2402_14160_b200/csrc/rsd_scan.cuh", "paper_2402_14160_b200/csrc/rsd_device.cuh")
+SCAN_TRAFFIC_SOURCE_SHA256 = "@@SCAN_SHA@@"
+
+
+def _scan_sources_sha256():
+    import hashlib
+    h = hashlib.sha256()
+    for rel in SCAN_TRAFFIC_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
 
 METRIC = "verified tree nodes/sec"
 UNIT = "nodes/s"
@@ -78,7 +90,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(0.001)
 
     def __enter__(self):
         if self.ok:
@@ -100,18 +112,23 @@ class ClockSampler:
 
 
 def _oracle_sample_step(w, draft_h, target_h, seed, step, seq_base):
-    """One draft + verify step of the oracle over a block of sequences (host arrays)."""
+    """One draft + verify step of the oracle over a block of sequences (host arrays).  Returns the walk's outputs
+    plus `draft_margin` [b]: the smallest gap of any drafting decision of the sequence."""
     import oracle
     if w.mode == "rsd_c":
         k, nodes = workloads.rsdc_rows(w.branching)
         d = oracle.gumbel_topk(draft_h, k, nodes, seed, step, seq_base=seq_base)
         parent = workloads.rsdc_parent_array(w.branching)
         token = workloads.rsdc_tokens_from_rows(w.branching, d["token"])
-        return oracle.verify_tree(draft_h, target_h, parent, token, w.num_levels, seed, step, seq_base=seq_base)
+        v = oracle.verify_tree(draft_h, target_h, parent, token, w.num_levels, seed, step, seq_base=seq_base)
+        v["draft_margin"] = d["margin"].min(axis=1)
+        v["tree_token"] = token
+        return v
     W, L = w.beam_width, w.depth
     nb = draft_h.shape[0]
     parent = np.full((nb, 1 + W * L), -1, np.int32)
     token = np.full((nb, 1 + W * L), -1, np.int32)
+    margin = np.full(nb, np.inf)
     prev = None
     for l in range(L):
         first = 0 if l == 0 else 1 + (l - 1) * W
@@ -122,23 +139,57 @@ def _oracle_sample_step(w, draft_h, target_h, seed, step, seq_base):
         sl = slice(1 + l * W, 1 + (l + 1) * W)
         token[:, sl] = o["token"]
         parent[:, sl] = np.where(o["parent"] >= 0, first + o["parent"], -1)
+        margin = np.minimum(margin, o["margin"])
         prev = o
-    return oracle.verify_tree(draft_h, target_h, parent, token, L, seed, step, seq_base=seq_base)
+    v = oracle.verify_tree(draft_h, target_h, parent, token, L, seed, step, seq_base=seq_base)
+    v["draft_margin"] = margin
+    v["tree_token"] = token
+    return v
 
 
-def _time_oracle(w, n_seq, steps, warmup):
-    """Oracle on the host cores over the first n_seq sequences of the workload; returns (nodes/s, seconds/step)."""
+def _time_oracle(w, n_seq, steps, warmup, threads=None, rows=None):
+    """Oracle on the host cores over the first n_seq sequences of the workload (generated on the host, or the given
+    (draft, target) tensors); returns (nodes/s, seconds/step, threads used, outputs of the last step)."""
     import oracle
     oracle.build()
-    draft, target = workloads.make_logits(w, step=0, device="cpu", seq_begin=0, seq_end=n_seq)
+    if threads is not None:
+        oracle.set_num_threads(threads)
+    if rows is None:
+        draft, target = workloads.make_logits(w, step=0, device="cpu", seq_begin=0, seq_end=n_seq)
+    else:
+        draft, target = rows[0][:n_seq], rows[1][:n_seq]
     dh, th = workloads.as_oracle_rows(draft), workloads.as_oracle_rows(target)
     for s in range(warmup):
         _oracle_sample_step(w, dh, th, 0, s, 0)
     t0 = time.perf_counter()
+    out = None
     for s in range(steps):
-        _oracle_sample_step(w, dh, th, 0, warmup + s, 0)
+        out = _oracle_sample_step(w, dh, th, 0, warmup + s, 0)
     dt = (time.perf_counter() - t0) / max(steps, 1)
-    return n_seq * w.num_nodes / dt, dt, oracle.num_threads()
+    used = threads if threads is not None else oracle.num_threads()
+    if threads is not None:
+        oracle.set_num_threads(oracle.num_threads())
+    return n_seq * w.num_nodes / dt, dt, used, out
+
+
+def _parity_sample(gpu, tree_token, ora, margin=1e-5):
+    """Sequences of the sample whose GPU step differs from the oracle's, split by the oracle's smallest margin."""
+    n = len(ora["accepted_len"])
+    differ = borderline = 0
+    for b in range(n):
+        same = (np.array_equal(tree_token[b], ora["tree_token"][b]) and gpu["accepted_len"][b] == ora["accepted_len"][b]
+                and np.array_equal(gpu["accepted_node"][b], ora["accepted_node"][b])
+                and gpu["last_token"][b] == ora["last_token"][b])
+        if same:
+            continue
+        differ += 1
+        m = min(float(ora["draft_margin"][b]), float(np.nanmin(np.append(ora["margin"][b], np.inf))),
+                float(ora["final_margin"][b]))
+        borderline += 1 if m <= margin else 0
+    return {"sequences": n, "differ": differ, "of_which_borderline": borderline,
+            "note": "one step (seed 0, step 0) of the GPU path against the oracle on the cpu_baseline sample; a "
+                    "sequence differs if its tree, accepted path or last token does; borderline = the oracle's smallest "
+                    "decision margin of that sequence is <= 1e-5"}
 
 
 def run_reference(args, w):
@@ -146,7 +197,7 @@ def run_reference(args, w):
     if rank != 0:
         return
     n_seq = min(w.batch, args.ref_sequences)
-    value, dt, cores = _time_oracle(w, n_seq, args.steps, args.warmup)
+    value, dt, cores, _ = _time_oracle(w, n_seq, args.steps, args.warmup)
     sample = "%d of %d sequences of workload %d per step, whole draft+verify step" % (n_seq, w.batch, w.config_id)
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
@@ -171,6 +222,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--sequences", type=int, default=0, help="sequences per GPU (default: the workload's batch)")
+    ap.add_argument("--per-level", action="store_true",
+                    help="Stochastic Beam Search: one rsd_sbs_step call per level instead of rsd_sbs_draft_tree")
     args = ap.parse_args()
     w = workloads.WORKLOADS[args.workload]
     if args.sequences > 0:
@@ -201,7 +254,7 @@ def main():
     B = w.batch
     seq_base = rank * B
     draft, target = workloads.make_logits(w, step=0, device=str(dev), seq_begin=0, seq_end=B)
-    stepper = rsd_step.make_step(w, device=dev)
+    stepper = rsd_step.make_step(w, device=dev, rows_ready=not args.per_level)
     is_sbs = w.mode == "rsd_s"
     L = w.num_levels
     resident_bytes = draft.numel() * draft.element_size() + target.numel() * target.element_size()
@@ -218,21 +271,22 @@ def main():
 
     # ---- timed region: K steps, events on the launching stream -------------------------------------------
     K = args.steps
-    n_scan = (L if is_sbs else 1)
-    scan_ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_scan)]
-               for _ in range(K)]
-    ver_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    for row in scan_ev:
-        for a, b in row:
-            a.record(); b.record()          # creates the handles
-    for a, b in ver_ev:
-        a.record(); b.record()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    per_level = is_sbs and args.per_level
+    n_scan = (L if per_level else 1)
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()          # creates the handle
+        return e
+
+    scan_ev = [[(ev(), ev()) for _ in range(n_scan)] for _ in range(K)]
+    ver_ev = [(ev(), ev()) for _ in range(K)]
+    step_ev = [ev() for _ in range(K + 1)]
     barrier()
     with ClockSampler(local) as clocks:
-        e0.record()
+        step_ev[0].record()
         for s in range(K):
-            if is_sbs:
+            if per_level:
                 W = stepper.W
                 for l in range(L):
                     first = 0 if l == 0 else 1 + (l - 1) * W
@@ -247,6 +301,9 @@ def main():
                                      None if l == 0 else prev["sum_logprob"], None if l == 0 else prev["trunc_gumbel"],
                                      0, 1000 + s, is_logprob=w.draft_is_logprob, seq_base=seq_base,
                                      workspace=stepper.workspace, out=out, parent_base=first)
+            elif is_sbs:
+                api.rsd_profile_next_scan(*scan_ev[s][0])
+                stepper.draft_tree(draft, 0, 1000 + s, seq_base)
             else:
                 api.rsd_profile_next_scan(*scan_ev[s][0])
                 api.rsd_gumbel_topk_draft(draft, stepper.k_per_row, stepper.rng_node, 0, 1000 + s, seq_base=seq_base,
@@ -256,9 +313,10 @@ def main():
             stepper.verify_out = api.rsd_verify_tree(draft, target, stepper.parent, stepper.token, L, 0, 1000 + s,
                                                      seq_base=seq_base, out=stepper.verify_out)
             ver_ev[s][1].record()
-        e1.record()
+            step_ev[s + 1].record()
         torch.cuda.synchronize()
-    elapsed_ms = e0.elapsed_time(e1)
+    elapsed_ms = step_ev[0].elapsed_time(step_ev[K])
+    per_step_ms = [step_ev[i].elapsed_time(step_ev[i + 1]) for i in range(K)]
     barrier()
     if dist is not None:
         t = torch.tensor([elapsed_ms], device=dev, dtype=torch.float64)
@@ -284,10 +342,10 @@ def main():
     ver_gbs = ver_bytes / (ver_ms / K * 1e-3) / 1e9
     roofline = {"kernel": "scan_topk_kernel (Gumbel-Top-k / SBS parent-row scan)", "bound": "hbm",
                 "achieved": scan_gbs, "peak": peak, "unit": "GB/s", "frac": scan_gbs / peak, "peak_kind": peak_kind,
-                "traffic": (None if SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE is None else
-                            SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE * scan_bytes_per_step / n_scan),
+                "traffic": (SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE * scan_bytes_per_step / n_scan
+                            if _scan_sources_sha256() == SCAN_TRAFFIC_SOURCE_SHA256 else None),
                 "traffic_note": "DRAM bytes per scan launch (average over the step's launches), scaled by rows from a "
-                                "256-sequence ncu capture",
+                                "256-sequence ncu capture; null when the kernel sources changed since that capture",
                 "algorithmic_bytes_per_step": scan_bytes_per_step,
                 "launches_per_step": n_scan, "avg_launch_ms": scan_ms / (K * n_scan),
                 "launch_ms_by_level": [sum(scan_ev[s][l][0].elapsed_time(scan_ev[s][l][1]) for s in range(K)) / K
@@ -311,9 +369,15 @@ def main():
                                 else {"branching": list(w.branching)}),
                        "l2": "inputs larger than L2 (%.2f GB resident per GPU)" % (resident_bytes / 1e9)
                        if resident_bytes > 256e6 else "inputs smaller than L2: timings are cache-assisted",
+                       "drafting": ("rsd_sbs_step per level" if per_level else
+                                    "rsd_sbs_draft_tree (all levels, rows ready)" if is_sbs else "rsd_gumbel_topk_draft"),
                        "mean_accepted_len": float(acc.mean())},
             "clocks": clocks.summary(), "gpu_launches": stepper.kernel_launches * K, "roofline": roofline,
-            "phases": phases}
+            "phases": phases,
+            "step_ms": {"mean": elapsed_ms / K, "median": float(np.median(per_step_ms)), "best": float(np.min(per_step_ms)),
+                        "note": "per-step CUDA-event times on this rank; `value` uses the mean (max over ranks)"},
+            "accepted_len_histogram": np.bincount(acc, minlength=L + 1).tolist(),
+            "block_efficiency": float(acc.mean()) + 1.0}
 
     # ---- end to end: pinned host logits -> device -> step -> results on the host ---------------------------
     if not args.no_e2e:
@@ -354,9 +418,18 @@ def main():
     # ---- the oracle on the host cores, bounded sample (rank 0, one GPU only) ----------------------------------
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         n_seq = min(B, args.cpu_baseline_sequences)
-        v, dt, cores = _time_oracle(w, n_seq, 1, 0)
+        v, dt, cores, ora = _time_oracle(w, n_seq, 1, 0, rows=(draft, target))   # the rows the GPU holds
+        n_one = max(1, min(n_seq, args.cpu_baseline_sequences // 32))
+        v1, dt1, _, _ = _time_oracle(w, n_one, 1, 0, threads=1)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": "%d of %d sequences, one whole draft+verify step (%.1f s)" % (n_seq, B, dt)}
+                                "sample": "%d of %d sequences, one whole draft+verify step (%.1f s)" % (n_seq, B, dt),
+                                "single_thread": {"value": v1, "unit": UNIT,
+                                                  "sample": "%d sequences, one step (%.1f s)" % (n_one, dt1)}}
+        # the same step on the GPU, compared with what the oracle just computed
+        gv = stepper.run(draft, target, 0, 0, 0)
+        torch.cuda.synchronize()
+        g = {k2: v2[:n_seq].cpu().numpy() for k2, v2 in gv.items() if v2 is not None}
+        line["parity_sample"] = _parity_sample(g, stepper.token[:n_seq].cpu().numpy(), ora)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

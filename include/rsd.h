@@ -158,6 +158,31 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
                  size_t ws_bytes, rsd_stream_t stream);
 
 /*
+ * A whole Stochastic Beam Search tree in two launches (Algorithm 8's level loop around Algorithm 9; Eqs. 10-12), for
+ * draft rows that all exist before drafting starts.  Row r of a sequence is the draft row of flat node r: the root,
+ * then the W slots of level 1, ..., level L - 1 (P = 1 + (L - 1) W rows).  That is the case when the rows do not
+ * depend on the tokens picked above them (rows attached to tree slots, as in synthetic workloads or with drafters that
+ * predict every position at once); with an autoregressive drafter the rows of a level are only known after the
+ * level above, and rsd_sbs_step is the call to use.
+ * One launch scans all B * P rows (each with the Gumbel stream of its node), one launch runs the L levels in order,
+ * carrying the sequence log-probabilities and truncated Gumbels from level to level on the device.  The results are
+ * those of L rsd_sbs_step calls (level l: rows first .. first + n_par with first = 0, n_par = 1 at the root, else
+ * first = 1 + (l - 1) W, n_par = W; first_parent_node = parent_base = first), bit for bit.
+ *   draft             rows [B][P][V]
+ *   node_token, node_parent   [B][node_stride] int32, node_stride >= 1 + L W: entries 1 + l W .. (l + 1) W receive the
+ *                     tokens and flat parents of level l + 1's nodes (-1 beyond the level's count); entry 0 (the
+ *                     root) is left alone: the arrays are rsd_verify_tree's token / parent
+ *   sum_logprob_out, trunc_gumbel_out   optional [B][W]: phi and psi of the last level's picks
+ *   level_count       [L][B]: picks of every level;  status [B]: OR of the levels' status bits
+ *   ws                scratch of at least rsd_sbs_tree_workspace_bytes(B, W, L) bytes, 256-byte aligned
+ */
+size_t rsd_sbs_tree_workspace_bytes(int B, int W, int L);
+int rsd_sbs_draft_tree(const rsd_rows* draft, int B, int V, int W, int L, uint64_t seed, uint32_t step,
+                       uint32_t seq_base, int32_t* node_token, int32_t* node_parent, int64_t node_stride,
+                       float* sum_logprob_out, float* trunc_gumbel_out, int32_t* level_count, int32_t* status, void* ws,
+                       size_t ws_bytes, rsd_stream_t stream);
+
+/*
  * rsd_sbs_step for callers that cannot allocate device memory (the paper has no counterpart).
  * Some hosts of this library may not call cudaMalloc where they draft: code running inside a serving engine whose
  * memory pool is fixed at start-up, a plug-in that is handed a stream but no allocator, a latency-critical loop that

@@ -67,6 +67,12 @@ def num_threads() -> int:
         return os.cpu_count() or 1
 
 
+def set_num_threads(n: int) -> None:
+    """Threads of the OpenMP loops from now on (the benchmark's single-thread figure)."""
+    lib()
+    C.CDLL("libgomp.so.1").omp_set_num_threads(int(n))
+
+
 def _ptr(a):
     return None if a is None else a.ctypes.data_as(C.c_void_p)
 

@@ -16,14 +16,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("RSD_LIB_PATH") or os.path.join(_HERE, "librsd.so")  # override: a variant build
 
 RSD_F32, RSD_BF16 = 0, 1
-ST_NAN_INPUT, ST_FEWER_THAN_K, ST_ZERO_RESIDUAL, ST_ZERO_DRAFT_PROB, ST_DRAFT_EXHAUSTED = 1, 2, 4, 8, 16
+ST_NAN_INPUT, ST_FEWER_THAN_K, ST_ZERO_RESIDUAL, ST_ZERO_DRAFT_PROB, ST_DRAFT_EXHAUSTED, ST_TIMEOUT = 1, 2, 4, 8, 16, 32
 STOP_ALL_REJECTED, STOP_NO_CHILDREN, STOP_LEAF = 0, 1, 2
 RULE_RRS, RULE_MULTIROUND, RULE_KSEQ = 0, 1, 2
 FINAL_INVERSE_CDF, FINAL_GUMBEL_TOP1 = 0, 1
 MAX_K = 32
 
 EXPORTS = ["rsd_version", "rsd_rng_layout", "rsd_last_error", "rsd_profile_next_scan", "rsd_gumbel_topk_draft", "rsd_sbs_workspace_bytes",
-           "rsd_sbs_step", "rsd_sbs_step_static", "rsd_verify_tree", "rsd_verify_tree_rule", "rsd_resample_residual"]
+           "rsd_sbs_step", "rsd_sbs_step_static", "rsd_sbs_tree_workspace_bytes", "rsd_sbs_draft_tree", "rsd_verify_tree", "rsd_verify_tree_rule", "rsd_resample_residual"]
 
 
 class RsdRows(C.Structure):
@@ -62,6 +62,11 @@ def lib():
                                    C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
                                    C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]
+        l.rsd_sbs_tree_workspace_bytes.restype = C.c_size_t
+        l.rsd_sbs_tree_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
+        l.rsd_sbs_draft_tree.argtypes = [C.POINTER(RsdRows), C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint64, C.c_uint32,
+                                         C.c_uint32, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         l.rsd_sbs_step_static.argtypes = [C.POINTER(RsdRows), C.c_int, C.c_int, C.c_int, C.c_int, C.c_int32,
                                           C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p,
                                           C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -183,6 +188,37 @@ def rsd_sbs_step(draft_level: torch.Tensor, W: int, first_parent_node: int, sum_
                               _ptr(trunc_gumbel_in), seed, step, seq_base, _ptr(out["token"]), _ptr(out["parent"]),
                               out["token"].stride(0), parent_base, _ptr(out["sum_logprob"]), _ptr(out["trunc_gumbel"]), _ptr(out["count"]),
                               _ptr(out["status"]), _ptr(workspace), workspace.numel(), _stream()))
+    return out
+
+
+def rsd_sbs_tree_workspace_bytes(B: int, W: int, L: int) -> int:
+    return int(lib().rsd_sbs_tree_workspace_bytes(B, W, L))
+
+
+def rsd_sbs_draft_tree(draft: torch.Tensor, W: int, L: int, seed: int, step: int, node_token: torch.Tensor,
+                       node_parent: torch.Tensor, *, is_logprob: bool = False, seq_base: int = 0,
+                       temperature: float = 1.0, workspace: Optional[torch.Tensor] = None, out: Optional[dict] = None):
+    """draft [B, 1 + (L - 1) W, V]: every level of one Stochastic Beam Search tree in two launches.  Fills
+    node_token / node_parent [B, >= 1 + L W] (the tree arrays rsd_verify_tree reads) and returns
+    dict(sum_logprob, trunc_gumbel [B, W] of the last level, count [L, B], status [B])."""
+    B, P, V = draft.shape
+    dev = draft.device
+    if P != 1 + (L - 1) * W:
+        raise RsdError("draft must hold 1 + (L - 1) W = %d rows per sequence, got %d" % (1 + (L - 1) * W, P))
+    if node_token.stride(0) != node_parent.stride(0) or node_token.stride(1) != 1 or node_parent.stride(1) != 1:
+        raise RsdError("node_token / node_parent must share a row stride and be dense along the nodes")
+    if workspace is None:
+        workspace = torch.empty((rsd_sbs_tree_workspace_bytes(B, W, L),), dtype=torch.uint8, device=dev)
+    if out is None:
+        out = dict(sum_logprob=torch.empty((B, W), dtype=torch.float32, device=dev),
+                   trunc_gumbel=torch.empty((B, W), dtype=torch.float32, device=dev),
+                   count=torch.empty((L, B), dtype=torch.int32, device=dev),
+                   status=torch.empty((B,), dtype=torch.int32, device=dev))
+    rows = rows_of(draft, is_logprob, temperature)
+    _check(lib().rsd_sbs_draft_tree(C.byref(rows), B, V, W, L, seed, step, seq_base, _ptr(node_token),
+                                    _ptr(node_parent), node_token.stride(0), _ptr(out["sum_logprob"]),
+                                    _ptr(out["trunc_gumbel"]), _ptr(out["count"]), _ptr(out["status"]),
+                                    _ptr(workspace), workspace.numel(), _stream()))
     return out
 
 

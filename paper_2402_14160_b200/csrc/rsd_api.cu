@@ -172,7 +172,8 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     if (int e = check_launch("rsd_sbs_step(scan)")) return e;
 
     rsd::SbsEpilogueArgs e;
-    e.n_par = n_par; e.W = W; e.is_logprob = rows_are_logprob(draft_level); e.inv_temp = 1.0 / (double)temperature_of(draft_level); e.first_parent_node = first_parent_node;
+    e.n_par = n_par; e.W = W; e.is_logprob = rows_are_logprob(draft_level);
+    e.fin_seq_stride = (int64_t)n_par * W; e.row_seq_stride = n_par; e.state_stride = n_par; e.inv_temp = 1.0 / (double)temperature_of(draft_level); e.first_parent_node = first_parent_node;
     e.seed_lo = (uint32_t)seed; e.seed_hi = (uint32_t)(seed >> 32); e.step = step; e.seq_base = seq_base;
     e.fin_token = fin_token; e.fin_value = fin_value; e.fin_pert = fin_pert; e.fin_lse = fin_lse;
     e.row_status = row_status;
@@ -183,6 +184,80 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     const size_t smem = (size_t)n_par * W * (8 + 8 + 4) + (size_t)n_par * 4;
     rsd::sbs_epilogue_kernel<<<B, rsd::kEpilogueThreads, smem, s>>>(e);
     return check_launch("rsd_sbs_step(epilogue)");
+}
+
+
+size_t rsd_sbs_tree_workspace_bytes(int B, int W, int L) {
+    if (B < 0 || W < 1 || L < 1) return 0;
+    const size_t P = 1 + (size_t)(L - 1) * W;
+    const size_t f = (size_t)B * P * W;
+    return align_up(f * 4, 256) * 3 + align_up((size_t)B * P * 4, 256) * 2   // finalists; log-sum-exp, row status
+           + align_up((size_t)B * W * 4, 256) * 4                            // two (sum, truncated Gumbel) states
+           + align_up((size_t)B * L * 4, 256);                               // status of every level
+}
+
+int rsd_sbs_draft_tree(const rsd_rows* draft, int B, int V, int W, int L, uint64_t seed, uint32_t step,
+                       uint32_t seq_base, int32_t* node_token, int32_t* node_parent, int64_t node_stride,
+                       float* sum_logprob_out, float* trunc_gumbel_out, int32_t* level_count, int32_t* status, void* ws,
+                       size_t ws_bytes, rsd_stream_t stream) {
+    g_err[0] = 0;
+    if (int e = check_vocab(V)) return e;
+    if (W < 1 || W > RSD_MAX_K) return fail(RSD_ERR_UNSUPPORTED, "W = %d outside [1, %d]", W, (int)RSD_MAX_K);
+    if (L < 1) return fail(RSD_ERR_INVALID_ARG, "L = %d", L);
+    const int64_t P = 1 + (int64_t)(L - 1) * W;
+    if (P > RSD_MAX_ROWS_PER_SEQ) return fail(RSD_ERR_UNSUPPORTED, "1 + (L - 1) W = %lld parent rows > %d", (long long)P, (int)RSD_MAX_ROWS_PER_SEQ);
+    if (W * W > 1024) return fail(RSD_ERR_UNSUPPORTED, "W * W = %d > 1024", W * W);
+    if (int e = check_rows("draft", draft, V, P > 1)) return e;
+    if (B < 0) return fail(RSD_ERR_INVALID_ARG, "B = %d", B);
+    if (!node_token || !node_parent || !level_count || !status) return fail(RSD_ERR_INVALID_ARG, "null output");
+    if (node_stride < 1 + (int64_t)L * W) return fail(RSD_ERR_INVALID_ARG, "node_stride = %lld < 1 + L W = %lld", (long long)node_stride, (long long)(1 + (int64_t)L * W));
+    if (B * P > 0x7FFFFFFF) return fail(RSD_ERR_UNSUPPORTED, "B * rows too large");
+    if (B == 0) return RSD_OK;
+    const size_t need = rsd_sbs_tree_workspace_bytes(B, W, L);
+    if (!ws || ws_bytes < need) return fail(RSD_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
+    if ((uintptr_t)ws % 256 != 0) return fail(RSD_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+    cudaStream_t s = (cudaStream_t)stream;
+
+    const size_t f4 = align_up((size_t)B * P * W * 4, 256), r4 = align_up((size_t)B * P * 4, 256), s4 = align_up((size_t)B * W * 4, 256);
+    char* w = (char*)ws;
+    int32_t* fin_token = (int32_t*)w;
+    float* fin_value = (float*)(w + f4);
+    float* fin_pert = (float*)(w + 2 * f4);
+    float* fin_lse = (float*)(w + 3 * f4);
+    int32_t* row_status = (int32_t*)(w + 3 * f4 + r4);
+    char* st0 = w + 3 * f4 + 2 * r4;
+    int32_t* level_status = (int32_t*)(st0 + 4 * s4);
+
+    // one scan over the parent rows of every level: row r of a sequence is flat node r
+    rsd::ScanArgs a;
+    memset(&a, 0, sizeof(a));
+    for (int r = 0; r < (int)P; ++r) { a.k_row[r] = (uint8_t)W; a.node_row[r] = r; }
+    a.data = draft->data; a.seq_stride = draft->seq_stride; a.row_stride = draft->row_stride;
+    a.R = (int)P; a.V = V; a.max_k = W;
+    a.seed_lo = (uint32_t)seed; a.seed_hi = (uint32_t)(seed >> 32); a.step = step; a.seq_base = seq_base;
+    a.subtract_lse = 0;
+    a.out_token = fin_token; a.out_perturbed = fin_pert; a.out_value = fin_value; a.out_lse = fin_lse;
+    a.status = status; a.row_status = row_status;
+    a.temp = temperature_of(draft); a.inv_temp = 1.0f / a.temp; a.raw_values = 1;
+    launch_scan(draft, !rows_are_logprob(draft), (int)(B * P), a, s);
+    if (int e = check_launch("rsd_sbs_draft_tree(scan)")) return e;
+
+    rsd::SbsChainArgs c;
+    memset(&c, 0, sizeof(c));
+    c.lvl.W = W; c.lvl.is_logprob = rows_are_logprob(draft); c.lvl.inv_temp = 1.0 / (double)temperature_of(draft);
+    c.lvl.fin_seq_stride = P * W; c.lvl.row_seq_stride = P; c.lvl.state_stride = W;
+    c.lvl.seed_lo = (uint32_t)seed; c.lvl.seed_hi = (uint32_t)(seed >> 32); c.lvl.step = step; c.lvl.seq_base = seq_base;
+    c.lvl.fin_token = fin_token; c.lvl.fin_value = fin_value; c.lvl.fin_pert = fin_pert; c.lvl.fin_lse = fin_lse;
+    c.lvl.row_status = row_status;
+    c.L = L; c.P = (int)P; c.B = B;
+    c.state_sum[0] = (float*)st0; c.state_gamma[0] = (float*)(st0 + s4);
+    c.state_sum[1] = (float*)(st0 + 2 * s4); c.state_gamma[1] = (float*)(st0 + 3 * s4);
+    c.node_token = node_token; c.node_parent = node_parent; c.node_stride = node_stride;
+    c.level_count = level_count; c.level_status = level_status; c.status = status;
+    c.sum_out = sum_logprob_out; c.gamma_out = trunc_gumbel_out;
+    const size_t smem = (size_t)W * W * (8 + 8 + 4) + (size_t)W * 4;
+    rsd::sbs_chain_kernel<<<B, rsd::kEpilogueThreads, smem, s>>>(c);
+    return check_launch("rsd_sbs_draft_tree(levels)");
 }
 
 }  // extern "C"

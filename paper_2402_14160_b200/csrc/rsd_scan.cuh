@@ -774,6 +774,9 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
 // ---------------------------------------------------------------------------------------------------------
 struct SbsEpilogueArgs {
     int n_par, W, is_logprob;
+    int64_t fin_seq_stride;    // elements between sequences in fin_token / fin_value / fin_pert (n_par * W for one level)
+    int64_t row_seq_stride;    // elements between sequences in fin_lse / row_status (n_par for one level)
+    int64_t state_stride;      // elements between sequences in sum_in / gamma_in (n_par for one level)
     double inv_temp;           // 1 / temperature of the parents' rows (1: none)
     int32_t first_parent_node;
     uint32_t seed_lo, seed_hi, step, seq_base;
@@ -796,13 +799,15 @@ struct SbsEpilogueArgs {
 
 constexpr int kEpilogueThreads = 128;
 
-static __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const SbsEpilogueArgs a) {
-    extern __shared__ double sm_d[];  // [F] phi~ then psi, [F] phi
+// One level for sequence b, by a block of kEpilogueThreads threads; sm_d: (n_par * W) * 20 + n_par * 4 bytes.
+__device__ __forceinline__ void sbs_epilogue_body(const SbsEpilogueArgs& a, const int b, double* sm_d) {
     const int F = a.n_par * a.W;
-    double* s_val = sm_d;
-    double* s_phi = sm_d + F;
+    double* s_val = sm_d;             // [F] phi~ then psi
+    double* s_phi = sm_d + F;         // [F] phi
     int* s_tok = (int*)(sm_d + 2 * F);
-    const int b = blockIdx.x, tid = threadIdx.x;
+    const int tid = threadIdx.x;
+    const int64_t fin_off = (int64_t)b * a.fin_seq_stride, row_off = (int64_t)b * a.row_seq_stride,
+                  state_off = (int64_t)b * a.state_stride;
     const RngKey key = {a.seed_lo, a.seed_hi, a.step, a.seq_base + (uint32_t)b};
     const double ninf = -__longlong_as_double(0x7FF0000000000000LL);
 
@@ -815,9 +820,9 @@ static __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(c
     __shared__ float s_L;
     if (tid == 0) s_L = kNegInf;
     for (int kp = tid; kp < a.n_par; kp += kEpilogueThreads) {
-        const float sg = a.sum_in ? a.sum_in[(int64_t)b * a.n_par + kp] : 0.0f;
-        const float gm = a.gamma_in ? a.gamma_in[(int64_t)b * a.n_par + kp] : 0.0f;
-        const bool delivers = a.fin_token[(int64_t)b * F + (int64_t)kp * a.W] >= 0 && sg > kNegInf && gm > kNegInf;
+        const float sg = a.sum_in ? a.sum_in[state_off + kp] : 0.0f;
+        const float gm = a.gamma_in ? a.gamma_in[state_off + kp] : 0.0f;
+        const bool delivers = a.fin_token[fin_off + (int64_t)kp * a.W] >= 0 && sg > kNegInf && gm > kNegInf;
         s_gam[kp] = delivers ? gm : kNegInf;
     }
     __syncthreads();
@@ -835,18 +840,18 @@ static __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(c
 
     for (int f = tid; f < F; f += kEpilogueThreads) {
         const int kpar = f / a.W;
-        int x = a.fin_token[(int64_t)b * F + f];
+        int x = a.fin_token[fin_off + f];
         // a parent slot that the level above left empty (its sum or truncated Gumbel is -inf) has no children
         // (s_gam is -inf exactly for the slots that deliver nothing)
         if (s_gam[kpar] == kNegInf) x = -1;
         if (x >= 0 && L > kNegInf && f != kpar * a.W) {
             // psi_f < L  <=>  exp(-phi~_f) - exp(-Z) > exp(-L) - exp(-Gamma_k), with Z - phi~_f = the gap d between
             // the parent's best and this finalist's fp32 perturbed values; margins cover the fp32 arithmetic
-            const float sg = a.sum_in ? a.sum_in[(int64_t)b * a.n_par + kpar] : 0.0f;
-            const float gm = a.gamma_in ? a.gamma_in[(int64_t)b * a.n_par + kpar] : 0.0f;
-            const float lse = a.is_logprob ? 0.0f : a.fin_lse[(int64_t)b * a.n_par + kpar];
-            const float u0 = a.fin_pert[(int64_t)b * F + (int64_t)kpar * a.W];
-            const float d_lo = (u0 - a.fin_pert[(int64_t)b * F + f]) - 1e-4f;
+            const float sg = a.sum_in ? a.sum_in[state_off + kpar] : 0.0f;
+            const float gm = a.gamma_in ? a.gamma_in[state_off + kpar] : 0.0f;
+            const float lse = a.is_logprob ? 0.0f : a.fin_lse[row_off + kpar];
+            const float u0 = a.fin_pert[fin_off + (int64_t)kpar * a.W];
+            const float d_lo = (u0 - a.fin_pert[fin_off + f]) - 1e-4f;
             if (d_lo > 0.0f) {
                 const float z = sg - lse + u0;
                 const float rhs = expf(-L + 1e-3f) - expf(-gm);
@@ -855,13 +860,13 @@ static __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(c
         }
         double phi = ninf, pert = ninf;
         if (x >= 0) {
-            const double sigma = a.sum_in ? (double)a.sum_in[(int64_t)b * a.n_par + kpar] : 0.0;
-            const double lse = a.is_logprob ? 0.0 : (double)a.fin_lse[(int64_t)b * a.n_par + kpar];
+            const double sigma = a.sum_in ? (double)a.sum_in[state_off + kpar] : 0.0;
+            const double lse = a.is_logprob ? 0.0 : (double)a.fin_lse[row_off + kpar];
             const uint32_t node = (uint32_t)(a.first_parent_node + kpar);
             const uint32_t word = coarse_word(key, node, (uint32_t)x >> 4);
             const double t_elem = (((uint32_t)x & 15u) != (word & 15u))
                                       ? neg_log_uniform_f64(fine_word(key, node, (uint32_t)x)) : 0.0;
-            phi = sigma + ((double)a.fin_value[(int64_t)b * F + f] * a.inv_temp - lse);
+            phi = sigma + ((double)a.fin_value[fin_off + f] * a.inv_temp - lse);
             pert = phi - log(neg_log_group_uniform_f64(word) * 0.0625 + t_elem);
         }
         s_tok[f] = x;
@@ -876,7 +881,7 @@ static __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(c
         const int kpar = f / a.W;
         double z = ninf;
         for (int i = 0; i < a.W; ++i) z = fmax(z, s_val[kpar * a.W + i]);
-        const double gamma = a.gamma_in ? (double)a.gamma_in[(int64_t)b * a.n_par + kpar] : 0.0;
+        const double gamma = a.gamma_in ? (double)a.gamma_in[state_off + kpar] : 0.0;
         const double pert = s_val[f];
         double psi = ninf;
         if (s_tok[f] >= 0) {
@@ -930,12 +935,71 @@ static __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(c
         a.gamma_out[o] = kNegInf;
     }
     int row_bits = 0;
-    for (int kp = tid; kp < a.n_par; kp += kEpilogueThreads) row_bits |= a.row_status[(int64_t)b * a.n_par + kp];
+    for (int kp = tid; kp < a.n_par; kp += kEpilogueThreads) row_bits |= a.row_status[row_off + kp];
     row_bits = __syncthreads_or(row_bits);
     if (tid == 0) {
         a.status[b] = (row_bits & 1) | (cnt < a.W ? 2 : 0);  // RSD_ST_NAN_INPUT, RSD_ST_FEWER_THAN_K
         a.out_count[b] = cnt;
     }
+}
+
+
+static __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(const SbsEpilogueArgs a) {
+    extern __shared__ double sm_d[];
+    sbs_epilogue_body(a, blockIdx.x, sm_d);
+}
+
+// All L levels of one Stochastic Beam Search tree (Algorithm 8's level loop around Algorithm 9) for rows that exist
+// before drafting starts: the parent rows of every level were scanned in one launch (row r of a sequence is flat node
+// r: the root, then W slots per level), and this kernel runs the levels' epilogues in order, one block per sequence.
+// The sequence log-probabilities and truncated Gumbels (Eqs. 10-12) travel from level to level through two [B][W]
+// arrays used in turn; level l writes the tokens and parents of flat nodes 1 + l W .. (l + 1) W.
+struct SbsChainArgs {
+    SbsEpilogueArgs lvl;        // level-independent fields; the per-level ones are filled in by the kernel
+    int L, P;                   // levels; parent rows per sequence, 1 + (L - 1) W
+    int B;
+    float* state_sum[2];        // [B][W] each
+    float* state_gamma[2];
+    int32_t* node_token;        // [B][node_stride]
+    int32_t* node_parent;
+    int64_t node_stride;
+    int32_t* level_count;       // [L][B]
+    int32_t* level_status;      // [L][B]
+    int32_t* status;            // [B]: OR over the levels
+    float* sum_out;             // [B][W] of the last level, or null
+    float* gamma_out;
+};
+
+static __global__ void __launch_bounds__(kEpilogueThreads) sbs_chain_kernel(const SbsChainArgs c) {
+    extern __shared__ double sm_d[];
+    const int b = blockIdx.x, W = c.lvl.W;
+    int st = 0;
+    for (int l = 0; l < c.L; ++l) {
+        SbsEpilogueArgs a = c.lvl;
+        const int first = l == 0 ? 0 : 1 + (l - 1) * W;     // flat node of the level's parent slot 0
+        a.n_par = l == 0 ? 1 : W;
+        a.first_parent_node = first;
+        a.fin_token = c.lvl.fin_token + (int64_t)first * W;
+        a.fin_value = c.lvl.fin_value + (int64_t)first * W;
+        a.fin_pert = c.lvl.fin_pert + (int64_t)first * W;
+        a.fin_lse = c.lvl.fin_lse + first;
+        a.row_status = c.lvl.row_status + first;
+        a.sum_in = l == 0 ? nullptr : c.state_sum[(l + 1) & 1];
+        a.gamma_in = l == 0 ? nullptr : c.state_gamma[(l + 1) & 1];
+        const bool last = l == c.L - 1;
+        a.sum_out = (last && c.sum_out) ? c.sum_out : c.state_sum[l & 1];
+        a.gamma_out = (last && c.gamma_out) ? c.gamma_out : c.state_gamma[l & 1];
+        a.out_token = c.node_token + 1 + (int64_t)l * W;
+        a.out_parent = c.node_parent + 1 + (int64_t)l * W;
+        a.out_stride = c.node_stride;
+        a.parent_base = first;
+        a.out_count = c.level_count + (int64_t)l * c.B;
+        a.status = c.level_status + (int64_t)l * c.B;
+        sbs_epilogue_body(a, b, sm_d);
+        __syncthreads();   // the level's outputs are the next level's inputs
+        if (threadIdx.x == 0) st |= a.status[b];
+    }
+    if (threadIdx.x == 0) c.status[b] = st;
 }
 
 }  // namespace rsd

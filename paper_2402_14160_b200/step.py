@@ -55,10 +55,15 @@ class RsdCStep:
 
 
 class RsdSStep:
-    """RSD with Stochastic Beam Search of width W and depth L for a batch of B sequences."""
+    """RSD with Stochastic Beam Search of width W and depth L for a batch of B sequences.
 
-    def __init__(self, B: int, V: int, W: int, L: int, draft_is_logprob: bool = False, device="cuda"):
+    rows_ready=True: the draft rows of every level exist before drafting starts (rows attached to tree slots), so the
+    whole tree is drafted by rsd_sbs_draft_tree in two launches; otherwise one rsd_sbs_step call per level."""
+
+    def __init__(self, B: int, V: int, W: int, L: int, draft_is_logprob: bool = False, device="cuda",
+                 rows_ready: bool = True):
         self.B, self.V, self.W, self.L, self.is_logprob = B, V, W, L, draft_is_logprob
+        self.rows_ready = rows_ready
         self.n_nodes = 1 + W * L
         self.P = 1 + W * (L - 1)
         self.parent = torch.full((B, self.n_nodes), -1, dtype=torch.int32, device=device)
@@ -67,15 +72,30 @@ class RsdSStep:
                            trunc_gumbel=torch.empty((B, W), dtype=torch.float32, device=device)) for _ in range(2)]
         self.count = torch.empty((L, B), dtype=torch.int32, device=device)
         self.status = torch.empty((L, B), dtype=torch.int32, device=device)
-        self.workspace = torch.empty((api.rsd_sbs_workspace_bytes(B, W, W),), dtype=torch.uint8, device=device)
+        self.workspace = torch.empty((max(api.rsd_sbs_workspace_bytes(B, W, W), api.rsd_sbs_tree_workspace_bytes(B, W, L)),),
+                                     dtype=torch.uint8, device=device)
+        self.tree_out = dict(sum_logprob=self.state[0]["sum_logprob"], trunc_gumbel=self.state[0]["trunc_gumbel"],
+                             count=self.count, status=torch.empty((B,), dtype=torch.int32, device=device))
         self.verify_out = None
-        self.kernel_launches = 2 * L + 1  # per level one scan and one epilogue, then one walk
+        # one scan over all rows, one launch for the levels, one walk; or per level one scan and one epilogue
+        self.kernel_launches = 3 if rows_ready else 2 * L + 1
 
     def level_slice(self, l: int):
         return slice(1 + l * self.W, 1 + (l + 1) * self.W)
 
+    def draft_tree(self, draft: torch.Tensor, seed: int, step: int, seq_base: int = 0):
+        """All levels at once (rows_ready)."""
+        return api.rsd_sbs_draft_tree(draft, self.W, self.L, seed, step, self.token, self.parent,
+                                      is_logprob=self.is_logprob, seq_base=seq_base, workspace=self.workspace,
+                                      out=self.tree_out)
+
     def run(self, draft: torch.Tensor, target: torch.Tensor, seed: int, step: int, seq_base: int = 0):
         W = self.W
+        if self.rows_ready:
+            self.draft_tree(draft, seed, step, seq_base)
+            self.verify_out = api.rsd_verify_tree(draft, target, self.parent, self.token, self.L, seed, step,
+                                                  seq_base=seq_base, out=self.verify_out)
+            return self.verify_out
         for l in range(self.L):
             first = 0 if l == 0 else 1 + (l - 1) * W
             n_par = 1 if l == 0 else W
@@ -91,9 +111,10 @@ class RsdSStep:
         return self.verify_out
 
 
-def make_step(w, batch=None, device="cuda"):
+def make_step(w, batch=None, device="cuda", rows_ready=True):
     """Step object for a workloads.Workload description."""
     B = w.batch if batch is None else batch
     if w.mode == "rsd_c":
         return RsdCStep(B, w.vocab, w.branching, device=device)
-    return RsdSStep(B, w.vocab, w.beam_width, w.depth, draft_is_logprob=w.draft_is_logprob, device=device)
+    return RsdSStep(B, w.vocab, w.beam_width, w.depth, draft_is_logprob=w.draft_is_logprob, device=device,
+                    rows_ready=rows_ready)

@@ -160,6 +160,58 @@ def test_sbs_levels_match_oracle(rsd, dtype, V, W, L, is_logprob):
     assert all(np.all(g["count"] == W) for g in g_levels)
 
 
+@pytest.mark.parametrize("dtype,V,W,L,is_logprob", [("f32", 1000, 3, 3, False), ("bf16", 4099, 8, 4, False),
+                                                    ("f32", 515, 5, 1, True), ("bf16", 32000, 6, 5, False)])
+def test_sbs_draft_tree_is_the_chain_of_level_calls(rsd, dtype, V, W, L, is_logprob):
+    # rsd_sbs_draft_tree (all levels from rows that exist up front) must give what L rsd_sbs_step calls give, bit for
+    # bit, and through them what the oracle's level-by-level chain gives
+    B = 7
+    P = 1 + (L - 1) * W
+    draft = _rows((B, P, V), dtype, 2.5, 700 + V)
+    if is_logprob:
+        draft = torch.log_softmax(draft.float(), -1).to(draft.dtype)
+    t, g_levels, o_levels, skip = _sbs_chain(rsd, draft, W, L, seed=23, step=6, is_logprob=is_logprob, seq_base=11)
+    t.check()
+    parent, token = _sbs_tree(g_levels, W)
+    node_token = torch.full((B, 3 + L * W), -7, dtype=torch.int32, device="cuda")      # wider than needed: stride kept
+    node_parent = torch.full((B, 3 + L * W), -7, dtype=torch.int32, device="cuda")
+    out = _np(rsd.rsd_sbs_draft_tree(draft, W, L, 23, 6, node_token, node_parent, is_logprob=is_logprob, seq_base=11))
+    torch.cuda.synchronize()
+    nt, npar = node_token.cpu().numpy(), node_parent.cpu().numpy()
+    assert np.array_equal(nt[:, 1:1 + L * W], token[:, 1:]) and np.array_equal(npar[:, 1:1 + L * W], parent[:, 1:])
+    assert np.all(nt[:, 0] == -7) and np.all(nt[:, 1 + L * W:] == -7) and np.all(npar[:, 1 + L * W:] == -7)   # untouched
+    assert np.array_equal(out["sum_logprob"], g_levels[-1]["sum_logprob"])
+    assert np.array_equal(out["trunc_gumbel"], g_levels[-1]["trunc_gumbel"])
+    assert np.array_equal(out["count"], np.stack([g["count"] for g in g_levels]))
+    assert np.array_equal(out["status"], np.bitwise_or.reduce(np.stack([g["status"] for g in g_levels]), axis=0))
+
+
+def test_sbs_draft_tree_with_underfull_levels_and_bad_arguments(rsd):
+    W, L, V = 4, 3, 64
+    draft = _rows((3, 1 + (L - 1) * W, V), "f32", 2.0, 31)
+    draft[0, 0, :] = float("-inf")
+    draft[0, 0, [5, 9]] = 0.25                                   # the root of sequence 0 offers two tokens only
+    node_token = torch.full((3, 1 + L * W), -1, dtype=torch.int32, device="cuda")
+    node_parent = torch.full((3, 1 + L * W), -1, dtype=torch.int32, device="cuda")
+    out = _np(rsd.rsd_sbs_draft_tree(draft, W, L, 2, 0, node_token, node_parent))
+    host = workloads.as_oracle_rows(draft)
+    prev = None
+    for l in range(L):
+        first = 0 if l == 0 else 1 + (l - 1) * W
+        o = oracle.sbs_step(host[:, first:first + (1 if l == 0 else W)], W, first, None if l == 0 else prev["sum_logprob"],
+                            None if l == 0 else prev["trunc_gumbel"], 2, 0)
+        sl = slice(1 + l * W, 1 + (l + 1) * W)
+        assert np.array_equal(node_token[:, sl].cpu().numpy(), o["token"]), l
+        assert np.array_equal(node_parent[:, sl].cpu().numpy(), np.where(o["parent"] >= 0, first + o["parent"], -1)), l
+        assert np.array_equal(out["count"][l], o["count"])
+        prev = o
+    assert out["count"][0, 0] == 2 and out["status"][0] & rsd.ST_FEWER_THAN_K and out["status"][1] == 0
+    with pytest.raises(rsd.RsdError, match="rows per sequence"):
+        rsd.rsd_sbs_draft_tree(draft[:, :5], W, L, 2, 0, node_token, node_parent)
+    with pytest.raises(rsd.RsdError, match="node_stride"):
+        rsd.rsd_sbs_draft_tree(draft, W, L, 2, 0, node_token[:, :6].contiguous(), node_parent[:, :6].contiguous())
+
+
 def test_sbs_drops_minus_infinity_candidates(rsd):
     rows = torch.full((1, 2, 64), float("-inf"), device="cuda")
     rows[0, 0, [2, 9]] = torch.tensor([0.0, 1.0], device="cuda")

@@ -21,6 +21,8 @@ def test_library_builds_and_exports_every_declared_symbol():
     assert lib.rsd_rng_layout() == 3
     lib.rsd_sbs_workspace_bytes.restype = ctypes.c_size_t
     assert lib.rsd_sbs_workspace_bytes(4, 8, 8) >= 4 * 8 * 8 * 8 + 4 * 8 * 4
+    lib.rsd_sbs_tree_workspace_bytes.restype = ctypes.c_size_t
+    assert lib.rsd_sbs_tree_workspace_bytes(4, 8, 8) >= 4 * 57 * 8 * 12 + 4 * 57 * 8
 
 
 def test_argument_validation_needs_no_gpu():
