@@ -117,6 +117,12 @@ def rows_of(t: torch.Tensor, is_logprob: bool = False, temperature: float = 1.0)
     raise RsdError("rows must be [B, R, V] or [B, V]")
 
 
+def _new(shape, dtype, device):
+    """Every output tensor this package allocates comes from here (one place, so that the tests can surround each of
+    them with guard words and check that no kernel writes outside its outputs)."""
+    return torch.empty(shape, dtype=dtype, device=device)
+
+
 def _host_i32(values: Sequence[int]):
     arr = (C.c_int32 * len(values))(*[int(v) for v in values])
     return arr
@@ -135,10 +141,10 @@ def rsd_gumbel_topk_draft(draft: torch.Tensor, k_per_row: Sequence[int], rng_nod
     max_k = int(max_k or max(k_per_row))
     dev = draft.device
     if out is None:
-        out = dict(token=torch.empty((B, R, max_k), dtype=torch.int32, device=dev),
-                   status=torch.empty((B,), dtype=torch.int32, device=dev),
-                   perturbed=torch.empty((B, R, max_k), dtype=torch.float32, device=dev) if want_values else None,
-                   logprob=torch.empty((B, R, max_k), dtype=torch.float32, device=dev) if want_values else None)
+        out = dict(token=_new((B, R, max_k), torch.int32, dev),
+                   status=_new((B,), torch.int32, dev),
+                   perturbed=_new((B, R, max_k), torch.float32, dev) if want_values else None,
+                   logprob=_new((B, R, max_k), torch.float32, dev) if want_values else None)
     rows = rows_of(draft, is_logprob, temperature)
     if node_token is not None and (node_token.dtype != torch.int32 or not node_token.is_contiguous()):
         raise RsdError("node_token must be contiguous int32")
@@ -173,14 +179,14 @@ def rsd_sbs_step(draft_level: torch.Tensor, W: int, first_parent_node: int, sum_
     dev = draft_level.device
     need = rsd_sbs_workspace_bytes(B, n_par, W)
     if workspace is None:
-        workspace = torch.empty((need,), dtype=torch.uint8, device=dev)
+        workspace = _new((need,), torch.uint8, dev)
     if out is None:
-        out = dict(token=torch.empty((B, W), dtype=torch.int32, device=dev),
-                   parent=torch.empty((B, W), dtype=torch.int32, device=dev),
-                   sum_logprob=torch.empty((B, W), dtype=torch.float32, device=dev),
-                   trunc_gumbel=torch.empty((B, W), dtype=torch.float32, device=dev),
-                   count=torch.empty((B,), dtype=torch.int32, device=dev),
-                   status=torch.empty((B,), dtype=torch.int32, device=dev))
+        out = dict(token=_new((B, W), torch.int32, dev),
+                   parent=_new((B, W), torch.int32, dev),
+                   sum_logprob=_new((B, W), torch.float32, dev),
+                   trunc_gumbel=_new((B, W), torch.float32, dev),
+                   count=_new((B,), torch.int32, dev),
+                   status=_new((B,), torch.int32, dev))
     rows = rows_of(draft_level, is_logprob, temperature)
     if out["token"].stride(0) != out["parent"].stride(0) or out["token"].stride(1) != 1 or out["parent"].stride(1) != 1:
         raise RsdError("out token/parent must share a row stride and be dense along the picks")
@@ -208,12 +214,12 @@ def rsd_sbs_draft_tree(draft: torch.Tensor, W: int, L: int, seed: int, step: int
     if node_token.stride(0) != node_parent.stride(0) or node_token.stride(1) != 1 or node_parent.stride(1) != 1:
         raise RsdError("node_token / node_parent must share a row stride and be dense along the nodes")
     if workspace is None:
-        workspace = torch.empty((rsd_sbs_tree_workspace_bytes(B, W, L),), dtype=torch.uint8, device=dev)
+        workspace = _new((rsd_sbs_tree_workspace_bytes(B, W, L),), torch.uint8, dev)
     if out is None:
-        out = dict(sum_logprob=torch.empty((B, W), dtype=torch.float32, device=dev),
-                   trunc_gumbel=torch.empty((B, W), dtype=torch.float32, device=dev),
-                   count=torch.empty((L, B), dtype=torch.int32, device=dev),
-                   status=torch.empty((B,), dtype=torch.int32, device=dev))
+        out = dict(sum_logprob=_new((B, W), torch.float32, dev),
+                   trunc_gumbel=_new((B, W), torch.float32, dev),
+                   count=_new((L, B), torch.int32, dev),
+                   status=_new((B,), torch.int32, dev))
     rows = rows_of(draft, is_logprob, temperature)
     _check(lib().rsd_sbs_draft_tree(C.byref(rows), B, V, W, L, seed, step, seq_base, _ptr(node_token),
                                     _ptr(node_parent), node_token.stride(0), _ptr(out["sum_logprob"]),
@@ -263,13 +269,13 @@ def rsd_verify_tree(draft: torch.Tensor, target: torch.Tensor, parent: torch.Ten
     if not (parent.is_contiguous() and token.is_contiguous()):
         raise RsdError("parent and token must be contiguous")
     if out is None:
-        out = dict(accepted_len=torch.empty((B,), dtype=torch.int32, device=dev),
-                   accepted_node=torch.empty((B, max(L, 1)), dtype=torch.int32, device=dev)[:, :L],
-                   accepted_token=torch.empty((B, max(L, 1)), dtype=torch.int32, device=dev)[:, :L],
-                   last_token=torch.empty((B,), dtype=torch.int32, device=dev),
-                   stop_reason=torch.empty((B,), dtype=torch.int32, device=dev),
-                   status=torch.empty((B,), dtype=torch.int32, device=dev))
-        out["theta"] = torch.empty((B, n_nodes), dtype=torch.float32, device=dev) if want_theta else None
+        out = dict(accepted_len=_new((B,), torch.int32, dev),
+                   accepted_node=_new((B, max(L, 1)), torch.int32, dev)[:, :L],
+                   accepted_token=_new((B, max(L, 1)), torch.int32, dev)[:, :L],
+                   last_token=_new((B,), torch.int32, dev),
+                   stop_reason=_new((B,), torch.int32, dev),
+                   status=_new((B,), torch.int32, dev))
+        out["theta"] = _new((B, n_nodes), torch.float32, dev) if want_theta else None
     tree = RsdTree(L, n_nodes, parent.data_ptr(), token.data_ptr(), 1 if parent.dim() == 1 else 0)
     d, t = rows_of(draft, False, draft_temperature), rows_of(target, False, target_temperature)
     outs = (_ptr(out["accepted_len"]), _ptr(out["accepted_node"]), _ptr(out["accepted_token"]),
@@ -297,9 +303,9 @@ def rsd_resample_residual(draft_row: Optional[torch.Tensor], target_row: torch.T
     """draft_row/target_row [B, V]; rejected [B, max_k] int32 (-1 padded) or None; rng_node [B] int32."""
     B, V = target_row.shape
     dev = target_row.device
-    token = torch.empty((B,), dtype=torch.int32, device=dev)
-    status = torch.empty((B,), dtype=torch.int32, device=dev)
-    residual = torch.empty((B, V), dtype=torch.float32, device=dev) if want_residual else None
+    token = _new((B,), torch.int32, dev)
+    status = _new((B,), torch.int32, dev)
+    residual = _new((B, V), torch.float32, dev) if want_residual else None
     t = rows_of(target_row, False, target_temperature)
     d = rows_of(draft_row, False, draft_temperature) if draft_row is not None else t
     max_k = 0 if rejected is None else rejected.shape[1]

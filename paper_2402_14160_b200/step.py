@@ -39,9 +39,9 @@ class RsdCStep:
         self.rng_node = list(range(self.P))
         self.max_k = max(k)
         self.parent = torch.tensor(parent, dtype=torch.int32, device=device)
-        self.token = torch.full((B, self.n_nodes), -1, dtype=torch.int32, device=device)
-        self.draft_out = dict(token=torch.empty((B, self.P, self.max_k), dtype=torch.int32, device=device),
-                              status=torch.empty((B,), dtype=torch.int32, device=device), perturbed=None, logprob=None)
+        self.token = api._new((B, self.n_nodes), torch.int32, device).fill_(-1)
+        self.draft_out = dict(token=api._new((B, self.P, self.max_k), torch.int32, device),
+                              status=api._new((B,), torch.int32, device), perturbed=None, logprob=None)
         self.verify_out = None
         self.kernel_launches = 2  # one scan, one walk
 
@@ -66,16 +66,16 @@ class RsdSStep:
         self.rows_ready = rows_ready
         self.n_nodes = 1 + W * L
         self.P = 1 + W * (L - 1)
-        self.parent = torch.full((B, self.n_nodes), -1, dtype=torch.int32, device=device)
-        self.token = torch.full((B, self.n_nodes), -1, dtype=torch.int32, device=device)
-        self.state = [dict(sum_logprob=torch.empty((B, W), dtype=torch.float32, device=device),
-                           trunc_gumbel=torch.empty((B, W), dtype=torch.float32, device=device)) for _ in range(2)]
-        self.count = torch.empty((L, B), dtype=torch.int32, device=device)
-        self.status = torch.empty((L, B), dtype=torch.int32, device=device)
-        self.workspace = torch.empty((max(api.rsd_sbs_workspace_bytes(B, W, W), api.rsd_sbs_tree_workspace_bytes(B, W, L)),),
-                                     dtype=torch.uint8, device=device)
+        self.parent = api._new((B, self.n_nodes), torch.int32, device).fill_(-1)
+        self.token = api._new((B, self.n_nodes), torch.int32, device).fill_(-1)
+        self.state = [dict(sum_logprob=api._new((B, W), torch.float32, device),
+                           trunc_gumbel=api._new((B, W), torch.float32, device)) for _ in range(2)]
+        self.count = api._new((L, B), torch.int32, device)
+        self.status = api._new((L, B), torch.int32, device)
+        self.workspace = api._new((max(api.rsd_sbs_workspace_bytes(B, W, W), api.rsd_sbs_tree_workspace_bytes(B, W, L)),),
+                                  torch.uint8, device)
         self.tree_out = dict(sum_logprob=self.state[0]["sum_logprob"], trunc_gumbel=self.state[0]["trunc_gumbel"],
-                             count=self.count, status=torch.empty((B,), dtype=torch.int32, device=device))
+                             count=self.count, status=api._new((B,), torch.int32, device))
         self.verify_out = None
         # one scan over all rows, one launch for the levels, one walk; or per level one scan and one epilogue
         self.kernel_launches = 3 if rows_ready else 2 * L + 1

@@ -1,5 +1,6 @@
 """The five benchmark workloads at full size: one draft + verify step on the GPU in the launch configuration the
-benchmark times, compared with the oracle on every sequence (small workloads) or on sampled sequences (large ones)."""
+benchmark times, compared with the oracle on every sequence (the large workloads in blocks of 128 sequences, which
+bounds the host memory the oracle's copies of the rows take)."""
 import os
 
 import numpy as np
@@ -78,11 +79,11 @@ def _compare_block(t, w, stepper, gpu_verify, ora, lo, hi):
     return bad
 
 
-def _run_config(cid, steps, blocks):
+def _run_config(cid, steps, blocks, rows_ready=True):
     import paper_2402_14160_b200 as rsd
     from paper_2402_14160_b200 import step as rsd_step
     w = workloads.WORKLOADS[cid]
-    stepper = rsd_step.make_step(w)
+    stepper = rsd_step.make_step(w, rows_ready=rows_ready)
     t = Tally()
     acc_len = []
     for s in range(steps):
@@ -118,9 +119,15 @@ def test_workload_3_rsd_s():
     _run_config(3, 1, [(0, 32)])
 
 
+def test_workload_3_rsd_s_level_by_level():
+    _run_config(3, 1, [(0, 32)], rows_ready=False)      # one rsd_sbs_step call per level instead of rsd_sbs_draft_tree
+
+
 def test_workload_4_opt_vocab_rsd_c():
-    _run_config(4, 1, [(0, 8), (248, 256)])
+    t = _run_config(4, 1, [(lo, lo + 128) for lo in range(0, 256, 128)])
+    assert t.decisions > 256 * 60
 
 
 def test_workload_5_serving_rsd_s():
-    _run_config(5, 1, [(0, 8), (1016, 1024)])
+    t = _run_config(5, 1, [(lo, lo + 128) for lo in range(0, 1024, 128)])
+    assert t.decisions > 1024 * 64

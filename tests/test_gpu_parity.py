@@ -338,6 +338,93 @@ def test_verify_tree_special_trees(rsd):
     assert np.array_equal(g["last_token"], o["last_token"])
 
 
+@pytest.mark.parametrize("dtype,V,branching,aligned", [("bf16", 64, (20, 20), True), ("f32", 48, (40,), True),
+                                                       ("f32", 50, (20, 20), False), ("bf16", 1000, (40, 2), True),
+                                                       ("f32", 51, (40,), False)])
+def test_verify_tree_wide_and_large_trees(rsd, dtype, V, branching, aligned):
+    # b = (20, 20): 421 nodes, more than the walk kernels keep in shared memory, so the children are searched in
+    # global memory; b = (40, ...): a node with 40 children, more rejections than a warp has lanes (the row values
+    # of the later children are no longer fetched ahead) and, with the draft far from the target, more removed
+    # tokens than the 32 the register-fed walk remembers.  aligned=False: rows at odd offsets (register-fed walk).
+    B = 24
+    L = len(branching)
+    parent = workloads.rsdc_parent_array(branching)
+    n_nodes = len(parent)
+    k, nodes = workloads.rsdc_rows(branching)
+    P = len(k)
+    pad = 0 if aligned else 3
+    base = _rows((B, n_nodes, V + pad), "f32", 1.0, 800 + V)
+    tgt = base - 2.5 * _rows((B, n_nodes, V + pad), "f32", 1.0, 801 + V).abs() * (base > 0.5)   # the draft's favourites are unlikely
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    draft = base[:, :P].to(tdt).contiguous()[:, :, pad:]
+    target = tgt.to(tdt).contiguous()[:, :, pad:]
+    o_draft = oracle.gumbel_topk(workloads.as_oracle_rows(draft.contiguous()), k, nodes, 4, 3)
+    token = workloads.rsdc_tokens_from_rows(branching, o_draft["token"])
+    par_t, tok_t = torch.from_numpy(parent).cuda(), torch.from_numpy(token).cuda()
+    g = _np(rsd.rsd_verify_tree(draft, target, par_t, tok_t, L, 4, 3, want_theta=True))
+    o = oracle.verify_tree(workloads.as_oracle_rows(draft.contiguous()), workloads.as_oracle_rows(target.contiguous()),
+                           parent, token, L, 4, 3)
+    t = Tally()
+    compare_verify(t, g, o, parent)
+    t.check()
+    assert np.array_equal(g["status"], o["status"])
+    tested = (~np.isnan(o["theta"])).sum(axis=1)
+    assert tested.max() >= branching[0] // 2                       # some walk went through many children of a node
+
+
+def test_verify_tree_repeated_sibling_tokens(rsd):
+    # Two children of a node carry the same token (a caller's tree; Gumbel-Top-k never drafts one): once the first is
+    # rejected its draft mass is gone (Eq. 1), so the second is a child the draft could not have produced: threshold 0
+    # (its residual mass is 0 too) and RSD_ST_ZERO_DRAFT_PROB, exactly as the oracle reports it.
+    rng = np.random.default_rng(8)
+    B, V = 16, 128
+    parent = np.array([-1, 0, 0, 0, 0], np.int32)
+    draft_h = rng.normal(0, 1, (B, 1, V)).astype(np.float32)
+    target_h = rng.normal(0, 1, (B, 5, V)).astype(np.float32)
+    token = np.tile(np.array([[-1, 5, 9, 5, 11]], np.int32), (B, 1))
+    target_h[:, 0, 5] -= 6.0                                       # token 5 is rejected almost surely
+    target_h[:, 0, 9] -= 6.0
+    for dtype in (torch.float32, torch.bfloat16):
+        draft, target = torch.from_numpy(draft_h).to(dtype).cuda(), torch.from_numpy(target_h).to(dtype).cuda()
+        g, o = _verify_both(rsd, draft, target, parent, token, 1, 31, 2)
+        t = Tally()
+        compare_verify(t, g, o, parent)
+        t.check()
+        assert np.array_equal(g["status"], o["status"])
+        reached = ~np.isnan(o["theta"][:, 3])
+        assert reached.sum() >= B // 2 and np.all(o["status"][reached] & rsd.ST_ZERO_DRAFT_PROB)
+        assert np.all(g["theta"][reached, 3] == 0.0)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_verify_tree_rows_far_from_zero_and_nan_logits(rsd, dtype):
+    # The copy-engine walk takes its first pass relative to a reference of 0: rows shifted by +-120 (sums over- or
+    # underflow), rows of which only one far-away entry is finite, and rows with NaN logits make it fall back on the
+    # rows' maxima and on its cleaning passes.
+    B, V, branching = 20, 4096 + 40, (3, 2)
+    parent = workloads.rsdc_parent_array(branching)
+    k, nodes = workloads.rsdc_rows(branching)
+    base = _rows((B, len(parent), V), "f32", 2.0, 61)
+    tgt = base + _rows((B, len(parent), V), "f32", 1.0, 62)
+    shift = torch.tensor([0.0, 120.0, -120.0, 300.0, -90.0] * 4, device="cuda").view(B, 1, 1)
+    base, tgt = base + shift, tgt - shift
+    base[5, 1, 100:] = float("-inf")                               # a draft row with 100 finite entries
+    tgt[6, 0, :] = float("-inf")
+    tgt[6, 0, 77] = -250.0                                         # a target row with one finite, far-away entry
+    tgt[7, 0, 1000] = float("nan")
+    base[8, 0, 2000] = float("nan")
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    draft, target = base[:, :len(k)].to(tdt).contiguous(), tgt.to(tdt).contiguous()
+    o_draft = oracle.gumbel_topk(workloads.as_oracle_rows(draft), k, nodes, 6, 0)
+    token = workloads.rsdc_tokens_from_rows(branching, o_draft["token"])
+    g, o = _verify_both(rsd, draft, target, parent, token, 2, 6, 0)
+    t = Tally()
+    compare_verify(t, g, o, parent)
+    t.check()
+    assert np.array_equal(g["status"], o["status"])
+    assert o["status"][7] & rsd.ST_NAN_INPUT and o["status"][8] & rsd.ST_NAN_INPUT
+
+
 def test_verify_tree_on_stochastic_beam_trees(rsd):
     w = workloads.scaled(workloads.WORKLOADS[3], batch=8, vocab=4000)
     draft, target = workloads.make_logits(w, step=0, device="cuda")
