@@ -353,8 +353,8 @@ def test_verify_tree_wide_and_large_trees(rsd, dtype, V, branching, aligned):
     k, nodes = workloads.rsdc_rows(branching)
     P = len(k)
     pad = 0 if aligned else 3
-    base = _rows((B, n_nodes, V + pad), "f32", 1.0, 800 + V)
-    tgt = base - 2.5 * _rows((B, n_nodes, V + pad), "f32", 1.0, 801 + V).abs() * (base > 0.5)   # the draft's favourites are unlikely
+    base = _rows((B, n_nodes, V + pad), "f32", 1.5, 800 + V)
+    tgt = -1.5 * base + _rows((B, n_nodes, V + pad), "f32", 0.5, 801 + V)     # what the draft likes the target does not
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     draft = base[:, :P].to(tdt).contiguous()[:, :, pad:]
     target = tgt.to(tdt).contiguous()[:, :, pad:]
