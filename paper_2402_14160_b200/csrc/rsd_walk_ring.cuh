@@ -3,8 +3,8 @@
 //
 // One block walks one sequence and reads only the rows of visited nodes.  The chain of residuals is carried in
 // closed form (see rsd_verify.cuh), so every pass is a read-only sweep over the node's target and draft rows: the
-// first pass gives both soft-max normalisers, each rejected child costs one more pass (served by L2, the rows were
-// just read), the last token is drawn from the tile sums of the last pass.
+// first pass gives both soft-max normalisers, each rejected child costs one more pass, the last token is drawn from
+// the tile sums of the last pass.
 //
 // A block has eight working warps and one control warp.  The control warp alone walks the tree: it takes every
 // decision (thresholds, acceptance tests, the chain's scalars, the last draw), tells the working warps which pass to
@@ -14,6 +14,11 @@
 // a register for it, the scalar part of the walk is executed once instead of by every warp, and three blocks share an
 // SM: while one walk waits for a decision or for its next node's rows, the other two keep the SM's special-function
 // unit and its memory pipe busy.
+// Chunk c of a row lives in slot c mod 4, and successive passes over one node run in opposite directions: a pass
+// ends with the last four chunks it read in the ring, the next pass starts with exactly those (no copy, no wait) and
+// fetches the others behind them, so half of a 32000-entry row pair is read from L2 again per rejection, not all.
+// Whatever the next decision needs and does not depend on the running pass (the child's uniform, its row values,
+// the scalars of Eq. 2) is prepared by the control warp while the pass runs.
 // Every wait on an mbarrier is bounded (about a second); a wait that runs out abandons the walk with RSD_ST_TIMEOUT.
 //
 // Used for rows whose base and strides are multiples of 16 bytes, recursive rejection sampling with the inverse-CDF
@@ -29,7 +34,7 @@ constexpr int kThreads = (kWorkWarps + 1) * 32;   // the last warp feeds the rin
 constexpr int kSlots = 4;                         // power of two
 constexpr int kRowChunkBytes = 8192;              // bytes of one row per slot (a slot holds a target and a draft chunk)
 constexpr int kTileElems = 512;                   // one warp-wide step: 16 elements per lane
-constexpr int kMaxChildren = 64;                  // children of a node whose row values are fetched ahead
+constexpr int kMaxRingChunks = 64;                // chunks per row the ring's bookkeeping covers (one bit each)
 constexpr int kMaxRemovedRing = 64;               // rejected tokens remembered per node (to recognise a repeated sibling)
 constexpr float kSumFloor = 8.673617379884035e-19f;   // 2^-60: a normaliser below this has lost its small terms to underflow
 constexpr long long kWaitCycles = 1ll << 31;      // about a second: a copy that has not landed by then never will
@@ -43,6 +48,8 @@ struct PassCmd {
     float kq, kp;        // log2(e) / temperature of the target and draft rows
     float cq, cp;        // reference * k: exponentials are 2^(value * k - c)
     float a_hi, a_lo;    // coefficient of the residual pass, as a two-float sum
+    int backward;        // 1: the pass takes the chunks from the last to the first
+    unsigned long long parity;   // bit c: phase parity of slot c mod kSlots' "full" barrier that holds chunk c
 };
 
 struct RingSmem {
@@ -149,67 +156,116 @@ struct Ring {
     RingSmem& sm;
     unsigned char* slots;      // [kSlots][2][kRowChunkBytes]: target chunk, then draft chunk
     int V, n_chunks, n_tiles;
-    uint32_t g0;               // chunks asked for before the current pass (all passes of the block)
+    // control warp only (identical on its lanes): the state of the ring as bit sets, so that a pass is planned
+    // without a loop
+    unsigned long long resident;   // chunks of the current node that sit in their slots
+    unsigned fill_par;             // bit s: parity of slot s' latest "full" phase (1 before the first copy)
+    unsigned round_par;            // bit s: parity of slot s' latest "empty" phase (1 before the first use)
+    unsigned round_used;           // bit s: the slot was given to the working warps at least once
+    int backward;                  // direction of the next pass over the current node
 
     static constexpr int kElem = (int)sizeof(T);
     static constexpr int kChunkElems = kRowChunkBytes / kElem;
     static constexpr int kTPC = kChunkElems / kTileElems;   // tiles per chunk: 8 (2-byte elements) or 4
+    static constexpr unsigned long long kEveryFourth = 0x1111111111111111ull;
 
-    // ---- control warp: ask for chunks [c_begin, c_end) of the current pass, in order ----------------------------------
-    __device__ __forceinline__ void produce(const char* rowq, const char* rowp, bool with_draft, int c_begin, int c_end) {
+    __device__ __forceinline__ void reset() {
+        resident = 0ull;
+        fill_par = (1u << kSlots) - 1u;
+        round_par = (1u << kSlots) - 1u;
+        round_used = 0u;
+        backward = 0;
+    }
+    __device__ __forceinline__ void forget_node() {
+        resident = 0ull;
+        backward = 0;
+    }
+
+    // ---- control warp: which chunks of the coming pass must be copied (`missing`), its direction, and its parity word
+    // (bit c: phase parity of the "full" barrier that will hold chunk c when the pass reaches it).  Chunk c lives in
+    // slot c mod 4; the pass ends with its last four chunks in the ring. ----------------------------------------------------
+    __device__ __forceinline__ void plan(int& dir, unsigned long long& parity, unsigned long long& missing) {
+        static_assert(kSlots == 4, "the bit tricks below assume four slots");
+        const unsigned long long all = n_chunks >= 64 ? ~0ull : (1ull << n_chunks) - 1ull;
+        dir = backward;
+        backward ^= 1;
+        missing = all & ~resident;
+        // number of copies into chunk c's slot up to and including chunk c, in pass order, modulo 2
+        unsigned long long x = missing;
+        if (dir) { x ^= x >> 4; x ^= x >> 8; x ^= x >> 16; x ^= x >> 32; }
+        else { x ^= x << 4; x ^= x << 8; x ^= x << 16; x ^= x << 32; }
+        parity = (x ^ ((unsigned long long)fill_par * kEveryFourth)) & all;
+#pragma unroll
+        for (int s = 0; s < kSlots; ++s) fill_par ^= (unsigned)(__popcll(missing & (kEveryFourth << s)) & 1) << s;
+        resident = dir ? (all & 0xFull) : (all & ~(all >> 4));
+    }
+
+    // ---- control warp: ask for chunk c (the slot's previous use must be over).  All lanes call it together. -------------
+    __device__ __forceinline__ void fetch(const char* rowq, const char* rowp, bool with_draft, int c, bool was_used, uint32_t wait_parity) {
         const int lane = threadIdx.x & 31;
+        const int slot = c & (kSlots - 1);
         const int row_bytes = V * kElem, row_bytes16 = row_bytes & ~15;
-        for (int c = c_begin; c < c_end; ++c) {
-            const uint32_t g = g0 + (uint32_t)c;
-            const int slot = (int)(g & (kSlots - 1));
-            if (g >= (uint32_t)kSlots) wait_bar(&sm.empty[slot], ((g / kSlots) - 1u) & 1u, &sm.abort);
-            const int off = c * kRowChunkBytes;
-            int bytes = row_bytes16 - off;
-            bytes = bytes > kRowChunkBytes ? kRowChunkBytes : (bytes < 0 ? 0 : bytes);
-            unsigned char* dq = slots + (size_t)slot * 2 * kRowChunkBytes;
-            unsigned char* dp = dq + kRowChunkBytes;
-            if (c == n_chunks - 1) {
-                // End of the row: the last V sizeof(T) mod 16 bytes cannot go through the copy engine and are copied
-                // by hand; what follows, up to the end of the tile, is filled with -inf so that the working warps
-                // never have to look at an index.  Published by the barrier arrival below.
-                const int first = row_bytes16 / kElem;                        // first element copied by hand
-                const int tile_end = ((V + kTileElems - 1) / kTileElems) * kTileElems;
-                for (int x = first + lane; x < tile_end; x += 32) {
-                    const int at = (x - c * kChunkElems) * kElem;
-                    if (kElem == 2) {
-                        *(uint16_t*)(dq + at) = x < V ? ((const uint16_t*)rowq)[x] : (uint16_t)0xFF80u;
-                        if (with_draft) *(uint16_t*)(dp + at) = x < V ? ((const uint16_t*)rowp)[x] : (uint16_t)0xFF80u;
-                    } else {
-                        *(uint32_t*)(dq + at) = x < V ? ((const uint32_t*)rowq)[x] : 0xFF800000u;
-                        if (with_draft) *(uint32_t*)(dp + at) = x < V ? ((const uint32_t*)rowp)[x] : 0xFF800000u;
-                    }
+        if (was_used) wait_bar(&sm.empty[slot], wait_parity, &sm.abort);
+        const int off = c * kRowChunkBytes;
+        int bytes = row_bytes16 - off;
+        bytes = bytes > kRowChunkBytes ? kRowChunkBytes : (bytes < 0 ? 0 : bytes);
+        unsigned char* dq = slots + (size_t)slot * 2 * kRowChunkBytes;
+        unsigned char* dp = dq + kRowChunkBytes;
+        if (c == n_chunks - 1) {
+            // End of the row: the last V sizeof(T) mod 16 bytes cannot go through the copy engine and are copied by
+            // hand; what follows, up to the end of the tile, is filled with -inf so that the working warps never have
+            // to look at an index.  Published by the barrier arrival below.
+            const int first = row_bytes16 / kElem;                        // first element copied by hand
+            const int tile_end = ((V + kTileElems - 1) / kTileElems) * kTileElems;
+            for (int x = first + lane; x < tile_end; x += 32) {
+                const int at = (x - c * kChunkElems) * kElem;
+                if (kElem == 2) {
+                    *(uint16_t*)(dq + at) = x < V ? ((const uint16_t*)rowq)[x] : (uint16_t)0xFF80u;
+                    if (with_draft) *(uint16_t*)(dp + at) = x < V ? ((const uint16_t*)rowp)[x] : (uint16_t)0xFF80u;
+                } else {
+                    *(uint32_t*)(dq + at) = x < V ? ((const uint32_t*)rowq)[x] : 0xFF800000u;
+                    if (with_draft) *(uint32_t*)(dp + at) = x < V ? ((const uint32_t*)rowp)[x] : 0xFF800000u;
                 }
-                __syncwarp();
             }
-            if (lane == 0) {
-                mbar_expect_tx(&sm.full[slot], with_draft ? 2u * (uint32_t)bytes : (uint32_t)bytes);
-                if (bytes > 0) {
-                    bulk_load(dq, rowq + off, (uint32_t)bytes, &sm.full[slot]);
-                    if (with_draft) bulk_load(dp, rowp + off, (uint32_t)bytes, &sm.full[slot]);
-                }
+            __syncwarp();
+        }
+        if (lane == 0) {
+            mbar_expect_tx(&sm.full[slot], with_draft ? 2u * (uint32_t)bytes : (uint32_t)bytes);
+            if (bytes > 0) {
+                bulk_load(dq, rowq + off, (uint32_t)bytes, &sm.full[slot]);
+                if (with_draft) bulk_load(dp, rowp + off, (uint32_t)bytes, &sm.full[slot]);
             }
         }
     }
 
-    // ---- working warps: every chunk of the pass in order; fn(tile, q tile, p tile) for this warp's tile of it -------
+    // ---- control warp: steps [i_begin, i_end) of the pass, in order ------------------------------------------------------------
+    __device__ __forceinline__ void produce(const char* rowq, const char* rowp, bool with_draft, int dir, unsigned long long missing,
+                                            int i_begin, int i_end) {
+        for (int i = i_begin; i < i_end; ++i) {
+            const int c = dir ? n_chunks - 1 - i : i;
+            const int slot = c & (kSlots - 1);
+            const bool was_used = (round_used >> slot) & 1u;
+            const uint32_t wait_parity = (round_par >> slot) & 1u;
+            round_used |= 1u << slot;                              // this step is the slot's next round
+            round_par ^= 1u << slot;
+            if ((missing >> c) & 1ull) fetch(rowq, rowp, with_draft, c, was_used, wait_parity);
+        }
+    }
+
+    // ---- working warps: every chunk of the pass in its order; fn(tile, q tile, p tile) for this warp's tile of it -------
     template <typename F>
-    __device__ __forceinline__ void consume(F&& fn) {
+    __device__ __forceinline__ void consume(const PassCmd& cmd, F&& fn) {
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-        for (int c = 0; c < n_chunks; ++c) {
-            const uint32_t g = g0 + (uint32_t)c;
-            const int slot = (int)(g & (kSlots - 1));
-            const int i = (warp - c * kTPC) & (kWorkWarps - 1);   // tile of the chunk with (c kTPC + i) mod 8 == warp
-            const int tile = c * kTPC + i;
+        for (int i = 0; i < n_chunks; ++i) {
+            const int c = cmd.backward ? n_chunks - 1 - i : i;
+            const int slot = c & (kSlots - 1);
+            const int t = (warp - c * kTPC) & (kWorkWarps - 1);   // tile of the chunk with (c kTPC + t) mod 8 == warp
+            const int tile = c * kTPC + t;
             // every warp waits for every chunk, with or without a tile in it: a warp can then never be a whole turn
             // of the ring ahead of another, so an "empty" phase counts each warp exactly once
-            wait_bar(&sm.full[slot], (g / kSlots) & 1u, &sm.abort);
-            if (i < kTPC && tile < n_tiles) {
-                const unsigned char* q = slots + (size_t)slot * 2 * kRowChunkBytes + (size_t)i * kTileElems * kElem;
+            wait_bar(&sm.full[slot], (uint32_t)(cmd.parity >> c) & 1u, &sm.abort);
+            if (t < kTPC && tile < n_tiles) {
+                const unsigned char* q = slots + (size_t)slot * 2 * kRowChunkBytes + (size_t)t * kTileElems * kElem;
                 fn(tile, q, q + kRowChunkBytes);
             }
             __syncwarp();
@@ -228,7 +284,7 @@ struct Ring {
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
         float s0 = 0.0f, s1 = 0.0f, m0 = kNegInf, m1 = kNegInf;
         bool saw_nan = false;
-        consume([&](int tile, const unsigned char* qt, const unsigned char* pt) {
+        consume(cmd, [&](int tile, const unsigned char* qt, const unsigned char* pt) {
             Packed<T> pq;
             load_pieces(pq, qt, lane);
             float q[16];
@@ -262,7 +318,6 @@ struct Ring {
                 if (lane == 0) sm.tile_sum[tile] = (double)ts;
             }
         });
-        g0 += (uint32_t)n_chunks;
         s0 = warp_sum_f32(s0);
         s1 = warp_sum_f32(s1);
         if (CLEAN) {
@@ -302,7 +357,8 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
     const int32_t* tok = a.token + (int64_t)b * a.num_nodes;
     constexpr int kChunkElems = Ring<T>::kChunkElems;
 
-    Ring<T> ring = {sm, ring_mem, a.V, (a.V + kChunkElems - 1) / kChunkElems, (a.V + kTileElems - 1) / kTileElems, 0u};
+    Ring<T> ring = {sm, ring_mem, a.V, (a.V + kChunkElems - 1) / kChunkElems, (a.V + kTileElems - 1) / kTileElems};
+    ring.reset();
     if (tid == 0) {
         for (int s = 0; s < kSlots; ++s) {
             mbar_init(&sm.full[s], 1);
@@ -371,34 +427,41 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
     st.kp = kLog2e * a.draft.inv_temp;
     const char* rowq = nullptr;
     const char* rowp = nullptr;
-    // One pass: publish the command, ask for the rows, collect the working warps' results.  The first chunks are
-    // asked for before the command is published: their slots are free (every working warp has released every slot
-    // of the pass before), and the copies travel while the working warps wake up.
-    auto run_pass = [&](int kind, bool store_tiles, double& S0, double& S1, float& M0, float& M1) {
+    // One pass: plan which chunks must be copied, publish the command, ask for the rows, collect the working warps'
+    // results.  The first kSlots steps are taken before the command is published: what they wait for, if anything, are
+    // slot uses of earlier passes, which every working warp finished before it reported its sums; so the copies travel
+    // while the working warps wake up.  `meanwhile` runs on the control warp while the pass is under way.
+    auto run_pass = [&](int kind, bool store_tiles, double& S0, double& S1, float& M0, float& M1, auto&& meanwhile) {
         const bool with_draft = kind != kPassTarget;
+        int dir;
+        unsigned long long parity, missing;
+        ring.plan(dir, parity, missing);
         if (lane == 0) {
             PassCmd cmd;
             cmd.kind = kind; cmd.clean = st.has_nan ? 1 : 0; cmd.store_tiles = store_tiles ? 1 : 0;
             cmd.kq = st.kq; cmd.kp = st.kp; cmd.cq = st.mq * st.kq; cmd.cp = st.mp * st.kp;
             cmd.a_hi = st.a_hi; cmd.a_lo = st.a_lo;
+            cmd.backward = dir; cmd.parity = parity;
             sm.cmd = cmd;
         }
         const int early = ring.n_chunks < kSlots ? ring.n_chunks : kSlots;
-        ring.produce(rowq, rowp, with_draft, 0, early);
+        ring.produce(rowq, rowp, with_draft, dir, missing, 0, early);
         __syncthreads();   // the command is in place
-        ring.produce(rowq, rowp, with_draft, early, ring.n_chunks);
-        ring.g0 += (uint32_t)ring.n_chunks;
+        ring.produce(rowq, rowp, with_draft, dir, missing, early, ring.n_chunks);
+        meanwhile();
         __syncthreads();   // the warps' sums are in place
-        S0 = 0.0; S1 = 0.0; M0 = kNegInf; M1 = kNegInf;
+        static_assert(kWorkWarps == 8, "fixed summation tree over eight warps");
+        float4 r[kWorkWarps];
 #pragma unroll
-        for (int w = 0; w < kWorkWarps; ++w) {   // fixed order
-            const float4 r = sm.red[w];
-            S0 += (double)r.x;
-            S1 += (double)r.y;
-            M0 = fmaxf(M0, r.z);
-            M1 = fmaxf(M1, r.w);
-        }
+        for (int w = 0; w < kWorkWarps; ++w) r[w] = sm.red[w];
+        S0 = (((double)r[0].x + (double)r[1].x) + ((double)r[2].x + (double)r[3].x)) +
+             (((double)r[4].x + (double)r[5].x) + ((double)r[6].x + (double)r[7].x));
+        S1 = (((double)r[0].y + (double)r[1].y) + ((double)r[2].y + (double)r[3].y)) +
+             (((double)r[4].y + (double)r[5].y) + ((double)r[6].y + (double)r[7].y));
+        M0 = fmaxf(fmaxf(fmaxf(r[0].z, r[1].z), fmaxf(r[2].z, r[3].z)), fmaxf(fmaxf(r[4].z, r[5].z), fmaxf(r[6].z, r[7].z)));
+        M1 = fmaxf(fmaxf(fmaxf(r[0].w, r[1].w), fmaxf(r[2].w, r[3].w)), fmaxf(fmaxf(r[4].w, r[5].w), fmaxf(r[6].w, r[7].w)));
     };
+    auto nothing = [] {};
 
     int status = 0, cur = 0, len = 0, reason = 0, last = -1;
     bool tiles_valid = false;   // sm.tile_sum holds the tile sums of the distribution the last token is drawn from
@@ -411,20 +474,30 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
         st.A = 0.0; st.P = 0.0; st.Z = 1.0; st.a_hi = st.a_lo = 0.0f; st.has_nan = false;
         st.mq = 0.0f; st.mp = 0.0f; st.Sp = 1.0;
         tiles_valid = false;
-        // The row values of the node's first 32 children (the thresholds need them right after the first pass): lane j
-        // fetches those of child j; the loads are in flight while the rows stream.
+        ring.forget_node();
+        // The node's first 32 children in stored order, one per lane: node, token and the two row values (the
+        // thresholds need them right after the first pass); the loads are in flight while the rows stream.
         int child_node = -1, child_x = -1;
         float child_lq = 0.0f, child_lp = 0.0f;
         if (st.with_draft) {
-            int cc = c;
-            for (int j = 0; j < 32 && cc >= 0; ++j) {
-                if (j == lane) {
-                    child_node = cc;
-                    child_x = cached ? sm.tok[cc] : tok[cc];
-                    child_lq = RowIO<T>::scalar(rowq, child_x);
-                    child_lp = RowIO<T>::scalar(rowp, child_x);
+            int found = 0;
+            for (int c0 = 1; c0 < a.num_nodes && found < 32; c0 += 32) {
+                const int cc = c0 + lane;
+                bool ok = false;
+                if (cc < a.num_nodes) {
+                    const int p = cached ? sm.par[cc] : par[cc];
+                    const int t = cached ? sm.tok[cc] : tok[cc];
+                    ok = p == cur && t >= 0 && t < a.V;
                 }
-                cc = find_child(cur, cc);
+                const unsigned m = __ballot_sync(0xFFFFFFFFu, ok);
+                const int k = __popc(m);
+                if (lane >= found && lane < found + k) child_node = c0 + (int)__fns(m, 0, lane - found + 1);   // its (lane - found)-th
+                found += k;
+            }
+            if (child_node >= 0) {
+                child_x = cached ? sm.tok[child_node] : tok[child_node];
+                child_lq = RowIO<T>::scalar(rowq, child_x);
+                child_lp = RowIO<T>::scalar(rowp, child_x);
             }
         }
         // First pass.  Exponentials are taken relative to a reference, 0 to begin with: the plain pass has no code for
@@ -435,7 +508,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             float M0, M1;
             const int kind = st.with_draft ? kPassFirst : kPassTarget;
             for (int attempt = 0; attempt < 3; ++attempt) {
-                run_pass(kind, !st.with_draft, S0, S1, M0, M1);
+                run_pass(kind, !st.with_draft, S0, S1, M0, M1, nothing);
                 if (sm.abort) { aborted = true; break; }
                 if (!st.with_draft) S1 = 1.0;
                 const bool good = S0 >= (double)kSumFloor && S0 < 1e300 && S1 >= (double)kSumFloor && S1 < 1e300;
@@ -460,68 +533,63 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             reason = (len >= a.L) ? 2 : 1;  // RSD_STOP_LEAF : RSD_STOP_NO_CHILDREN
             break;
         }
-        int accepted = -1, j = 0;
+        const double inv_Sq = 1.0 / st.Sq, inv_Sp = 1.0 / st.Sp, ratio = st.Sq * inv_Sp;
         int rem_x[4];            // rejected tokens of this node, lanes hold them four at a time (lane i: entries 4 i ..)
         int n_removed = 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) rem_x[i] = -1;
-        while (c >= 0) {
-            int x;
+        // What the test of child j needs and no pass changes: its token, its probabilities under the node's two rows,
+        // whether an earlier sibling with the same token was rejected, and its uniform.
+        int j = 0, x = -1;
+        double qx = 0.0, px_row = 0.0, U = 0.0;
+        bool repeated = false;
+        auto prepare = [&](int child) {
             float lq, lp;
             if (j < 32) {
                 x = __shfl_sync(0xFFFFFFFFu, child_x, j);
                 lq = __shfl_sync(0xFFFFFFFFu, child_lq, j);
                 lp = __shfl_sync(0xFFFFFFFFu, child_lp, j);
             } else {
-                x = cached ? sm.tok[c] : tok[c];
+                x = cached ? sm.tok[child] : tok[child];
                 lq = RowIO<T>::scalar(rowq, x);
                 lp = RowIO<T>::scalar(rowp, x);
             }
             const float qh = (lq == lq) ? ex2_approx(fmaf(lq, st.kq, -st.mq * st.kq)) : 0.0f;
             const float ph = (lp == lp) ? ex2_approx(fmaf(lp, st.kp, -st.mp * st.kp)) : 0.0f;
-            const double qx = (double)qh / st.Sq, px_row = (double)ph / st.Sp;
-            // a sibling with the same token was rejected before: its draft mass is gone (Eq. 1)
+            qx = (double)qh * inv_Sq;
+            px_row = (double)ph * inv_Sp;
             bool mine = false;
 #pragma unroll
             for (int i = 0; i < 4; ++i) mine |= rem_x[i] == x;
-            const bool repeated = __any_sync(0xFFFFFFFFu, mine);
+            repeated = __any_sync(0xFFFFFFFFu, mine);   // its draft mass is gone (Eq. 1)
+            const uint4 rw = rng_draw(key, (uint32_t)cur, kTagAccept, (uint32_t)j);
+            U = (double)(rw.x >> 8) * (1.0 / 16777216.0);
+        };
+        prepare(c);
+        double inv_1mP = 1.0;    // 1 / (1 - P)
+        int accepted = -1;
+        while (c >= 0) {
+            // Eq. 3 in closed form: accept iff U < min(1, r (1 - P) / (Z p(x))), r = (q(x) - A p(x))+, tested without
+            // the division; a child the draft cannot produce any more is taken iff it has residual mass
             const double px = repeated ? 0.0 : px_row;
             const double r = fmax(qx - st.A * px_row, 0.0);
-            double theta;
-            if (px > 0.0) theta = fmin(1.0, r * (1.0 - st.P) / (st.Z * px));
-            else { status |= 8; theta = r > 0.0 ? 1.0 : 0.0; }   // RSD_ST_ZERO_DRAFT_PROB
-            const uint4 rw = rng_draw(key, (uint32_t)cur, kTagAccept, (uint32_t)j);
-            const double U = (double)(rw.x >> 8) * (1.0 / 16777216.0);
-            if (a.dbg_theta && lane == 0) a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)theta;
-            if (U < theta) { accepted = c; break; }
+            bool take;
+            if (px > 0.0) take = U * st.Z * px < r * (1.0 - st.P);
+            else { status |= 8; take = r > 0.0; }   // RSD_ST_ZERO_DRAFT_PROB
+            if (a.dbg_theta && lane == 0)
+                a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)(px > 0.0 ? fmin(1.0, r * (1.0 - st.P) / (st.Z * px)) : (r > 0.0 ? 1.0 : 0.0));
+            if (take) { accepted = c; break; }
+            // rejected.  Eqs. 1-2 in closed form: A_{j+1} = A_j + Z_j / (1 - P_j), Z_{j+1} = sum (q - A_{j+1} p)+
             ++j;
             const int next = j < 32 ? __shfl_sync(0xFFFFFFFFu, child_node, j) : find_child(cur, c);
-            // Eqs. 1-2 in closed form: A_{j+1} = A_j + Z_j / (1 - P_j), Z_{j+1} = sum (q - A_{j+1} p)+
             const double A_old = st.A;
-            st.A = st.A + st.Z / (1.0 - st.P);
+            st.A = fma(st.Z, inv_1mP, st.A);
             {
-                const double aa = st.A * st.Sq / st.Sp;
+                const double aa = st.A * ratio;
                 st.a_hi = (float)aa;
                 st.a_lo = (float)(aa - (double)st.a_hi);
             }
-            double zhat, none;
-            float f0, f1;
-            const bool maybe_last = next < 0;   // no sibling left: the last token is drawn from this residual
-            run_pass(kPassResidual, maybe_last, zhat, none, f0, f1);
-            if (sm.abort) { aborted = true; break; }
-            const double Z_new = zhat / st.Sq;
-            if (Z_new > 0.0 && Z_new < 1.7e308) {
-                st.Z = Z_new;
-                tiles_valid = maybe_last;
-            } else {
-                status |= 4;   // RSD_ST_ZERO_RESIDUAL: keep the previous residual
-                st.A = A_old;
-                const double aa = st.A * st.Sq / st.Sp;
-                st.a_hi = (float)aa;
-                st.a_lo = (float)(aa - (double)st.a_hi);
-                tiles_valid = false;
-            }
-            st.P += px;
+            const double P_new = st.P + px;
             if (!repeated && n_removed < kMaxRemovedRing) {
                 if (lane == (n_removed >> 2)) {
 #pragma unroll
@@ -530,6 +598,27 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
                 }
                 ++n_removed;
             }
+            double zhat, none;
+            float f0, f1;
+            const bool maybe_last = next < 0;   // no sibling left: the last token is drawn from this residual
+            run_pass(kPassResidual, maybe_last, zhat, none, f0, f1, [&] {
+                inv_1mP = 1.0 / (1.0 - P_new);
+                if (next >= 0) prepare(next);
+            });
+            if (sm.abort) { aborted = true; break; }
+            const double Z_new = zhat * inv_Sq;
+            if (Z_new > 0.0 && Z_new < 1.7e308) {
+                st.Z = Z_new;
+                tiles_valid = maybe_last;
+            } else {
+                status |= 4;   // RSD_ST_ZERO_RESIDUAL: keep the previous residual
+                st.A = A_old;
+                const double aa = st.A * ratio;
+                st.a_hi = (float)aa;
+                st.a_lo = (float)(aa - (double)st.a_hi);
+                tiles_valid = false;
+            }
+            st.P = P_new;
             if (!(1.0 - st.P > 0.0)) { status |= 16; break; }   // RSD_ST_DRAFT_EXHAUSTED
             c = next;
         }
@@ -550,17 +639,16 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
     if (!aborted && !tiles_valid) {   // rare: the last pass was not kept, or it did not store its tile sums
         double s, none;
         float f0, f1;
-        if (!residual) rowp = rowq;
-        run_pass(residual ? kPassResidual : kPassTarget, true, s, none, f0, f1);
+        if (!residual) { rowp = rowq; ring.forget_node(); }   // (the slots' draft halves are not refreshed by this pass)
+        run_pass(residual ? kPassResidual : kPassTarget, true, s, none, f0, f1, nothing);
         aborted = sm.abort != 0;
     }
     // the working warps are done: let them go, then finish alone
     if (lane == 0) sm.cmd.kind = kPassEnd;
     if (aborted) {
         // A wait ran out.  Before the block gives its shared memory back, wait once more (bounded) for the copies it
-        // may still have in flight: the last kSlots chunks it asked for.
-        for (uint32_t g = ring.g0 > (uint32_t)kSlots ? ring.g0 - kSlots : 0u; g < ring.g0; ++g)
-            wait_bar(&sm.full[g & (kSlots - 1)], (g / kSlots) & 1u, &sm.abort);
+        // may still have in flight: the latest one of every slot.
+        for (int s = 0; s < kSlots; ++s) wait_bar(&sm.full[s], (ring.fill_par >> s) & 1u, &sm.abort);   // (a slot never filled passes at once)
         status |= 32;   // RSD_ST_TIMEOUT
     }
     __syncthreads();
