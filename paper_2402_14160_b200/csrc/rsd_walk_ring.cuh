@@ -238,6 +238,39 @@ struct Ring {
         }
     }
 
+    // ---- control warp: the first `early` (<= kSlots) steps of the pass at once, lane i taking step i: their slots are
+    // distinct, and what they wait for, if anything, are uses of earlier passes, which are over.  The row's last chunk
+    // needs the whole warp (hand-copied tail) and goes first if it is among them. -------------------------------------------
+    __device__ __forceinline__ void produce_early(const char* rowq, const char* rowp, bool with_draft, int dir,
+                                                  unsigned long long missing, int early) {
+        const int lane = threadIdx.x & 31;
+        const int row_bytes16 = (V * kElem) & ~15;
+        const int i_last = dir ? 0 : n_chunks - 1;                 // step of chunk n_chunks - 1
+        if (i_last < early && ((missing >> (n_chunks - 1)) & 1ull)) {
+            const int slot = (n_chunks - 1) & (kSlots - 1);
+            fetch(rowq, rowp, with_draft, n_chunks - 1, (round_used >> slot) & 1u, (round_par >> slot) & 1u);
+        }
+        if (lane < early && lane != i_last) {
+            const int c = dir ? n_chunks - 1 - lane : lane;
+            const int slot = c & (kSlots - 1);
+            if ((missing >> c) & 1ull) {
+                if ((round_used >> slot) & 1u) wait_bar(&sm.empty[slot], (round_par >> slot) & 1u, &sm.abort);
+                const int off = c * kRowChunkBytes;                // (not the last chunk: a whole chunk)
+                const uint32_t bytes = (uint32_t)(row_bytes16 - off > kRowChunkBytes ? kRowChunkBytes : row_bytes16 - off);
+                unsigned char* dq = slots + (size_t)slot * 2 * kRowChunkBytes;
+                mbar_expect_tx(&sm.full[slot], with_draft ? 2u * bytes : bytes);
+                bulk_load(dq, rowq + off, bytes, &sm.full[slot]);
+                if (with_draft) bulk_load(dq + kRowChunkBytes, rowp + off, bytes, &sm.full[slot]);
+            }
+        }
+        __syncwarp();
+        for (int i = 0; i < early; ++i) {                          // each of these steps is its slot's next round
+            const int slot = (dir ? n_chunks - 1 - i : i) & (kSlots - 1);
+            round_used |= 1u << slot;
+            round_par ^= 1u << slot;
+        }
+    }
+
     // ---- control warp: steps [i_begin, i_end) of the pass, in order ------------------------------------------------------------
     __device__ __forceinline__ void produce(const char* rowq, const char* rowp, bool with_draft, int dir, unsigned long long missing,
                                             int i_begin, int i_end) {
@@ -445,7 +478,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             sm.cmd = cmd;
         }
         const int early = ring.n_chunks < kSlots ? ring.n_chunks : kSlots;
-        ring.produce(rowq, rowp, with_draft, dir, missing, 0, early);
+        ring.produce_early(rowq, rowp, with_draft, dir, missing, early);
         __syncthreads();   // the command is in place
         ring.produce(rowq, rowp, with_draft, dir, missing, early, ring.n_chunks);
         meanwhile();
