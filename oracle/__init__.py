@@ -263,3 +263,28 @@ def resample_residual(draft, target, rejected, rng_node, seed, step, *, seq_base
                                        C.c_uint64(seed), C.c_uint32(step), C.c_uint32(seq_base),
                                        _ptr(out), _ptr(res), _ptr(margin), _ptr(status))
     return dict(token=out, residual=res, margin=margin, status=status)
+
+
+def filter_rows(rows, top_k=0, top_p=1.0, *, temperature=1.0):
+    """rows [B,R,V] -> dict(keep [B,R,V] bool, kept [B,R], margin [B,R]): top-k then nucleus filtering of every row
+    (after the temperature); a filtered token counts as -inf from then on."""
+    a, dt = _rows(rows)
+    B, R, V = a.shape
+    assert a.strides[2] == a.itemsize
+    keep = np.zeros((B, R, V), np.uint8)
+    kept = np.zeros((B, R), np.int32)
+    margin = np.zeros((B, R), np.float64)
+    lib().rsd_oracle_filter_rows(_ptr(a), C.c_int(dt), C.c_double(temperature), C.c_int64(a.strides[0] // a.itemsize),
+                                 C.c_int64(a.strides[1] // a.itemsize), C.c_int(B), C.c_int(R), C.c_int(V),
+                                 C.c_int(int(top_k)), C.c_double(float(top_p)), _ptr(keep), _ptr(kept), _ptr(margin))
+    return dict(keep=keep.astype(bool), kept=kept, margin=margin)
+
+
+def apply_filter(rows, keep):
+    """The rows with -inf at every filtered entry (same storage type: float32, or bf16 bit patterns)."""
+    out = np.array(rows, copy=True)
+    if out.dtype == np.uint16:
+        out[~keep] = 0xFF80
+    else:
+        out[~keep] = -np.inf
+    return out

@@ -13,6 +13,7 @@
  *   - Stochastic Beam Search step .................. Eqs. 10-12, Algorithm 9
  *   - recursive rejection sampling (one sibling chain) Eqs. 1-4, Algorithm 1
  *   - verification walk over the draft tree ......... Section 3.2.2, Algorithm 6
+ *   - top-k / nucleus filtering of a row ............ Section 4 (sampling settings), Algorithms 4 and 9 (-inf filter)
  *
  * Random numbers.  The paper only says "standard Gumbel" and "Uniform[0,1]".
  * Both sides of the parity check draw them from the counter-based generator
@@ -225,6 +226,83 @@ static void log_softmax_row(double* v, int V, int is_logprob) {
 static void softmax_row(const double* logits, int V, double* prob) {
     double lse = log_sum_exp(logits, V);
     for (int x = 0; x < V; ++x) prob[x] = isinf(lse) ? 0.0 : exp(logits[x] - lse);
+}
+
+/* ------------------------------------------------------------------------ */
+/* logit warping: top-k and nucleus (top-p) filtering (Section 4)            */
+/* ------------------------------------------------------------------------ */
+/*
+ * Section 4 samples with temperature 0.3 / 1.0 and, for one task, nucleus (top-p) sampling with p = 0.95; the
+ * paper gives no formula.  Reading: the usual order of logit warpers, temperature -> top-k -> top-p, each applied
+ * to what the one before left:
+ *   top-k   keep the k tokens with the largest probability (equal values: the smaller token first);
+ *   top-p   sort what is left by probability, largest first (equal values: the smaller token first), renormalise,
+ *           and keep the shortest prefix whose mass reaches top_p (at least one token).
+ * A filtered token counts as log-probability -inf from then on ("filter elements whose log-prob is -inf",
+ * Algorithms 4 and 9).  top_k <= 0 or >= V and top_p <= 0 or >= 1 mean "no filter".
+ *
+ * keep[x] = 1 for kept tokens.  *margin = distance of top_p from the two cumulative masses that bracket it
+ * (the mass of the kept prefix, and that prefix without its last token), as fractions of the total; +inf if no
+ * nucleus filter applies.  Returns the number of kept tokens.
+ */
+typedef struct { double v; int x; } orc_entry;
+static int orc_entry_cmp(const void* a, const void* b) {
+    const orc_entry* ea = (const orc_entry*)a;
+    const orc_entry* eb = (const orc_entry*)b;
+    if (ea->v > eb->v) return -1;
+    if (ea->v < eb->v) return 1;
+    return (ea->x > eb->x) - (ea->x < eb->x);
+}
+
+int rsd_oracle_filter_row(const double* scaled /* row / temperature, NaN already -inf */, int V, int top_k, double top_p,
+                          uint8_t* keep, double* margin) {
+    orc_entry* e = (orc_entry*)malloc(sizeof(orc_entry) * (size_t)V);
+    int n = 0;
+    for (int x = 0; x < V; ++x) {
+        keep[x] = 0;
+        if (scaled[x] > -INFINITY) { e[n].v = scaled[x]; e[n].x = x; ++n; }
+    }
+    qsort(e, (size_t)n, sizeof(orc_entry), orc_entry_cmp);   /* decreasing value, then increasing token */
+    if (top_k > 0 && top_k < V && n > top_k) n = top_k;
+    if (margin) *margin = INFINITY;
+    if (top_p > 0.0 && top_p < 1.0 && n > 0) {
+        double total = 0.0;
+        for (int i = 0; i < n; ++i) total += exp(e[i].v - e[0].v);
+        double run = 0.0;
+        int m = n;
+        for (int i = 0; i < n; ++i) {
+            double before = run;
+            run += exp(e[i].v - e[0].v);
+            if (run >= top_p * total) {
+                m = i + 1;
+                if (margin) {
+                    double a = run / total - top_p, b = top_p - before / total;
+                    *margin = a < b ? a : b;
+                }
+                break;
+            }
+        }
+        n = m;
+    }
+    for (int i = 0; i < n; ++i) keep[e[i].x] = 1;
+    free(e);
+    return n;
+}
+
+/* rows [B][R][V] -> keep [B][R][V] (1 = kept), kept [B][R], margin [B][R] */
+int rsd_oracle_filter_rows(const void* data, int dtype, double temperature, int64_t seq_stride, int64_t row_stride,
+                           int B, int R, int V, int top_k, double top_p, uint8_t* keep, int32_t* kept, double* margin) {
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        for (int r = 0; r < R; ++r) {
+            double* v = (double*)malloc(sizeof(double) * (size_t)V);
+            load_row(data, dtype, b * seq_stride + r * row_stride, V, temperature, v);
+            kept[(int64_t)b * R + r] = rsd_oracle_filter_row(v, V, top_k, top_p, keep + ((int64_t)b * R + r) * V,
+                                                             margin ? margin + (int64_t)b * R + r : NULL);
+            free(v);
+        }
+    }
+    return 0;
 }
 
 /* ------------------------------------------------------------------------ */
