@@ -110,6 +110,27 @@ const char* rsd_last_error(void);
 int rsd_profile_next_scan(void* before, void* after);
 
 /*
+ * Logit warping of rows before drafting or verification: top-k and nucleus (top-p) filtering (Section 4 samples with
+ * temperature 0.3 / 1.0 and, for one task, top-p 0.95; the paper gives no formula).  The order is the usual one,
+ * temperature -> top-k -> top-p, each applied to what the one before left:
+ *   top-k   keep the top_k largest values of a row (equal values: the smaller token first)
+ *   top-p   of what is left, in order of decreasing probability under softmax(value / temperature) (equal values: the
+ *           smaller token first), keep the shortest prefix whose share of the mass reaches top_p (at least one token)
+ * A filtered token counts as log-probability -inf from then on (Algorithms 4 and 9 drop such entries): the call writes a
+ * copy of the rows with -inf at the filtered entries and the stored values (not divided by the temperature) elsewhere,
+ * to be passed to the drafting and verification calls in place of the rows, with the same temperature.  Draft and
+ * target rows are filtered separately, each with its own settings.
+ *   rows        [B][R][V]; rows->temperature enters the nucleus masses only; NaN entries count as -inf (RSD_ST_NAN_INPUT)
+ *   top_k       0 (or >= V): none;   top_p  >= 1: none
+ *   out_rows    [B][R][V] dense, the rows' element type; may not overlap the input
+ *   out_kept    optional [B][R] int32: entries kept in each row;   status [B]
+ * A row must fit in shared memory with the call's other data (up to 104,000 2-byte or 52,000 4-byte entries); longer
+ * rows are refused with RSD_ERR_UNSUPPORTED.
+ */
+int rsd_filter_rows(const rsd_rows* rows, int B, int R, int V, int top_k, float top_p, void* out_rows, int32_t* out_kept,
+                    int32_t* status, rsd_stream_t stream);
+
+/*
  * Gumbel-Top-k drafting for RSD with constant branching factors (Section 3.2.1, Eqs. 5-8; Algorithm 4).
  * For each of the B*R rows: phi = log-softmax(row) (Eq. 5), phi~ = phi + G (Eq. 6), and the k_per_row[r] tokens
  * with the largest phi~ in decreasing order (Eq. 7); equal values go to the smaller token.  The noise of row r is

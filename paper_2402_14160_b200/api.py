@@ -22,7 +22,7 @@ RULE_RRS, RULE_MULTIROUND, RULE_KSEQ = 0, 1, 2
 FINAL_INVERSE_CDF, FINAL_GUMBEL_TOP1 = 0, 1
 MAX_K = 32
 
-EXPORTS = ["rsd_version", "rsd_rng_layout", "rsd_last_error", "rsd_profile_next_scan", "rsd_gumbel_topk_draft", "rsd_sbs_workspace_bytes",
+EXPORTS = ["rsd_version", "rsd_rng_layout", "rsd_last_error", "rsd_profile_next_scan", "rsd_filter_rows", "rsd_gumbel_topk_draft", "rsd_sbs_workspace_bytes",
            "rsd_sbs_step", "rsd_sbs_step_static", "rsd_sbs_tree_workspace_bytes", "rsd_sbs_draft_tree", "rsd_verify_tree", "rsd_verify_tree_rule", "rsd_resample_residual"]
 
 
@@ -62,6 +62,8 @@ def lib():
                                    C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
                                    C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]
+        l.rsd_filter_rows.argtypes = [C.POINTER(RsdRows), C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, C.c_void_p,
+                                      C.c_void_p, C.c_void_p, C.c_void_p]
         l.rsd_sbs_tree_workspace_bytes.restype = C.c_size_t
         l.rsd_sbs_tree_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int]
         l.rsd_sbs_draft_tree.argtypes = [C.POINTER(RsdRows), C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint64, C.c_uint32,
@@ -126,6 +128,23 @@ def _new(shape, dtype, device):
 def _host_i32(values: Sequence[int]):
     arr = (C.c_int32 * len(values))(*[int(v) for v in values])
     return arr
+
+
+def rsd_filter_rows(rows: torch.Tensor, top_k: int = 0, top_p: float = 1.0, *, temperature: float = 1.0,
+                    out: Optional[dict] = None):
+    """rows [B, R, V] -> dict(rows [B, R, V] with -inf at the entries that top-k / nucleus filtering removes, kept [B, R],
+    status [B]).  Pass the result to the drafting and verification calls in place of the rows, with the same temperature."""
+    B, R, V = rows.shape
+    dev = rows.device
+    if out is None:
+        out = dict(rows=_new((B, R, V), rows.dtype, dev), kept=_new((B, R), torch.int32, dev),
+                   status=_new((B,), torch.int32, dev))
+    if not out["rows"].is_contiguous() or out["rows"].dtype != rows.dtype:
+        raise RsdError("out rows must be contiguous and of the rows' dtype")
+    r = rows_of(rows, False, temperature)
+    _check(lib().rsd_filter_rows(C.byref(r), B, R, V, int(top_k), float(top_p), _ptr(out["rows"]), _ptr(out["kept"]),
+                                 _ptr(out["status"]), _stream()))
+    return out
 
 
 def rsd_gumbel_topk_draft(draft: torch.Tensor, k_per_row: Sequence[int], rng_node: Sequence[int], seed: int,

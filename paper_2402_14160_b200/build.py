@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librsd.so")
 SOURCES = ["rsd_api.cu", "rsd_api_verify.cu"]
-HEADERS = ["rsd_api_common.h", "rsd_device.cuh", "rsd_scan.cuh", "rsd_verify.cuh", "rsd_verify_walk.inc", "rsd_walk_ring.cuh", os.path.join("..", "..", "include", "rsd.h")]
+HEADERS = ["rsd_api_common.h", "rsd_device.cuh", "rsd_scan.cuh", "rsd_filter.cuh", "rsd_verify.cuh", "rsd_verify_walk.inc", "rsd_walk_ring.cuh", os.path.join("..", "..", "include", "rsd.h")]
 
 
 def _stale() -> bool:

@@ -3,10 +3,12 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 
 #include "rsd_api_common.h"
 #include "rsd_scan.cuh"
+#include "rsd_filter.cuh"
 
 namespace rsd_host {
 thread_local char g_err[512] = "";
@@ -186,6 +188,48 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     return check_launch("rsd_sbs_step(epilogue)");
 }
 
+
+int rsd_filter_rows(const rsd_rows* rows, int B, int R, int V, int top_k, float top_p, void* out_rows, int32_t* out_kept,
+                    int32_t* status, rsd_stream_t stream) {
+    g_err[0] = 0;
+    if (int e = check_vocab(V)) return e;
+    if (int e = check_rows("rows", rows, V, R > 1)) return e;
+    if (B < 0 || R < 1) return fail(RSD_ERR_INVALID_ARG, "B = %d, R = %d", B, R);
+    if (top_k < 0) return fail(RSD_ERR_INVALID_ARG, "top_k = %d must be >= 0 (0: none)", top_k);
+    if (!(top_p > 0.0f)) return fail(RSD_ERR_INVALID_ARG, "top_p = %g must be > 0 (>= 1: none)", (double)top_p);
+    if (!out_rows || !status) return fail(RSD_ERR_INVALID_ARG, "null output");
+    if ((int64_t)B * R > 0x7FFFFFFF) return fail(RSD_ERR_UNSUPPORTED, "B * R too large");
+    const size_t elem = rows->dtype == RSD_F32 ? 4 : 2;
+    const size_t smem = (size_t)V * elem + 16;
+    constexpr size_t kSharedPerBlock = 227 * 1024;
+    if (smem + sizeof(rsd::FilterSmem) + 256 > kSharedPerBlock)
+        return fail(RSD_ERR_UNSUPPORTED, "rows of %d %zu-byte entries do not fit in shared memory (at most %zu entries)", V, elem,
+                    (kSharedPerBlock - sizeof(rsd::FilterSmem) - 272) / elem);
+    if (B == 0) return RSD_OK;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(status, 0, sizeof(int32_t) * (size_t)B, s) != cudaSuccess) return check_launch("memset(status)");
+    rsd::FilterArgs a;
+    a.data = rows->data; a.out = out_rows; a.seq_stride = rows->seq_stride; a.row_stride = rows->row_stride;
+    a.R = R; a.V = V; a.top_k = top_k; a.top_p = top_p;
+    a.log2e_over_t = rsd::kLog2e / temperature_of(rows);
+    a.kept = out_kept; a.status = status;
+    // the attribute belongs to the (function, device) pair: raised once per device to the largest row that fits
+    static std::atomic<bool> raised[2][64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return check_launch("cudaGetDevice");
+    const int which = rows->dtype == RSD_F32 ? 0 : 1;
+    if (dev < 0 || dev >= 64 || !raised[which][dev].load(std::memory_order_acquire)) {
+        const int most = (int)(kSharedPerBlock - sizeof(rsd::FilterSmem) - 256);
+        const cudaError_t e = rows->dtype == RSD_F32
+                                  ? cudaFuncSetAttribute(rsd::filter_rows_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, most)
+                                  : cudaFuncSetAttribute(rsd::filter_rows_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, most);
+        if (e != cudaSuccess) return check_launch("cudaFuncSetAttribute");
+        if (dev >= 0 && dev < 64) raised[which][dev].store(true, std::memory_order_release);
+    }
+    if (rows->dtype == RSD_F32) rsd::filter_rows_kernel<float><<<B * R, rsd::kFilterThreads, smem, s>>>(a);
+    else rsd::filter_rows_kernel<__nv_bfloat16><<<B * R, rsd::kFilterThreads, smem, s>>>(a);
+    return check_launch("rsd_filter_rows");
+}
 
 size_t rsd_sbs_tree_workspace_bytes(int B, int W, int L) {
     if (B < 0 || W < 1 || L < 1) return 0;
