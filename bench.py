@@ -222,6 +222,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--sequences", type=int, default=0, help="sequences per GPU (default: the workload's batch)")
+    ap.add_argument("--top-p", type=float, default=1.0, help="nucleus filtering of the draft and target rows in every step (1: off)")
+    ap.add_argument("--top-k", type=int, default=0, help="top-k filtering of the draft and target rows in every step (0: off)")
     ap.add_argument("--per-level", action="store_true",
                     help="Stochastic Beam Search: one rsd_sbs_step call per level instead of rsd_sbs_draft_tree")
     args = ap.parse_args()
@@ -265,7 +267,26 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # optional logit warping: the rows of every step go through rsd_filter_rows first (two more launches per step)
+    warp_rows = args.top_p < 1.0 or args.top_k > 0
+    raw_draft, raw_target = draft, target
+    filt = None
+    if warp_rows:
+        filt = [api.rsd_filter_rows(raw_draft, args.top_k, args.top_p), api.rsd_filter_rows(raw_target, args.top_k, args.top_p)]
+        draft, target = filt[0]["rows"], filt[1]["rows"]
+        filter_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+
+    def warp_step(s=None):
+        if warp_rows:
+            if s is not None:
+                filter_ev[s][0].record()
+            api.rsd_filter_rows(raw_draft, args.top_k, args.top_p, out=filt[0])
+            api.rsd_filter_rows(raw_target, args.top_k, args.top_p, out=filt[1])
+            if s is not None:
+                filter_ev[s][1].record()
+
     for s in range(max(args.warmup, 3)):
+        warp_step()
         stepper.run(draft, target, 0, s, seq_base)
     barrier()
 
@@ -286,6 +307,7 @@ def main():
     with ClockSampler(local) as clocks:
         step_ev[0].record()
         for s in range(K):
+            warp_step(s)
             if per_level:
                 W = stepper.W
                 for l in range(L):
@@ -371,8 +393,12 @@ def main():
                        if resident_bytes > 256e6 else "inputs smaller than L2: timings are cache-assisted",
                        "drafting": ("rsd_sbs_step per level" if per_level else
                                     "rsd_sbs_draft_tree (all levels, rows ready)" if is_sbs else "rsd_gumbel_topk_draft"),
+                       "logit_warping": ({"top_k": args.top_k, "top_p": args.top_p,
+                                          "filter_ms_per_step": sum(a.elapsed_time(b) for a, b in filter_ev) / K,
+                                          "rows_filtered_per_step": B * (w.num_parents + w.num_nodes + 1)}
+                                         if warp_rows else None),
                        "mean_accepted_len": float(acc.mean())},
-            "clocks": clocks.summary(), "gpu_launches": stepper.kernel_launches * K, "roofline": roofline,
+            "clocks": clocks.summary(), "gpu_launches": (stepper.kernel_launches + (2 if warp_rows else 0)) * K, "roofline": roofline,
             "phases": phases,
             "step_ms": {"mean": elapsed_ms / K, "median": float(np.median(per_step_ms)), "best": float(np.min(per_step_ms)),
                         "note": "per-step CUDA-event times on this rank; `value` uses the mean (max over ranks)"},
@@ -383,15 +409,16 @@ def main():
     if not args.no_e2e:
         h_draft = torch.empty(draft.shape, dtype=draft.dtype, pin_memory=True)
         h_target = torch.empty(target.shape, dtype=target.dtype, pin_memory=True)
-        h_draft.copy_(draft)
-        h_target.copy_(target)
+        h_draft.copy_(raw_draft)
+        h_target.copy_(raw_target)
         res_host = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True)
                     for k, v in stepper.verify_out.items() if v is not None}
         Ke = max(1, args.e2e_steps)
 
         def e2e_step(s):
-            draft.copy_(h_draft, non_blocking=True)
-            target.copy_(h_target, non_blocking=True)
+            raw_draft.copy_(h_draft, non_blocking=True)
+            raw_target.copy_(h_target, non_blocking=True)
+            warp_step()
             o = stepper.run(draft, target, 0, 2000 + s, seq_base)
             for k2, v in res_host.items():
                 v.copy_(o[k2], non_blocking=True)

@@ -7,11 +7,14 @@
 //           shortest prefix whose share of the mass reaches top_p (at least one token)
 //
 // One block per row.  The row is copied to shared memory once; both cuts are then found without sorting: the value
-// of the last kept token by a 16-ary search over the ordered bit patterns of the values (each pass sorts the tokens
-// of the current interval into 16 equal sub-intervals and counts them, or sums their weights exp(value / T), in bins
-// private to each thread; four passes settle a 16-bit pattern, eight a 32-bit one), and the last kept token among
-// equal values by a prefix count in token order.  Sums are taken in a fixed order (per thread, over the threads of a
-// bin, over the bins), so the result does not depend on timing.
+// of the last kept token by a 16-ary search over the ordered bit patterns of the values.  Each pass sorts the tokens
+// of the current interval into 16 sub-intervals (equal steps in value while the interval is wide, which is where the
+// tokens spread evenly; equal steps in bit pattern once it is narrow) and counts them and sums their weights
+// exp(value / T) in bins private to each thread.  The first pass also gives the row's total mass.  As soon as the
+// interval holds few enough tokens their indices are gathered, in token order, and every later pass runs over that
+// short list instead of the row.  The last kept token among equal values comes from a prefix count in token order.
+// Sums are taken in a fixed order (per thread, over the threads of a bin, over the bins), so the result does not
+// depend on timing.
 #pragma once
 #include "rsd_device.cuh"
 #include "rsd_scan.cuh"   // ex2_approx, better()
@@ -20,8 +23,9 @@ namespace rsd {
 
 constexpr int kFilterThreads = 256;
 constexpr int kFilterWarps = kFilterThreads / 32;
-constexpr int kTrials = 2;                       // trial values a tally can take at once
 constexpr int kBins = 16;                        // sub-intervals per search pass
+constexpr int kListCap = 8192;                   // tokens gathered into a list (indices as 16 bits: rows up to 65,536)
+constexpr float kValueRange = 24.0f;             // value-linear bins cover this many nats of value / T below the interval's top
 
 struct FilterArgs {
     const void* data;
@@ -36,11 +40,13 @@ struct FilterArgs {
 };
 
 struct FilterSmem {
-    float bins[kBins][kFilterThreads];           // per-thread bins of a search pass (counts are stored as floats' bits)
-    double bin_total[kBins];
-    double red_d[kFilterWarps][kTrials];
-    int red_i[kFilterWarps][kTrials];
-    float red_f[kFilterWarps];
+    float mass[kBins][kFilterThreads];           // per-thread bins of a search pass
+    uint16_t count[kBins][kFilterThreads];
+    uint32_t bound[kBins + 1];                   // bin q holds the codes bound[q] .. bound[q + 1] - 1 (the last: .. hi)
+    double mass_total[kBins];
+    int count_total[kBins];
+    uint16_t list[kListCap];                     // indices of the tokens still in play, in token order
+    int red_i[kFilterWarps][2];
     int scan_i[kFilterWarps];
     int found;
     int nan_flag;
@@ -63,6 +69,7 @@ struct RowCodes<__nv_bfloat16> {
         return __uint_as_float(h << 16);
     }
     __device__ static __forceinline__ bool is_nan(const unsigned char* row, int i) { return (((const uint16_t*)row)[i] & 0x7FFFu) > 0x7F80u; }
+    __device__ static __forceinline__ uint32_t code_of_float(float v) { return code_of_bits(__float_as_uint(v) >> 16); }   // (truncated)
     static constexpr uint32_t kNegInfCode = 0x007Fu;                               // code of -inf (0xFF80)
     static constexpr uint32_t kNegInfBits = 0xFF80u;
 };
@@ -78,6 +85,7 @@ struct RowCodes<float> {
         return __uint_as_float((c & 0x80000000u) ? (c & 0x7FFFFFFFu) : ~c);
     }
     __device__ static __forceinline__ bool is_nan(const unsigned char* row, int i) { return (((const uint32_t*)row)[i] & 0x7FFFFFFFu) > 0x7F800000u; }
+    __device__ static __forceinline__ uint32_t code_of_float(float v) { return code_of_bits(__float_as_uint(v)); }
     static constexpr uint32_t kNegInfCode = 0x007FFFFFu;
     static constexpr uint32_t kNegInfBits = 0xFF800000u;
 };
@@ -96,115 +104,170 @@ struct RowFilter {
     const unsigned char* row;   // shared memory
     int V;
     float k, neg_c;             // weight of a value: 2^(value * k + neg_c)
+    int n_list;                 // >= 0: the tokens still in play are sm.list[0 .. n_list); -1: the whole row
 
     __device__ __forceinline__ float weight(uint32_t code) const { return ex2_approx(fmaf(RowCodes<T>::value_of_code(code), k, neg_c)); }
+    __device__ __forceinline__ int items() const { return n_list >= 0 ? n_list : V; }
+    __device__ __forceinline__ int index(int m) const { return n_list >= 0 ? (int)sm.list[m] : m; }
 
-    // For each of the trial codes t[0] < ... < t[n-1]: over the tokens within `inside` whose code is >= t[j], their number
-    // (WEIGH = false) or the sum of their weights (WEIGH = true).  Identical on all threads.
-    template <bool WEIGH>
-    __device__ __forceinline__ void tally(const uint32_t (&t)[kTrials], int n, const Cut& inside, double (&out)[kTrials]) {
+    // What the search found: the code t of the last kept value, the mass and the number of the tokens strictly above it,
+    // and the total mass of the tokens the search started from.
+    struct Found {
+        uint32_t t;
+        double above_mass;
+        int above_count;
+        double total_mass;
+    };
+
+    // The largest code t in [lo, hi] with F(t) >= need, F(t) = the number (BY_MASS = false) or the weight (BY_MASS = true)
+    // of the tokens within `inside` whose code is >= t.  need = need_abs, or, when need_abs < 0, need_frac times the
+    // total weight of the tokens within `inside` (they all lie in [lo, hi]: the first pass measures it).  F is
+    // non-increasing, F(lo) >= need, nothing within `inside` lies above hi.
+    template <bool BY_MASS>
+    __device__ __forceinline__ Found search(uint32_t lo, uint32_t hi, double need_abs, double need_frac, const Cut& inside) {
         const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-        float acc[kTrials];
-        int cnt[kTrials];
-#pragma unroll
-        for (int j = 0; j < kTrials; ++j) { acc[j] = 0.0f; cnt[j] = 0; }
-        for (int i = tid; i < V; i += kFilterThreads) {
-            const uint32_t code = RowCodes<T>::code(row, i);
-            if (!within(inside, code, i) || code <= RowCodes<T>::kNegInfCode) continue;
-            const float w = WEIGH ? weight(code) : 0.0f;
-#pragma unroll
-            for (int j = 0; j < kTrials; ++j) {
-                if (j < n && code >= t[j]) {
-                    if (WEIGH) acc[j] += w;
-                    else ++cnt[j];
+        Found r = {lo, 0.0, 0, 0.0};
+        double need = need_abs;
+        int level = 0;
+        for (;; ++level) {
+            // ---- the 16 sub-intervals ------------------------------------------------------------------------------------------
+            const uint32_t span = hi - lo;
+            const bool by_value = level < 2 && span > 4096u;
+            if (tid <= kBins) {
+                uint32_t bd;
+                if (tid == 0) bd = lo;
+                else if (tid == kBins) bd = hi;          // (unused as a lower bound; bin 15 ends at hi)
+                else if (by_value) {
+                    const float v_hi = RowCodes<T>::value_of_code(hi);
+                    const float v_lo = fmaxf(RowCodes<T>::value_of_code(lo), v_hi - kValueRange * kLog2e / k);
+                    const uint32_t c = RowCodes<T>::code_of_float(v_lo + (v_hi - v_lo) * (float)tid * (1.0f / kBins));
+                    bd = c <= lo ? lo + 1u : (c > hi ? hi : c);
+                } else {
+                    const int shift = max(0, 32 - __clz(span | 1u) - 4);      // (span >> shift) < 16
+                    const uint32_t c = lo + ((uint32_t)tid << shift);
+                    bd = (c < lo || c > hi) ? hi : c;                        // bins past the interval's end are empty ...
+                    if (c > hi || c < lo) bd = hi;                           // ... they all start at hi, and only the last holds it
                 }
+                sm.bound[tid] = bd;
             }
-        }
 #pragma unroll
-        for (int j = 0; j < kTrials; ++j) {
-            if (WEIGH) {
-                float v = acc[j];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-                if (lane == 0) sm.red_d[warp][j] = (double)v;
-            } else {
-                const int v = __reduce_add_sync(0xFFFFFFFFu, cnt[j]);
-                if (lane == 0) sm.red_i[warp][j] = v;
-            }
-        }
-        __syncthreads();
-#pragma unroll
-        for (int j = 0; j < kTrials; ++j) {
-            double s = 0.0;
-#pragma unroll
-            for (int w = 0; w < kFilterWarps; ++w) s += WEIGH ? sm.red_d[w][j] : (double)sm.red_i[w][j];   // fixed order
-            out[j] = s;
-        }
-        __syncthreads();
-    }
-
-    // The largest code t in [lo, hi] with F(t) >= need, where F(t) is the number (WEIGH = false) or the weight
-    // (WEIGH = true) of the tokens within `inside` whose code is >= t.  F is non-increasing; the caller guarantees
-    // F(lo) >= need and that nothing within `inside` lies above hi.  Also returns F(t + 1), the tally strictly above t.
-    template <bool WEIGH>
-    __device__ __forceinline__ uint32_t search(uint32_t lo, uint32_t hi, double need, const Cut& inside, double& above) {
-        const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-        above = 0.0;
-        while (lo < hi) {
-            const uint32_t span = hi - lo;                                   // >= 1
-            const int shift = max(0, 32 - __clz(span) - 4);                  // (span >> shift) < 16
-#pragma unroll
-            for (int q = 0; q < kBins; ++q) sm.bins[q][tid] = 0.0f;
-            for (int i = tid; i < V; i += kFilterThreads) {
+            for (int q = 0; q < kBins; ++q) { sm.mass[q][tid] = 0.0f; sm.count[q][tid] = 0; }
+            __syncthreads();
+            // bins that start at the same code: only the last of them is used (the search below takes the largest q)
+            const int n_items = items();
+            for (int m = tid; m < n_items; m += kFilterThreads) {
+                const int i = index(m);
                 const uint32_t code = RowCodes<T>::code(row, i);
                 if (code < lo || code > hi || !within(inside, code, i) || code <= RowCodes<T>::kNegInfCode) continue;
-                const int q = (int)((code - lo) >> shift);
-                if (WEIGH) sm.bins[q][tid] += weight(code);
-                else sm.bins[q][tid] = __int_as_float(__float_as_int(sm.bins[q][tid]) + 1);
+                int q = code >= sm.bound[8] ? 8 : 0;
+                q += code >= sm.bound[q + 4] ? 4 : 0;
+                q += code >= sm.bound[q + 2] ? 2 : 0;
+                q += code >= sm.bound[q + 1] ? 1 : 0;
+                if (q == kBins) q = kBins - 1;                               // code == hi == bound[16]
+                sm.mass[q][tid] += weight(code);
+                sm.count[q][tid] += 1;
             }
             __syncthreads();
-            // totals of the bins: warp w adds up bins 2 w and 2 w + 1, every lane eight threads' entries in order, then a
-            // fixed tree over the lanes
+            // ---- totals of the bins: warp w adds up bins 2 w and 2 w + 1, every lane eight threads' entries in order,
+            // then a fixed tree over the lanes ----------------------------------------------------------------------------------
 #pragma unroll
             for (int h = 0; h < kBins / kFilterWarps; ++h) {
                 const int q = warp * (kBins / kFilterWarps) + h;
                 double v = 0.0;
+                int c = 0;
 #pragma unroll
                 for (int e = 0; e < kFilterThreads / 32; ++e) {
-                    const float x = sm.bins[q][lane * (kFilterThreads / 32) + e];
-                    v += WEIGH ? (double)x : (double)__float_as_int(x);
+                    v += (double)sm.mass[q][lane * (kFilterThreads / 32) + e];
+                    c += (int)sm.count[q][lane * (kFilterThreads / 32) + e];
                 }
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-                if (lane == 0) sm.bin_total[q] = v;
+                c = __reduce_add_sync(0xFFFFFFFFu, c);
+                if (lane == 0) { sm.mass_total[q] = v; sm.count_total[q] = c; }
             }
             __syncthreads();
-            // from the top bin down: the first bin that brings the tally to `need` holds t
-            double run = above;
+            if (level == 0) {
+                double tot = 0.0;
+                for (int q = 0; q < kBins; ++q) tot += sm.mass_total[q];
+                r.total_mass = tot;
+                if (need_abs < 0.0) need = need_frac * tot;
+            }
+            // ---- from the top bin down: the first bin that brings the tally to `need` holds t ------------------------------
+            double run_m = r.above_mass;
+            int run_c = r.above_count;
             int pick = 0;
             for (int q = kBins - 1; q >= 0; --q) {
-                const double with_q = run + sm.bin_total[q];
-                if (with_q >= need) { pick = q; break; }
-                run = with_q;
+                const double f = BY_MASS ? run_m + sm.mass_total[q] : (double)(run_c + sm.count_total[q]);
+                if (f >= need) { pick = q; break; }
+                run_m += sm.mass_total[q];
+                run_c += sm.count_total[q];
             }
-            above = run;
-            const uint32_t new_lo = lo + ((uint32_t)pick << shift);
-            const uint32_t width = shift >= 32 ? 0xFFFFFFFFu : ((1u << shift) - 1u);
-            hi = (new_lo + width < new_lo || new_lo + width > hi) ? hi : new_lo + width;
-            lo = new_lo;
+            r.above_mass = run_m;
+            r.above_count = run_c;
+            const uint32_t new_lo = sm.bound[pick];
+            uint32_t new_hi = hi;
+            if (pick < kBins - 1) {
+                const uint32_t nb = sm.bound[pick + 1];
+                new_hi = nb > new_lo ? nb - 1u : new_lo;          // (an empty bin cannot be picked unless need <= what lies above)
+                if (nb <= new_lo) new_hi = new_lo;
+            }
+            const int population = sm.count_total[pick];
             __syncthreads();
+            lo = new_lo;
+            hi = new_hi;
+            if (lo >= hi) break;
+            // few enough tokens left: gather them, in token order, and go on over the list
+            if (n_list < 0 && population <= kListCap && V <= 65536) gather(lo, hi, inside);
         }
-        return lo;
+        r.t = lo;
+        return r;
     }
 
-    // Index of the j-th (1-based) token, in token order, that has code `code` and lies within `inside`; -1 if there are
-    // fewer.  Threads own consecutive runs of tokens; one prefix count over the block.
-    __device__ __forceinline__ int nth_with_code(uint32_t code, int j, const Cut& inside) {
+    // The indices of the tokens within `inside` with a code in [lo, hi], in token order, into sm.list.
+    __device__ __forceinline__ void gather(uint32_t lo, uint32_t hi, const Cut& inside) {
         const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
         const int per = (V + kFilterThreads - 1) / kFilterThreads;
         const int i0 = tid * per, i1 = min(V, i0 + per);
         int mine = 0;
-        for (int i = i0; i < i1; ++i) mine += (RowCodes<T>::code(row, i) == code && within(inside, code, i)) ? 1 : 0;
+        for (int i = i0; i < i1; ++i) {
+            const uint32_t code = RowCodes<T>::code(row, i);
+            mine += (code >= lo && code <= hi && within(inside, code, i) && code > RowCodes<T>::kNegInfCode) ? 1 : 0;
+        }
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (lane == 31) sm.scan_i[warp] = incl;
+        __syncthreads();
+        int at = incl - mine, total = 0;
+        for (int w = 0; w < kFilterWarps; ++w) {
+            if (w < warp) at += sm.scan_i[w];
+            total += sm.scan_i[w];
+        }
+        if (total <= kListCap) {
+            for (int i = i0; i < i1; ++i) {
+                const uint32_t code = RowCodes<T>::code(row, i);
+                if (code >= lo && code <= hi && within(inside, code, i) && code > RowCodes<T>::kNegInfCode) sm.list[at++] = (uint16_t)i;
+            }
+        }
+        __syncthreads();
+        if (total <= kListCap) n_list = total;
+    }
+
+    // Number of the tokens in play that have code `code` and lie within `inside`, and the index of the j-th (1-based) of
+    // them in token order (-1 if there are fewer).  Threads own consecutive runs; one prefix count over the block.
+    __device__ __forceinline__ int nth_with_code(uint32_t code, int j, const Cut& inside, int& how_many) {
+        const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+        const int n_items = items();
+        const int per = (n_items + kFilterThreads - 1) / kFilterThreads;
+        const int m0 = tid * per, m1 = min(n_items, m0 + per);
+        int mine = 0;
+        for (int m = m0; m < m1; ++m) {
+            const int i = index(m);
+            mine += (RowCodes<T>::code(row, i) == code && within(inside, code, i)) ? 1 : 0;
+        }
         int incl = mine;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -214,11 +277,16 @@ struct RowFilter {
         if (lane == 31) sm.scan_i[warp] = incl;
         if (tid == 0) sm.found = -1;
         __syncthreads();
-        int before = incl - mine;
-        for (int w = 0; w < warp; ++w) before += sm.scan_i[w];
+        int before = incl - mine, total = 0;
+        for (int w = 0; w < kFilterWarps; ++w) {
+            if (w < warp) before += sm.scan_i[w];
+            total += sm.scan_i[w];
+        }
+        how_many = total;
         if (mine > 0 && before < j && j <= before + mine) {
             int seen = before;
-            for (int i = i0; i < i1; ++i) {
+            for (int m = m0; m < m1; ++m) {
+                const int i = index(m);
                 if (RowCodes<T>::code(row, i) == code && within(inside, code, i) && ++seen == j) { sm.found = i; break; }
             }
         }
@@ -276,49 +344,39 @@ __global__ void __launch_bounds__(kFilterThreads) filter_rows_kernel(const Filte
 
     const float vmax = RowCodes<T>::value_of_code(top);
     const bool plus_inf = vmax == -kNegInf;                       // a +inf entry: it alone carries the mass
-    RowFilter<T> f = {sm, row_sm, V, a.log2e_over_t, (finite > 0 && !plus_inf) ? -vmax * a.log2e_over_t : 0.0f};
+    RowFilter<T> f = {sm, row_sm, V, a.log2e_over_t, (finite > 0 && !plus_inf) ? -vmax * a.log2e_over_t : 0.0f, -1};
     Cut cut = {RowCodes<T>::kNegInfCode, V};                      // everything finite
     int kept = finite;
 
     // ---- top-k: the value of the k-th largest entry, then the last kept token among its equals -------------------------
     if (a.top_k > 0 && a.top_k < V && finite > a.top_k) {
-        double above;
-        const uint32_t t = f.template search<false>(RowCodes<T>::kNegInfCode + 1u, top, (double)a.top_k, cut, above);
-        const int j = a.top_k - (int)above;                      // that many of the entries equal to t are kept
-        const int tok = f.nth_with_code(t, j, cut);
-        cut.code = t;
+        const typename RowFilter<T>::Found r = f.template search<false>(RowCodes<T>::kNegInfCode + 1u, top, (double)a.top_k, 0.0, cut);
+        int ties;
+        const int tok = f.nth_with_code(r.t, a.top_k - r.above_count, cut, ties);   // that many of the entries equal to t stay
+        cut.code = r.t;
         cut.tok = tok >= 0 ? tok : V;
         kept = a.top_k;
+        f.n_list = -1;                                            // (the list was gathered for the old cut)
     }
     // ---- top-p: of what is left, the shortest prefix (value descending, token ascending) whose mass reaches top_p -------
     if (a.top_p > 0.0f && a.top_p < 1.0f && kept > 0 && !plus_inf) {
-        uint32_t t1[kTrials];
-        double tot[kTrials];
-        t1[0] = cut.code;                                         // (every entry within the cut has a code >= cut.code)
-        f.template tally<true>(t1, 1, cut, tot);
-        const double need = (double)a.top_p * tot[0];
-        double above;
-        const uint32_t t = f.template search<true>(cut.code, top, need, cut, above);
+        const typename RowFilter<T>::Found r = f.template search<true>(cut.code, top, -1.0, (double)a.top_p, cut);
+        const double need = (double)a.top_p * r.total_mass;
         // entries equal to t within the cut: each weighs w; the first j of them (token order) complete the prefix
-        double ties_d[kTrials];
-        uint32_t tt[kTrials];
-        tt[0] = t;
-        tt[1] = t + 1u;
-        f.template tally<false>(tt, t == 0xFFFFFFFFu ? 1 : 2, cut, ties_d);
-        const int ties = (int)(ties_d[0] - (t == 0xFFFFFFFFu ? 0.0 : ties_d[1]));
-        const double w = (double)f.weight(t);
+        int ties;
+        f.nth_with_code(r.t, 1, cut, ties);
+        const double w = (double)f.weight(r.t);
         int j = ties;
         if (w > 0.0) {
-            const double want = ceil((need - above) / w);
+            const double want = ceil((need - r.above_mass) / w);
             j = want < 1.0 ? 1 : (want > (double)ties ? ties : (int)want);
-            while (j > 1 && above + (double)(j - 1) * w >= need) --j;
-            while (j < ties && above + (double)j * w < need) ++j;
+            while (j > 1 && r.above_mass + (double)(j - 1) * w >= need) --j;
+            while (j < ties && r.above_mass + (double)j * w < need) ++j;
         }
-        const int tok = f.nth_with_code(t, j, cut);
-        const int n_above = t == 0xFFFFFFFFu ? 0 : (int)ties_d[1];
-        cut.code = t;
+        const int tok = f.nth_with_code(r.t, j, cut, ties);
+        cut.code = r.t;
         cut.tok = tok >= 0 ? tok : V;
-        kept = n_above + j;
+        kept = r.above_count + j;
     }
 
     // ---- the row with -inf at the filtered entries ------------------------------------------------------------------------------
