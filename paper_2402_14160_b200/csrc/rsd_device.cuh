@@ -109,6 +109,51 @@ __device__ __forceinline__ void ld_stream_256(const void* p, uint4& lo, uint4& h
                  : "l"(p));
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// mbarrier and bulk copy (global -> this block's shared memory; this GPU's own memory, no cluster, no multicast)
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// `bytes` a multiple of 16, both addresses 16-byte aligned; completion counts on `bar`
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+constexpr long long kCopyWaitCycles = 1ll << 31;   // about a second: a copy that has not landed by then never will
+// Wait for phase `parity` of `bar`, at most about a second.  A wait that runs out sets *gave_up and returns: the caller
+// goes on with whatever the memory holds and reports RSD_ST_TIMEOUT at its next decision point.
+__device__ __forceinline__ void wait_bar(unsigned long long* bar, uint32_t parity, int* gave_up) {
+    if (mbar_try_wait(bar, parity)) return;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kCopyWaitCycles) {
+            *gave_up = 1;
+            return;
+        }
+    }
+}
+
 template <typename T>
 struct RowIO;
 

@@ -37,7 +37,6 @@ constexpr int kTileElems = 512;                   // one warp-wide step: 16 elem
 constexpr int kMaxRingChunks = 64;                // chunks per row the ring's bookkeeping covers (one bit each)
 constexpr int kMaxRemovedRing = 64;               // rejected tokens remembered per node (to recognise a repeated sibling)
 constexpr float kSumFloor = 8.673617379884035e-19f;   // 2^-60: a normaliser below this has lost its small terms to underflow
-constexpr long long kWaitCycles = 1ll << 31;      // about a second: a copy that has not landed by then never will
 constexpr int kRingBytes = kSlots * 2 * kRowChunkBytes;
 
 // What the working warps do next (written by the control warp, read after a block barrier).
@@ -61,48 +60,6 @@ struct RingSmem {
     int nan_seen;                                 // a cleaning pass met a NaN
     int abort;                                    // a wait ran out: the walk is abandoned and reported
 };
-
-// ---- mbarrier / bulk copy (this GPU's own memory; no cluster, no multicast) -------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// global -> shared, `bytes` a multiple of 16, both addresses 16-byte aligned; completion counts on `bar`
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(dst)),
-                 "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
-// Wait for phase `parity` of `bar`, at most about a second.  A wait that runs out sets *abort and returns: the
-// caller goes on with whatever the slot holds and the walk is abandoned at the next block-wide decision point.
-__device__ __forceinline__ void wait_bar(unsigned long long* bar, uint32_t parity, int* abort) {
-    if (mbar_try_wait(bar, parity)) return;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > kWaitCycles) {
-            *abort = 1;
-            return;
-        }
-    }
-}
 
 // A lane's 16 values of a 512-element tile in shared memory: the 16-byte pieces lane, lane + 32, ... of the tile
 // (conflict-free 128-bit loads).  Which elements a lane sums does not matter; the one place that needs token order
