@@ -29,9 +29,9 @@ import workloads  # noqa: E402
 # DRAM bytes moved per algorithmic byte by the scan kernel, from the committed ncu summary of the scan kernel
 # (dram__bytes_read + dram__bytes_write over rows x V x 2 bytes; the traffic grows in proportion to the rows scanned),
 # together with the SHA-256 of the kernel sources it was measured on: when the sources differ, `traffic` is null.
-SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.042
+SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.012
 SCAN_TRAFFIC_SOURCES = ("paper_2402_14160_b200/csrc/rsd_scan.cuh", "paper_2402_14160_b200/csrc/rsd_device.cuh")
-SCAN_TRAFFIC_SOURCE_SHA256 = "@@SCAN_SHA@@"
+SCAN_TRAFFIC_SOURCE_SHA256 = "0ad4f3a8a91fc861805a8345e9affd3d0e9078dee366a6b41505a02def29b3f6"
 
 
 def _scan_sources_sha256():
@@ -367,7 +367,8 @@ def main():
                 "traffic": (SCAN_TRAFFIC_PER_ALGORITHMIC_BYTE * scan_bytes_per_step / n_scan
                             if _scan_sources_sha256() == SCAN_TRAFFIC_SOURCE_SHA256 else None),
                 "traffic_note": "DRAM bytes per scan launch (average over the step's launches), scaled by rows from a "
-                                "256-sequence ncu capture; null when the kernel sources changed since that capture",
+                                "256-sequence ncu capture (14,592 rows in one launch); null when the kernel sources "
+                                "changed since that capture",
                 "algorithmic_bytes_per_step": scan_bytes_per_step,
                 "launches_per_step": n_scan, "avg_launch_ms": scan_ms / (K * n_scan),
                 "launch_ms_by_level": [sum(scan_ev[s][l][0].elapsed_time(scan_ev[s][l][1]) for s in range(K)) / K
