@@ -165,6 +165,23 @@ struct Packed<float> {
 #pragma unroll
         for (int i = 0; i < 4; ++i) w[i] = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
     }
+    static __device__ __forceinline__ uint32_t clean_word(uint32_t q) {
+        return (q & 0x7FFFFFFFu) > 0x7F800000u ? 0xFF800000u : q;
+    }
+    __device__ __forceinline__ void clean_nan() {   // NaN elements become -inf
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            w[i] = make_uint4(clean_word(w[i].x), clean_word(w[i].y), clean_word(w[i].z), clean_word(w[i].w));
+    }
+    // f(pair) for the 8 pairs of neighbouring values, as packed fp32, in order
+    template <typename F>
+    __device__ __forceinline__ void for_each_pair(F f) const {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f(f32x2(__uint_as_float(w[i].x), __uint_as_float(w[i].y)));
+            f(f32x2(__uint_as_float(w[i].z), __uint_as_float(w[i].w)));
+        }
+    }
     __device__ __forceinline__ void load_aligned(const void* group, bool wide) {  // 64 bytes, 16- or 32-byte aligned
         if (wide) {
             ld_stream_256(group, w[0], w[1]);
@@ -205,6 +222,26 @@ struct Packed<__nv_bfloat16> {
     }
     __device__ __forceinline__ void fill_neg_inf() {
         w[0] = w[1] = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+    }
+    static __device__ __forceinline__ uint32_t clean_word(uint32_t q) {
+        if ((q & 0x7FFFu) > 0x7F80u) q = (q & 0xFFFF0000u) | 0xFF80u;
+        if ((q & 0x7FFF0000u) > 0x7F800000u) q = (q & 0xFFFFu) | 0xFF800000u;
+        return q;
+    }
+    __device__ __forceinline__ void clean_nan() {   // NaN elements become -inf
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+            w[i] = make_uint4(clean_word(w[i].x), clean_word(w[i].y), clean_word(w[i].z), clean_word(w[i].w));
+    }
+    // f(pair) for the 8 pairs of neighbouring values, as packed fp32, in order
+    template <typename F>
+    __device__ __forceinline__ void for_each_pair(F f) const {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const uint32_t q[4] = {w[i].x, w[i].y, w[i].z, w[i].w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) f(f32x2(__uint_as_float(q[j] << 16), __uint_as_float(q[j] & 0xFFFF0000u)));
+        }
     }
     __device__ __forceinline__ void load_aligned(const void* group, bool wide) {  // 32 bytes, 16- or 32-byte aligned
         if (wide) {
@@ -405,7 +442,7 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
     unsigned long long acc0 = f32x2(0.0f, 0.0f), acc1 = acc0;
     const uint32_t slot = (uint32_t)__cvta_generic_to_shared(shared_buf) + (uint32_t)tid * GroupSlot<T>::kStride;
     // work on one group whose 16 values are in `cur`; `word` is the group's coarse-stream word, `ub_g` = &ub[group]
-    auto body = [&](const Packed<T>& cur, float* ub_g, uint32_t word) {
+    auto body = [&](Packed<T>& cur, float* ub_g, uint32_t word) {   // may rewrite cur
         slot_store(slot, cur);
         float g_lo, g_hi;
         group_noise_bounds(word >> 4, g_lo, g_hi);
@@ -413,16 +450,12 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
         *ub_g = fmaf(gmax, inv_temp, g_hi);                    // NaN if the group holds a NaN: looked at later
         best = fmaxf(best, fmaf(slot_element<T>(slot, word & 15u), inv_temp, g_lo));  // fmaxf drops NaN
         if (NEED_LSE) {
-            float v[16];
-            cur.unpack(v);
+            // The sums are taken straight from the packed words, a pair at a time, so that no more than a few unpacked
+            // values are alive at once; the rare cases below rewrite the group in place first.
             if (!(gmax <= lse_thr)) {  // rare: a NaN in the group, the first finite group, or a jump of more than 40
                 if (gmax != gmax) {    // NaN counts as -inf
-                    gmax = kNegInf;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        if (v[j] != v[j]) v[j] = kNegInf;
-                        gmax = fmaxf(gmax, v[j]);
-                    }
+                    cur.clean_nan();
+                    gmax = group_max_nan(cur);
                 }
                 if (gmax > lse_thr) {
                     const float c_new = ceilf(gmax * log2e_t);
@@ -437,14 +470,15 @@ __global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanAr
                 }
             }
             const unsigned long long l2 = f32x2(log2e_t, log2e_t), c2 = f32x2(lse_negc, lse_negc);
-#pragma unroll
-            for (int j = 0; j < 16; j += 4) {  // two elements per fma / add, two accumulators
-                float e0, e1, e2, e3;
-                split_f32x2(fma_f32x2(f32x2(v[j], v[j + 1]), l2, c2), e0, e1);
-                split_f32x2(fma_f32x2(f32x2(v[j + 2], v[j + 3]), l2, c2), e2, e3);
-                acc0 = add_f32x2(acc0, f32x2(ex2_approx(e0), ex2_approx(e1)));
-                acc1 = add_f32x2(acc1, f32x2(ex2_approx(e2), ex2_approx(e3)));
-            }
+            int turn = 0;
+            cur.for_each_pair([&](unsigned long long p) {   // two elements per fma / add, two accumulators in turn
+                float e0, e1;
+                split_f32x2(fma_f32x2(p, l2, c2), e0, e1);
+                const unsigned long long x = f32x2(ex2_approx(e0), ex2_approx(e1));
+                if (turn & 1) acc1 = add_f32x2(acc1, x);
+                else acc0 = add_f32x2(acc0, x);
+                ++turn;
+            });
         }
     };
     // Two buffers: the group two turns ahead is requested as soon as a buffer has been consumed.  Chunks that lie
