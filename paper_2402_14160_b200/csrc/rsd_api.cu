@@ -175,7 +175,7 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
 
     rsd::SbsEpilogueArgs e;
     e.n_par = n_par; e.W = W; e.is_logprob = rows_are_logprob(draft_level);
-    e.fin_seq_stride = (int64_t)n_par * W; e.row_seq_stride = n_par; e.state_stride = n_par; e.inv_temp = 1.0 / (double)temperature_of(draft_level); e.first_parent_node = first_parent_node;
+    e.fin_seq_stride = (int64_t)n_par * W; e.row_seq_stride = n_par; e.state_stride = n_par; e.out_state_stride = W; e.inv_temp = 1.0 / (double)temperature_of(draft_level); e.first_parent_node = first_parent_node;
     e.seed_lo = (uint32_t)seed; e.seed_hi = (uint32_t)(seed >> 32); e.step = step; e.seq_base = seq_base;
     e.fin_token = fin_token; e.fin_value = fin_value; e.fin_pert = fin_pert; e.fin_lse = fin_lse;
     e.row_status = row_status;
@@ -183,7 +183,7 @@ int rsd_sbs_step(const rsd_rows* draft_level, int B, int n_par, int V, int W, in
     e.out_token = out_token; e.out_parent = out_parent; e.out_stride = out_stride; e.parent_base = parent_base;
     e.sum_out = sum_logprob_out; e.gamma_out = trunc_gumbel_out;
     e.out_count = out_count; e.status = status;
-    const size_t smem = (size_t)n_par * W * (8 + 8 + 4) + (size_t)n_par * 4;
+    const size_t smem = rsd::sbs_level_scratch_bytes(n_par, W);
     rsd::sbs_epilogue_kernel<<<B, rsd::kEpilogueThreads, smem, s>>>(e);
     return check_launch("rsd_sbs_step(epilogue)");
 }
@@ -294,12 +294,12 @@ int rsd_sbs_draft_tree(const rsd_rows* draft, int B, int V, int W, int L, uint64
     c.lvl.fin_token = fin_token; c.lvl.fin_value = fin_value; c.lvl.fin_pert = fin_pert; c.lvl.fin_lse = fin_lse;
     c.lvl.row_status = row_status;
     c.L = L; c.P = (int)P; c.B = B;
-    c.state_sum[0] = (float*)st0; c.state_gamma[0] = (float*)(st0 + s4);
-    c.state_sum[1] = (float*)(st0 + 2 * s4); c.state_gamma[1] = (float*)(st0 + 3 * s4);
     c.node_token = node_token; c.node_parent = node_parent; c.node_stride = node_stride;
     c.level_count = level_count; c.level_status = level_status; c.status = status;
     c.sum_out = sum_logprob_out; c.gamma_out = trunc_gumbel_out;
-    const size_t smem = (size_t)W * W * (8 + 8 + 4) + (size_t)W * 4;
+    // the finalists of a sequence are staged in shared memory when they fit well inside the default 48 KB
+    c.staged = rsd::sbs_chain_smem_bytes(W, (int)P, true) <= 40 * 1024 ? 1 : 0;
+    const size_t smem = rsd::sbs_chain_smem_bytes(W, (int)P, c.staged != 0);
     rsd::sbs_chain_kernel<<<B, rsd::kEpilogueThreads, smem, s>>>(c);
     return check_launch("rsd_sbs_draft_tree(levels)");
 }

@@ -811,6 +811,7 @@ struct SbsEpilogueArgs {
     int64_t fin_seq_stride;    // elements between sequences in fin_token / fin_value / fin_pert (n_par * W for one level)
     int64_t row_seq_stride;    // elements between sequences in fin_lse / row_status (n_par for one level)
     int64_t state_stride;      // elements between sequences in sum_in / gamma_in (n_par for one level)
+    int64_t out_state_stride;  // elements between sequences in sum_out / gamma_out (W; 0 when they hold one sequence)
     double inv_temp;           // 1 / temperature of the parents' rows (1: none)
     int32_t first_parent_node;
     uint32_t seed_lo, seed_hi, step, seq_base;
@@ -833,34 +834,56 @@ struct SbsEpilogueArgs {
 
 constexpr int kEpilogueThreads = 128;
 
-// One level for sequence b, by a block of kEpilogueThreads threads; sm_d: (n_par * W) * 20 + n_par * 4 bytes.
+// bytes of shared memory one level needs in sbs_epilogue_body, rounded up to 16
+__host__ __device__ inline size_t sbs_level_scratch_bytes(int n_par, int W) {
+    return (((size_t)n_par * W * 32 + (size_t)n_par * 12) + 15) & ~(size_t)15;
+}
+
+// order-preserving map of a double to an unsigned integer (for an atomic maximum), and back; 0 stands for "none"
+__device__ __forceinline__ unsigned long long double_to_ordered(double v) {
+    const unsigned long long u = (unsigned long long)__double_as_longlong(v);
+    return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+}
+__device__ __forceinline__ double ordered_to_double(unsigned long long k) {
+    if (k == 0) return -__longlong_as_double(0x7FF0000000000000LL);
+    return __longlong_as_double((long long)((k >> 63) ? (k & 0x7FFFFFFFFFFFFFFFull) : ~k));
+}
+
+// One level for sequence b, by a block of kEpilogueThreads threads; sm_d: sbs_level_scratch_bytes(n_par, W) bytes.
 __device__ __forceinline__ void sbs_epilogue_body(const SbsEpilogueArgs& a, const int b, double* sm_d) {
     const int F = a.n_par * a.W;
-    double* s_val = sm_d;             // [F] phi~ then psi
-    double* s_phi = sm_d + F;         // [F] phi
-    int* s_tok = (int*)(sm_d + 2 * F);
+    // the finalists that pass the first test are gathered in a list; entry i of the arrays below belongs to list[i]
+    double* s_pert = sm_d;                   // [F] phi~
+    double* s_phi = sm_d + F;                // [F] phi
+    double* s_psi = sm_d + 2 * F;            // [F] psi
+    unsigned long long* s_z = (unsigned long long*)(sm_d + 3 * F);   // [n_par] largest phi~ of the parent, ordered
+    int* s_list = (int*)(s_z + a.n_par);     // [F] finalist index f = parent * W + place
+    int* s_tok = s_list + F;                 // [F] its token
+    float* s_gam = (float*)(s_tok + F);      // [n_par]
     const int tid = threadIdx.x;
     const int64_t fin_off = (int64_t)b * a.fin_seq_stride, row_off = (int64_t)b * a.row_seq_stride,
                   state_off = (int64_t)b * a.state_stride;
     const RngKey key = {a.seed_lo, a.seed_hi, a.step, a.seq_base + (uint32_t)b};
-    const double ninf = -__longlong_as_double(0x7FF0000000000000LL);
 
     // A child enters the beam only if its psi reaches the W-th best psi of the level.  The best child of parent j has
     // psi = Gamma_j exactly, so that bound is at least L = the W-th largest Gamma among the parents that deliver a
     // child (valid parent, at least one finalist); L = -inf when fewer than W do.  Finalists that a cheap fp32 test
     // shows to lie clearly below L are dropped before the double-precision work; a parent's best finalist is
-    // always kept (it defines Z).
-    float* s_gam = (float*)(s_tok + F);   // [n_par]
+    // always kept.
     __shared__ float s_L;
-    if (tid == 0) s_L = kNegInf;
+    __shared__ int s_row_bits, s_n;
+    if (tid == 0) { s_L = kNegInf; s_row_bits = 0; s_n = 0; }
     for (int kp = tid; kp < a.n_par; kp += kEpilogueThreads) {
         const float sg = a.sum_in ? a.sum_in[state_off + kp] : 0.0f;
         const float gm = a.gamma_in ? a.gamma_in[state_off + kp] : 0.0f;
+        // a parent slot that the level above left empty (its sum or truncated Gumbel is -inf) has no children
         const bool delivers = a.fin_token[fin_off + (int64_t)kp * a.W] >= 0 && sg > kNegInf && gm > kNegInf;
         s_gam[kp] = delivers ? gm : kNegInf;
+        s_z[kp] = 0;
     }
     __syncthreads();
     for (int kp = tid; kp < a.n_par; kp += kEpilogueThreads) {
+        if (const int bits = a.row_status[row_off + kp]) atomicOr(&s_row_bits, bits);
         const float g = s_gam[kp];
         int rank = 0;
         for (int j = 0; j < a.n_par; ++j) {
@@ -875,9 +898,7 @@ __device__ __forceinline__ void sbs_epilogue_body(const SbsEpilogueArgs& a, cons
     for (int f = tid; f < F; f += kEpilogueThreads) {
         const int kpar = f / a.W;
         int x = a.fin_token[fin_off + f];
-        // a parent slot that the level above left empty (its sum or truncated Gumbel is -inf) has no children
-        // (s_gam is -inf exactly for the slots that deliver nothing)
-        if (s_gam[kpar] == kNegInf) x = -1;
+        if (s_gam[kpar] == kNegInf) x = -1;   // s_gam is -inf exactly for the slots that deliver nothing
         if (x >= 0 && L > kNegInf && f != kpar * a.W) {
             // psi_f < L  <=>  exp(-phi~_f) - exp(-Z) > exp(-L) - exp(-Gamma_k), with Z - phi~_f = the gap d between
             // the parent's best and this finalist's fp32 perturbed values; margins cover the fp32 arithmetic
@@ -892,87 +913,76 @@ __device__ __forceinline__ void sbs_epilogue_body(const SbsEpilogueArgs& a, cons
                 if (rhs <= 0.0f || -z + logf(expm1f(d_lo)) > logf(rhs) + 1e-2f) x = -1;   // cannot reach the beam
             }
         }
-        double phi = ninf, pert = ninf;
-        if (x >= 0) {
-            const double sigma = a.sum_in ? (double)a.sum_in[state_off + kpar] : 0.0;
-            const double lse = a.is_logprob ? 0.0 : (double)a.fin_lse[row_off + kpar];
-            const uint32_t node = (uint32_t)(a.first_parent_node + kpar);
-            const uint32_t word = coarse_word(key, node, (uint32_t)x >> 4);
-            const double t_elem = (((uint32_t)x & 15u) != (word & 15u))
-                                      ? neg_log_uniform_f64(fine_word(key, node, (uint32_t)x)) : 0.0;
-            phi = sigma + ((double)a.fin_value[fin_off + f] * a.inv_temp - lse);
-            pert = phi - log(neg_log_group_uniform_f64(word) * 0.0625 + t_elem);
-        }
-        s_tok[f] = x;
-        s_phi[f] = phi;
-        s_val[f] = pert;
+        if (x >= 0) s_list[atomicAdd(&s_n, 1)] = f;   // the order of the list does not matter below
     }
     __syncthreads();
-    // psi of every finalist (Z = the parent's largest phi~)
-    double my_psi[8];  // up to 8 finalists per thread: F <= 1024
-    int n_mine = 0;
-    for (int f = tid; f < F; f += kEpilogueThreads, ++n_mine) {
-        const int kpar = f / a.W;
-        double z = ninf;
-        for (int i = 0; i < a.W; ++i) z = fmax(z, s_val[kpar * a.W + i]);
+    const int n = s_n;
+
+    // phi and phi~ of the listed finalists, with the noise recomputed in double; Z = the parent's largest phi~
+    for (int i = tid; i < n; i += kEpilogueThreads) {
+        const int f = s_list[i], kpar = f / a.W;
+        const int x = a.fin_token[fin_off + f];
+        const double sigma = a.sum_in ? (double)a.sum_in[state_off + kpar] : 0.0;
+        const double lse = a.is_logprob ? 0.0 : (double)a.fin_lse[row_off + kpar];
+        const uint32_t node = (uint32_t)(a.first_parent_node + kpar);
+        const uint32_t word = coarse_word(key, node, (uint32_t)x >> 4);
+        const double t_elem = (((uint32_t)x & 15u) != (word & 15u))
+                                  ? neg_log_uniform_f64(fine_word(key, node, (uint32_t)x)) : 0.0;
+        const double phi = sigma + ((double)a.fin_value[fin_off + f] * a.inv_temp - lse);
+        const double pert = phi - log(neg_log_group_uniform_f64(word) * 0.0625 + t_elem);
+        s_tok[i] = x;
+        s_phi[i] = phi;
+        s_pert[i] = pert;
+        atomicMax(&s_z[kpar], double_to_ordered(pert));
+    }
+    __syncthreads();
+    for (int i = tid; i < n; i += kEpilogueThreads) {
+        const int kpar = s_list[i] / a.W;
+        const double z = ordered_to_double(s_z[kpar]);
         const double gamma = a.gamma_in ? (double)a.gamma_in[state_off + kpar] : 0.0;
-        const double pert = s_val[f];
-        double psi = ninf;
-        if (s_tok[f] >= 0) {
-            const double d = pert - z;
-            if (d >= 0.0) psi = gamma;
-            else {
-                const double w = log1p(-exp(d));
-                const double v = gamma - pert + w;
-                psi = gamma - fmax(v, 0.0) - log1p(exp(-fabs(v)));
-            }
+        const double pert = s_pert[i];
+        const double d = pert - z;
+        double psi = gamma;
+        if (!(d >= 0.0)) {
+            const double w = log1p(-exp(d));
+            const double v = gamma - pert + w;
+            psi = gamma - fmax(v, 0.0) - log1p(exp(-fabs(v)));
         }
-        my_psi[n_mine] = psi;
+        s_psi[i] = psi;
     }
     __syncthreads();
-    n_mine = 0;
-    for (int f = tid; f < F; f += kEpilogueThreads, ++n_mine) s_val[f] = my_psi[n_mine];
-    __syncthreads();
-    int valid_here = 0;
-    for (int f = tid; f < F; f += kEpilogueThreads) {
-        const int x = s_tok[f];
-        if (x < 0) continue;
-        ++valid_here;
-        const double psi = s_val[f];
+    // Rank by (psi desc, parent asc, token asc); the finalists of a parent are neighbours in f, so f orders the
+    // parents, and within a parent the token decides.
+    for (int i = tid; i < n; i += kEpilogueThreads) {
+        const double psi = s_psi[i];
+        const int f = s_list[i], x = s_tok[i], kpar = f / a.W;
+        const int own = kpar * a.W;   // first finalist of f's parent
         int rank = 0;
-        for (int e = 0; e < F; ++e) {
-            if (s_tok[e] < 0) continue;
-            const double pe = s_val[e];
-            // order: psi desc, then parent asc, then token asc; e's parent <= f's parent iff e / W <= f / W
-            const bool e_first = pe > psi || (pe == psi && (e / a.W < f / a.W || (e / a.W == f / a.W && s_tok[e] < x)));
-            rank += e_first ? 1 : 0;
+#pragma unroll 4
+        for (int e = 0; e < n; ++e) {
+            const double pe = s_psi[e];
+            const int fe = s_list[e];
+            const bool tie_first = fe < own || (fe < own + a.W && s_tok[e] < x);   // earlier parent, or same parent and smaller token
+            rank += (pe > psi || (pe == psi && tie_first)) ? 1 : 0;
         }
         if (rank < a.W) {
-            const int64_t o = (int64_t)b * a.W + rank;
+            const int64_t o = (int64_t)b * a.out_state_stride + rank;
             a.out_token[(int64_t)b * a.out_stride + rank] = x;
-            a.out_parent[(int64_t)b * a.out_stride + rank] = a.parent_base + f / a.W;
-            a.sum_out[o] = (float)s_phi[f];
+            a.out_parent[(int64_t)b * a.out_stride + rank] = a.parent_base + kpar;
+            a.sum_out[o] = (float)s_phi[i];
             a.gamma_out[o] = (float)psi;
         }
     }
-    __shared__ int s_cnt;
-    if (tid == 0) s_cnt = 0;
-    __syncthreads();
-    if (valid_here) atomicAdd(&s_cnt, valid_here);
-    __syncthreads();
-    const int cnt = s_cnt < a.W ? s_cnt : a.W;
+    const int cnt = n < a.W ? n : a.W;
     if (tid >= cnt && tid < a.W) {
-        const int64_t o = (int64_t)b * a.W + tid;
+        const int64_t o = (int64_t)b * a.out_state_stride + tid;
         a.out_token[(int64_t)b * a.out_stride + tid] = -1;
         a.out_parent[(int64_t)b * a.out_stride + tid] = -1;
         a.sum_out[o] = kNegInf;
         a.gamma_out[o] = kNegInf;
     }
-    int row_bits = 0;
-    for (int kp = tid; kp < a.n_par; kp += kEpilogueThreads) row_bits |= a.row_status[row_off + kp];
-    row_bits = __syncthreads_or(row_bits);
     if (tid == 0) {
-        a.status[b] = (row_bits & 1) | (cnt < a.W ? 2 : 0);  // RSD_ST_NAN_INPUT, RSD_ST_FEWER_THAN_K
+        a.status[b] = (s_row_bits & 1) | (cnt < a.W ? 2 : 0);  // RSD_ST_NAN_INPUT, RSD_ST_FEWER_THAN_K
         a.out_count[b] = cnt;
     }
 }
@@ -986,14 +996,15 @@ static __global__ void __launch_bounds__(kEpilogueThreads) sbs_epilogue_kernel(c
 // All L levels of one Stochastic Beam Search tree (Algorithm 8's level loop around Algorithm 9) for rows that exist
 // before drafting starts: the parent rows of every level were scanned in one launch (row r of a sequence is flat node
 // r: the root, then W slots per level), and this kernel runs the levels' epilogues in order, one block per sequence.
-// The sequence log-probabilities and truncated Gumbels (Eqs. 10-12) travel from level to level through two [B][W]
-// arrays used in turn; level l writes the tokens and parents of flat nodes 1 + l W .. (l + 1) W.
+// The sequence log-probabilities and truncated Gumbels (Eqs. 10-12) travel from level to level through two pairs of
+// W-element arrays in shared memory used in turn; level l writes the tokens and parents of flat nodes
+// 1 + l W .. (l + 1) W.  When `staged` is set the sequence's finalists (P W tokens, values and perturbed values, P
+// log-sum-exps and row flags) are copied to shared memory once, so that no level waits for global memory.
 struct SbsChainArgs {
     SbsEpilogueArgs lvl;        // level-independent fields; the per-level ones are filled in by the kernel
     int L, P;                   // levels; parent rows per sequence, 1 + (L - 1) W
     int B;
-    float* state_sum[2];        // [B][W] each
-    float* state_gamma[2];
+    int staged;                 // 1: the dynamic shared memory also holds the finalists' copies
     int32_t* node_token;        // [B][node_stride]
     int32_t* node_parent;
     int64_t node_stride;
@@ -1004,25 +1015,61 @@ struct SbsChainArgs {
     float* gamma_out;
 };
 
+// dynamic shared memory of sbs_chain_kernel
+__host__ __device__ inline size_t sbs_chain_smem_bytes(int W, int P, bool staged) {
+    return sbs_level_scratch_bytes(W, W) + (size_t)4 * W * 4 + (staged ? (size_t)P * W * 12 + (size_t)P * 8 : 0);
+}
+
 static __global__ void __launch_bounds__(kEpilogueThreads) sbs_chain_kernel(const SbsChainArgs c) {
     extern __shared__ double sm_d[];
-    const int b = blockIdx.x, W = c.lvl.W;
+    const int b = blockIdx.x, W = c.lvl.W, tid = threadIdx.x, F = c.P * W;
+    float* const state = (float*)((unsigned char*)sm_d + sbs_level_scratch_bytes(W, W));   // sum[2][W], gamma[2][W]
+    int32_t* const s_tok = (int32_t*)(state + 4 * W);
+    float* const s_val = (float*)(s_tok + F);
+    float* const s_pert = s_val + F;
+    float* const s_lse = s_pert + F;
+    int32_t* const s_rs = (int32_t*)(s_lse + c.P);
+    if (c.staged) {
+        const int64_t f0 = (int64_t)b * F, r0 = (int64_t)b * c.P;
+        for (int i = tid; i < F; i += kEpilogueThreads) {
+            s_tok[i] = c.lvl.fin_token[f0 + i];
+            s_val[i] = c.lvl.fin_value[f0 + i];
+            s_pert[i] = c.lvl.fin_pert[f0 + i];
+        }
+        for (int i = tid; i < c.P; i += kEpilogueThreads) {
+            s_lse[i] = c.lvl.fin_lse[r0 + i];
+            s_rs[i] = c.lvl.row_status[r0 + i];
+        }
+        __syncthreads();
+    }
     int st = 0;
     for (int l = 0; l < c.L; ++l) {
         SbsEpilogueArgs a = c.lvl;
         const int first = l == 0 ? 0 : 1 + (l - 1) * W;     // flat node of the level's parent slot 0
         a.n_par = l == 0 ? 1 : W;
         a.first_parent_node = first;
-        a.fin_token = c.lvl.fin_token + (int64_t)first * W;
-        a.fin_value = c.lvl.fin_value + (int64_t)first * W;
-        a.fin_pert = c.lvl.fin_pert + (int64_t)first * W;
-        a.fin_lse = c.lvl.fin_lse + first;
-        a.row_status = c.lvl.row_status + first;
-        a.sum_in = l == 0 ? nullptr : c.state_sum[(l + 1) & 1];
-        a.gamma_in = l == 0 ? nullptr : c.state_gamma[(l + 1) & 1];
+        if (c.staged) {
+            a.fin_seq_stride = 0;
+            a.row_seq_stride = 0;
+            a.fin_token = s_tok + first * W;
+            a.fin_value = s_val + first * W;
+            a.fin_pert = s_pert + first * W;
+            a.fin_lse = s_lse + first;
+            a.row_status = s_rs + first;
+        } else {
+            a.fin_token = c.lvl.fin_token + (int64_t)first * W;
+            a.fin_value = c.lvl.fin_value + (int64_t)first * W;
+            a.fin_pert = c.lvl.fin_pert + (int64_t)first * W;
+            a.fin_lse = c.lvl.fin_lse + first;
+            a.row_status = c.lvl.row_status + first;
+        }
+        a.state_stride = 0;
+        a.sum_in = l == 0 ? nullptr : state + ((l + 1) & 1) * W;
+        a.gamma_in = l == 0 ? nullptr : state + (2 + ((l + 1) & 1)) * W;
         const bool last = l == c.L - 1;
-        a.sum_out = (last && c.sum_out) ? c.sum_out : c.state_sum[l & 1];
-        a.gamma_out = (last && c.gamma_out) ? c.gamma_out : c.state_gamma[l & 1];
+        a.out_state_stride = 0;
+        a.sum_out = state + (l & 1) * W;
+        a.gamma_out = state + (2 + (l & 1)) * W;
         a.out_token = c.node_token + 1 + (int64_t)l * W;
         a.out_parent = c.node_parent + 1 + (int64_t)l * W;
         a.out_stride = c.node_stride;
@@ -1031,9 +1078,13 @@ static __global__ void __launch_bounds__(kEpilogueThreads) sbs_chain_kernel(cons
         a.status = c.level_status + (int64_t)l * c.B;
         sbs_epilogue_body(a, b, sm_d);
         __syncthreads();   // the level's outputs are the next level's inputs
-        if (threadIdx.x == 0) st |= a.status[b];
+        if (tid == 0) st |= a.status[b];
+        if (last && tid < W) {
+            if (c.sum_out) c.sum_out[(int64_t)b * W + tid] = a.sum_out[tid];
+            if (c.gamma_out) c.gamma_out[(int64_t)b * W + tid] = a.gamma_out[tid];
+        }
     }
-    if (threadIdx.x == 0) c.status[b] = st;
+    if (tid == 0) c.status[b] = st;
 }
 
 }  // namespace rsd
