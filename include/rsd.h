@@ -124,8 +124,10 @@ int rsd_profile_next_scan(void* before, void* after);
  *   top_k       0 (or >= V): none;   top_p  >= 1: none
  *   out_rows    [B][R][V] dense, the rows' element type; may not overlap the input
  *   out_kept    optional [B][R] int32: entries kept in each row;   status [B]
- * A row must fit in shared memory with the call's other data (up to 104,000 2-byte or 52,000 4-byte entries); longer
- * rows are refused with RSD_ERR_UNSUPPORTED.
+ * Values that compare equal (+0 and -0 among them) are one value: the smaller token goes first.
+ * A row must fit in shared memory with the call's other data (up to about 99,000 2-byte or 49,000 4-byte entries);
+ * longer rows are refused with RSD_ERR_UNSUPPORTED.  A row whose copy into shared memory does not arrive within about a
+ * second sets RSD_ST_TIMEOUT for its sequence, and nothing is written for it.
  */
 int rsd_filter_rows(const rsd_rows* rows, int B, int R, int V, int top_k, float top_p, void* out_rows, int32_t* out_kept,
                     int32_t* status, rsd_stream_t stream);

@@ -24,7 +24,7 @@ def _rows(shape, dtype, sigma, seed):
     return t.to(torch.bfloat16 if dtype == "bf16" else torch.float32).cuda()
 
 
-def _check_filter(rsd, rows, top_k, top_p, T):
+def _check_filter(rsd, rows, top_k, top_p, T, max_borderline=None):
     """GPU mask == oracle mask for every row whose nucleus cut is not borderline; returns the GPU's filtered rows."""
     g = rsd.rsd_filter_rows(rows, top_k, top_p, temperature=T)
     host = workloads.as_oracle_rows(rows.contiguous())
@@ -43,7 +43,7 @@ def _check_filter(rsd, rows, top_k, top_p, T):
                 continue
             assert o["margin"][b, r] <= 1e-5, ("filter", b, r, int(kept[b, r]), int(o["kept"][b, r]), float(o["margin"][b, r]))
             borderline += 1
-    assert borderline <= max(1, B * R // 100)
+    assert borderline <= (max(1, B * R // 100) if max_borderline is None else max_borderline)
     return g
 
 
@@ -81,6 +81,31 @@ def test_filter_rows_ties_masked_entries_unaligned_rows_and_errors(rsd):
         rsd.rsd_filter_rows(rows, 0, 0.0)
     with pytest.raises(rsd.RsdError, match="shared memory"):
         rsd.rsd_filter_rows(torch.zeros((1, 1, 120000), device="cuda"), 0, 0.9)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_filter_rows_degenerate_rows(rsd, dtype):
+    # rows the histogram over values cannot split: all entries equal, zeros of both signs, one entry that carries all the
+    # mass, two values only, a very wide spread; plus a vocabulary above 65,536 entries (no list of 16-bit indices)
+    V = 4096
+    g = torch.Generator(device="cpu").manual_seed(77)
+    rows = torch.zeros((1, 7, V), dtype=torch.float32)
+    rows[0, 0, :] = 0.25
+    rows[0, 1, :] = torch.where(torch.rand(V, generator=g) < 0.5, torch.tensor(-0.0), torch.tensor(0.0))
+    rows[0, 1, 5::400] = 1.0
+    rows[0, 2, :] = torch.randn(V, generator=g)
+    rows[0, 2, 1234] = 30.0
+    rows[0, 3, :] = torch.where(torch.rand(V, generator=g) < 0.5, torch.tensor(-1.0), torch.tensor(1.0))
+    rows[0, 4, :] = torch.randn(V, generator=g) * 8.0
+    rows[0, 5, :] = torch.arange(V, dtype=torch.float32) / 64.0 - 40.0
+    rows[0, 6, :] = torch.randn(V, generator=g) * 1e-3
+    rows = rows.to(torch.bfloat16 if dtype == "bf16" else torch.float32).cuda()
+    # (equal entries put cumulative masses exactly on round fractions: rows whose cut the oracle calls borderline may differ)
+    for top_k, top_p, T in ((0, 0.9, 1.0), (0, 0.5, 1.0), (100, 1.0, 1.0), (3000, 0.7, 1.0), (0, 0.99, 0.3), (0, 0.999999, 1.0)):
+        _check_filter(rsd, rows, top_k, top_p, T, max_borderline=3)
+    big = _rows((1, 2, 70000), dtype, 2.0, 78) if dtype == "bf16" else _rows((1, 2, 40000), dtype, 2.0, 78)
+    _check_filter(rsd, big, 0, 0.9, 1.0)
+    _check_filter(rsd, big, 500, 0.95, 1.0)
 
 
 @pytest.mark.parametrize("dtype,V", [("bf16", 4099), ("f32", 1000)])
