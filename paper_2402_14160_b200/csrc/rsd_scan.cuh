@@ -390,8 +390,9 @@ __device__ __forceinline__ float slot_element<__nv_bfloat16>(uint32_t addr, uint
 // One block per row.
 // ALIGNED: rows start on 16-byte boundaries and V is a multiple of 16 (vector loads); WIDE: 32-byte boundaries as well.
 // TEMP: a sampling temperature other than 1 applies (otherwise the scale factors are compile-time constants).
+// Nine blocks per SM for 2-byte rows (56 registers: a group in flight is 8 registers), eight for 4-byte rows.
 template <typename T, bool ALIGNED, bool WIDE, bool NEED_LSE, bool TEMP>
-__global__ void __launch_bounds__(kScanThreads, 8) scan_topk_kernel(const ScanArgs a) {
+__global__ void __launch_bounds__(kScanThreads, sizeof(T) == 2 ? 9 : 8) scan_topk_kernel(const ScanArgs a) {
     extern __shared__ float ub[];                    // [n_groups] upper bound of each group's perturbed values
     // One buffer, two uses: the threads' group slots during the streaming loop, the queues of the stages after it.
     constexpr int kQueueBytes = 4 * (kCandCap + 3 * kTaskCap + 4 * kFinCap);
