@@ -369,21 +369,24 @@ struct RowFilter {
         if (population > kListCap) return false;
         // ---- the codes of the picked bin: the bin index does not increase with the code, so both ends come from a
         // bisection over the codes with the same arithmetic as the sweep ----------------------------------------------------
-        uint32_t first_in, last_in;                                  // smallest and largest code of [lo, hi] in the bin
-        {
+        if (threadIdx.x == 0) {                                      // (two threads of two warps: the others sleep at the barrier)
             uint32_t a_ = lo, b_ = hi;                               // smallest code with bin <= pick
             while (a_ < b_) {
                 const uint32_t mid = a_ + ((b_ - a_) >> 1);
                 if (cb.bin(RowCodes<T>::value_of_code(mid)) <= pick) b_ = mid; else a_ = mid + 1u;
             }
-            first_in = a_;
-            a_ = lo; b_ = hi;                                        // largest code with bin >= pick
+            sm.bound[0] = a_;
+        } else if (threadIdx.x == 32) {
+            uint32_t a_ = lo, b_ = hi;                               // largest code with bin >= pick
             while (a_ < b_) {
                 const uint32_t mid = a_ + ((b_ - a_ + 1u) >> 1);
                 if (cb.bin(RowCodes<T>::value_of_code(mid)) >= pick) a_ = mid; else b_ = mid - 1u;
             }
-            last_in = a_;
+            sm.bound[1] = a_;
         }
+        __syncthreads();
+        const uint32_t first_in = sm.bound[0], last_in = sm.bound[1];   // smallest and largest code of [lo, hi] in the bin
+        __syncthreads();
         if (first_in > last_in) return false;
         gather(first_in, last_in, inside, everything);
         if (n_list < 0) return false;
@@ -663,7 +666,7 @@ __global__ void __launch_bounds__(kFilterThreads) filter_rows_kernel(const Filte
         if (kElem == 2) ((uint16_t*)row_sm)[i] = (uint16_t)h;
         else ((uint32_t*)row_sm)[i] = h;
     }
-    if (bulk) wait_bar(&sm.row_bar, 0, &sm.copy_gave_up);
+    if (bulk && warp == 0) wait_bar(&sm.row_bar, 0, &sm.copy_gave_up);   // one warp polls, the others sleep at the barrier
     __syncthreads();
     if (sm.copy_gave_up) {                                        // the copy never landed: report, write nothing
         if (tid == 0) atomicOr(&a.status[b], 32);                 // RSD_ST_TIMEOUT

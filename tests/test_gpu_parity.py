@@ -161,7 +161,9 @@ def test_sbs_levels_match_oracle(rsd, dtype, V, W, L, is_logprob):
 
 
 @pytest.mark.parametrize("dtype,V,W,L,is_logprob", [("f32", 1000, 3, 3, False), ("bf16", 4099, 8, 4, False),
-                                                    ("f32", 515, 5, 1, True), ("bf16", 32000, 6, 5, False)])
+                                                    ("f32", 515, 5, 1, True), ("bf16", 32000, 6, 5, False),
+                                                    ("f32", 300, 32, 3, False),    # finalists too many for shared memory
+                                                    ("bf16", 520, 16, 6, False)])  # 1296 finalists, staged
 def test_sbs_draft_tree_is_the_chain_of_level_calls(rsd, dtype, V, W, L, is_logprob):
     # rsd_sbs_draft_tree (all levels from rows that exist up front) must give what L rsd_sbs_step calls give, bit for
     # bit, and through them what the oracle's level-by-level chain gives
