@@ -668,6 +668,8 @@ __global__ void __launch_bounds__(kFilterThreads) filter_rows_kernel(const Filte
     }
     if (bulk && warp == 0) wait_bar(&sm.row_bar, 0, &sm.copy_gave_up);   // one warp polls, the others sleep at the barrier
     __syncthreads();
+    if (bulk && warp != 0 && !sm.copy_gave_up) wait_bar(&sm.row_bar, 0, &sm.copy_gave_up);   // (done: every thread has now seen the copy's completion itself)
+    __syncthreads();
     if (sm.copy_gave_up) {                                        // the copy never landed: report, write nothing
         if (tid == 0) atomicOr(&a.status[b], 32);                 // RSD_ST_TIMEOUT
         return;
