@@ -9,6 +9,10 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
+import workloads
+from tests.parity import Tally, compare_sbs_level
+
 pytestmark = pytest.mark.gpu
 
 
@@ -54,6 +58,14 @@ def test_static_scratch_entry_point_matches_the_caller_scratch_one_twice():
             a, b = ref[key].cpu().numpy().astype(np.float64), got[key].cpu().numpy().astype(np.float64)
             assert np.all(np.abs(a - b) <= 1e-6 + 1e-5 * np.abs(a)), key
         assert int(got["count"].min()) == W
+        # and against the oracle itself, decision by decision with its margins
+        host = workloads.as_oracle_rows(rows)
+        o = oracle.sbs_step(host, W, first_node, None if sig is None else sig.cpu().numpy(),
+                            None if gam is None else gam.cpu().numpy(), 21, step, seq_base=3)
+        o["parent"] = np.where(o["parent"] >= 0, o["parent"] + first_node, -1)    # (parent_base of the call)
+        t = Tally()
+        compare_sbs_level(t, {k: v.cpu().numpy() for k, v in got.items()}, o, W, set())
+        t.check()
         done += 1
     assert done == 2
 
