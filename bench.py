@@ -406,6 +406,34 @@ def main():
             "accepted_len_histogram": np.bincount(acc, minlength=L + 1).tolist(),
             "block_efficiency": float(acc.mean()) + 1.0}
 
+    # ---- two batches in flight (not the headline): the same steps, alternating between two streams -----------------
+    # A serving engine that decodes two batches at once lets one batch's row scan fill the SMs that the other batch's
+    # last, longest walks leave idle.  Both batches read the same resident rows here; trees, seeds and results are
+    # their own.
+    if world == 1 and not per_level and not warp_rows:
+        streams = [torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)]
+        steppers = [stepper, rsd_step.make_step(w, device=dev, rows_ready=True)]
+        for s in range(4):
+            with torch.cuda.stream(streams[s % 2]):
+                steppers[s % 2].run(draft, target, 0, 500 + s, seq_base)
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for st in streams:
+            st.wait_event(t0)
+        for s in range(K):
+            with torch.cuda.stream(streams[s % 2]):
+                steppers[s % 2].run(draft, target, 0, 2000 + s, seq_base)
+        for st in streams:
+            torch.cuda.current_stream().wait_stream(st)
+        t1.record()
+        torch.cuda.synchronize()
+        two_ms = t0.elapsed_time(t1)
+        line["two_batches_in_flight"] = {
+            "value": nodes_per_step * K / (two_ms * 1e-3), "unit": UNIT, "ms_per_step": two_ms / K,
+            "note": "the same K steps issued alternately on two streams (two independent batches over the same resident "
+                    "rows): one batch's scan overlaps the other's walk; `value` above is one batch at a time"}
+
     # ---- end to end: pinned host logits -> device -> step -> results on the host ---------------------------
     if not args.no_e2e:
         h_draft = torch.empty(draft.shape, dtype=draft.dtype, pin_memory=True)
