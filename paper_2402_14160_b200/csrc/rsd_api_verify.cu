@@ -94,8 +94,10 @@ int rsd_verify_tree_rule(const rsd_rows* draft, const rsd_rows* target, const rs
     } while (0)
     const bool wide_blocks = B <= sm_count();
     if (rule == RSD_RULE_RRS && final_sampler == RSD_FINAL_INVERSE_CDF) {
-        // rows on 16-byte boundaries: the walk whose passes are fed by the copy engine
-        if (aligned) {
+        // rows on 16-byte boundaries, of at most 64 chunks (the ring keeps its chunks as bits of one word): the walk
+        // whose passes are fed by the copy engine
+        const size_t row_bytes = (size_t)V * (draft->dtype == RSD_F32 ? 4 : 2);
+        if (aligned && (row_bytes + rsd::walk_ring::kRowChunkBytes - 1) / rsd::walk_ring::kRowChunkBytes <= 64) {
             if (draft->dtype == RSD_F32) launch_ring_walk<float>(a, B, s);
             else launch_ring_walk<__nv_bfloat16>(a, B, s);
         }

@@ -59,7 +59,21 @@ struct RingSmem {
     int par[kMaxCachedNodes], tok[kMaxCachedNodes];
     int nan_seen;                                 // a cleaning pass met a NaN
     int abort;                                    // a wait ran out: the walk is abandoned and reported
+    // for the pass that sums what is left of the draft row: the tokens rejected at the node so far, and per working
+    // warp the chunks in which its tile holds one of them
+    int gone_tok[kMaxRemovedRing];
+    int n_gone_tok;
+    unsigned gone_chunks[kWorkWarps][2];
 };
+
+// Which lane and which of its 16 values hold element `o` (0..511) of a tile as load_pieces() deals them out.
+template <typename T>
+__device__ __forceinline__ void piece_of(int o, int& lane, int& j) {
+    constexpr int kPer = 16 / (int)sizeof(T);     // elements per 16-byte piece
+    const int piece = o / kPer;
+    lane = piece & 31;
+    j = (piece >> 5) * kPer + o % kPer;
+}
 
 // A lane's 16 values of a 512-element tile in shared memory: the 16-byte pieces lane, lane + 32, ... of the tile
 // (conflict-free 128-bit loads).  Which elements a lane sums does not matter; the one place that needs token order
@@ -95,14 +109,14 @@ __device__ __forceinline__ void values16(const Packed<T>& pk, float (&v)[16]) {
     }
 }
 
-enum { kPassEnd = -1, kPassFirst = 0, kPassTarget = 1, kPassResidual = 2 };
+enum { kPassEnd = -1, kPassFirst = 0, kPassTarget = 1, kPassResidual = 2, kPassRest = 3 };
 
 // State of the walk at one node (control warp only): the closed-form chain of rsd_verify.cuh.
 struct NodeState {
     float mq, mp;       // reference values of the exponentials (raw units)
     float kq, kp;       // log2(e) / temperature
     double Sq, Sp;      // normalisers relative to the references
-    double A, P, Z;     // chain state
+    double A, Z;        // chain state (1 - P is kept by the walk itself)
     float a_hi, a_lo;   // A Sq / Sp as a two-float sum
     bool with_draft;    // false: a node without children, only its target row is read
     bool has_nan;       // a NaN was seen in the node's rows: the passes clean their inputs
@@ -267,6 +281,7 @@ struct Ring {
     //   kPassFirst     both rows: sums of exp(lt k_q - c_q) and exp(ld k_p - c_p)
     //   kPassTarget    target row only: sum of the weights exp(lt k_q - c_q)
     //   kPassResidual  both rows: sum of the weights (qh - a ph)+
+    //   kPassRest      draft row: sum of exp(ld k_p - c_p) without the tokens listed in sm.gone_tok
     // CLEAN passes turn NaN into -inf (reported through sm.nan_seen) and also return the rows' maxima; the plain ones
     // carry no code for either.  STORE_TILES: the sum of every tile goes to sm.tile_sum.
     template <int KIND, bool CLEAN, bool STORE_TILES>
@@ -274,7 +289,33 @@ struct Ring {
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
         float s0 = 0.0f, s1 = 0.0f, m0 = kNegInf, m1 = kNegInf;
         bool saw_nan = false;
+        // bit c: this warp's tile of chunk c holds one of the listed tokens
+        const unsigned long long gone_tiles_of_warp =
+            KIND == kPassRest ? ((unsigned long long)sm.gone_chunks[warp][1] << 32) | sm.gone_chunks[warp][0] : 0ull;
         consume(cmd, [&](int tile, const unsigned char* qt, const unsigned char* pt) {
+            if (KIND == kPassRest) {
+                Packed<T> pp;
+                load_pieces(pp, pt, lane);
+                float p[16];
+                if (CLEAN) m1 = fmaxf(m1, clean<T>(pp, p, saw_nan));
+                else pp.unpack(p);
+                exp16(p, cmd.kp, cmd.cp, p);
+                if ((gone_tiles_of_warp >> (tile / kTPC)) & 1ull) {
+                    for (int i = 0; i < sm.n_gone_tok; ++i) {
+                        const int o = sm.gone_tok[i] - tile * kTileElems;
+                        if (o < 0 || o >= kTileElems) continue;
+                        int l_, j_;
+                        piece_of<T>(o, l_, j_);
+                        if (l_ == lane) {
+#pragma unroll
+                            for (int jj = 0; jj < 16; ++jj)
+                                if (jj == j_) p[jj] = 0.0f;
+                        }
+                    }
+                }
+                s0 += tree_sum16(p);
+                return;
+            }
             Packed<T> pq;
             load_pieces(pq, qt, lane);
             float q[16];
@@ -381,6 +422,9 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             } else if (cmd.kind == kPassTarget) {
                 if (cmd.clean) ring.template work<kPassTarget, true, true>(cmd);
                 else ring.template work<kPassTarget, false, true>(cmd);
+            } else if (cmd.kind == kPassRest) {
+                if (cmd.clean) ring.template work<kPassRest, true, false>(cmd);
+                else ring.template work<kPassRest, false, false>(cmd);
             } else {
                 if (cmd.clean) {
                     if (cmd.store_tiles) ring.template work<kPassResidual, true, true>(cmd);
@@ -421,7 +465,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
     // results.  The first kSlots steps are taken before the command is published: what they wait for, if anything, are
     // slot uses of earlier passes, which every working warp finished before it reported its sums; so the copies travel
     // while the working warps wake up.  `meanwhile` runs on the control warp while the pass is under way.
-    auto run_pass = [&](int kind, bool store_tiles, double& S0, double& S1, float& M0, float& M1, auto&& meanwhile) {
+    auto run_pass = [&](int kind, bool store_tiles, double& S0, double& S1, float& M0, float& M1, auto&& meanwhile, auto&& early) {
         const bool with_draft = kind != kPassTarget;
         int dir;
         unsigned long long parity, missing;
@@ -434,10 +478,11 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             cmd.backward = dir; cmd.parity = parity;
             sm.cmd = cmd;
         }
-        const int early = ring.n_chunks < kSlots ? ring.n_chunks : kSlots;
-        ring.produce_early(rowq, rowp, with_draft, dir, missing, early);
+        const int n_early = ring.n_chunks < kSlots ? ring.n_chunks : kSlots;
+        ring.produce_early(rowq, rowp, with_draft, dir, missing, n_early);
+        early();           // (what else the working warps need: written while the first copies travel)
         __syncthreads();   // the command is in place
-        ring.produce(rowq, rowp, with_draft, dir, missing, early, ring.n_chunks);
+        ring.produce(rowq, rowp, with_draft, dir, missing, n_early, ring.n_chunks);
         meanwhile();
         __syncthreads();   // the warps' sums are in place
         static_assert(kWorkWarps == 8, "fixed summation tree over eight warps");
@@ -461,7 +506,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
         st.with_draft = !(c < 0 || len >= a.L);
         rowq = row_ptr<T>(a.target, b, cur);
         rowp = st.with_draft ? row_ptr<T>(a.draft, b, cur) : rowq;
-        st.A = 0.0; st.P = 0.0; st.Z = 1.0; st.a_hi = st.a_lo = 0.0f; st.has_nan = false;
+        st.A = 0.0; st.Z = 1.0; st.a_hi = st.a_lo = 0.0f; st.has_nan = false;
         st.mq = 0.0f; st.mp = 0.0f; st.Sp = 1.0;
         tiles_valid = false;
         ring.forget_node();
@@ -498,7 +543,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             float M0, M1;
             const int kind = st.with_draft ? kPassFirst : kPassTarget;
             for (int attempt = 0; attempt < 3; ++attempt) {
-                run_pass(kind, !st.with_draft, S0, S1, M0, M1, nothing);
+                run_pass(kind, !st.with_draft, S0, S1, M0, M1, nothing, nothing);
                 if (sm.abort) { aborted = true; break; }
                 if (!st.with_draft) S1 = 1.0;
                 const bool good = S0 >= (double)kSumFloor && S0 < 1e300 && S1 >= (double)kSumFloor && S1 < 1e300;
@@ -556,7 +601,25 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             U = (double)(rw.x >> 8) * (1.0 / 16777216.0);
         };
         prepare(c);
+        // 1 - P of the closed form, the draft mass still in play.  It is carried by subtraction while that is accurate:
+        // every p(x) has the relative error of a fast exponential and of the fp32 sums behind S_p, and with a peaked
+        // draft the rejected tokens can hold all but 1e-7 of the mass.  Once the error bound passes 2e-6 of what is left,
+        // a pass sums the draft row anew without the rejected tokens.
+        double one_mP = 1.0, one_mP_err = 0.0;
         double inv_1mP = 1.0;    // 1 / (1 - P)
+        auto publish_gone = [&] {   // the rejected tokens for that pass (lane i holds entries 4 i .. 4 i + 3)
+            if (lane < 2 * kWorkWarps) (&sm.gone_chunks[0][0])[lane] = 0u;
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (rem_x[i] >= 0) {
+                    sm.gone_tok[4 * lane + i] = rem_x[i];
+                    const int tile = rem_x[i] / kTileElems, chunk = tile / Ring<T>::kTPC;   // tile t belongs to warp t mod 8
+                    atomicOr(&sm.gone_chunks[tile & (kWorkWarps - 1)][chunk >> 5], 1u << (chunk & 31));
+                }
+            }
+            if (lane == 0) sm.n_gone_tok = n_removed;
+        };
         int accepted = -1;
         while (c >= 0) {
             // Eq. 3 in closed form: accept iff U < min(1, r (1 - P) / (Z p(x))), r = (q(x) - A p(x))+, tested without
@@ -564,10 +627,10 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             const double px = repeated ? 0.0 : px_row;
             const double r = fmax(qx - st.A * px_row, 0.0);
             bool take;
-            if (px > 0.0) take = U * st.Z * px < r * (1.0 - st.P);
+            if (px > 0.0) take = U * st.Z * px < r * one_mP;
             else { status |= 8; take = r > 0.0; }   // RSD_ST_ZERO_DRAFT_PROB
             if (a.dbg_theta && lane == 0)
-                a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)(px > 0.0 ? fmin(1.0, r * (1.0 - st.P) / (st.Z * px)) : (r > 0.0 ? 1.0 : 0.0));
+                a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)(px > 0.0 ? fmin(1.0, r * one_mP / (st.Z * px)) : (r > 0.0 ? 1.0 : 0.0));
             if (take) { accepted = c; break; }
             // rejected.  Eqs. 1-2 in closed form: A_{j+1} = A_j + Z_j / (1 - P_j), Z_{j+1} = sum (q - A_{j+1} p)+
             ++j;
@@ -579,7 +642,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
                 st.a_hi = (float)aa;
                 st.a_lo = (float)(aa - (double)st.a_hi);
             }
-            const double P_new = st.P + px;
+            double one_mP_new = one_mP - px, err_new = one_mP_err + 4e-7 * px;   // (px = 0 for a repeated token)
             if (!repeated && n_removed < kMaxRemovedRing) {
                 if (lane == (n_removed >> 2)) {
 #pragma unroll
@@ -592,9 +655,9 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             float f0, f1;
             const bool maybe_last = next < 0;   // no sibling left: the last token is drawn from this residual
             run_pass(kPassResidual, maybe_last, zhat, none, f0, f1, [&] {
-                inv_1mP = 1.0 / (1.0 - P_new);
+                inv_1mP = 1.0 / one_mP_new;
                 if (next >= 0) prepare(next);
-            });
+            }, nothing);
             if (sm.abort) { aborted = true; break; }
             const double Z_new = zhat * inv_Sq;
             if (Z_new > 0.0 && Z_new < 1.7e308) {
@@ -608,8 +671,18 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
                 st.a_lo = (float)(aa - (double)st.a_hi);
                 tiles_valid = false;
             }
-            st.P = P_new;
-            if (!(1.0 - st.P > 0.0)) { status |= 16; break; }   // RSD_ST_DRAFT_EXHAUSTED
+            if (next >= 0 && err_new > 2e-6 * one_mP_new && n_removed < kMaxRemovedRing) {   // (every rejected token is listed)
+                double rest, none2;
+                float g0, g1;
+                run_pass(kPassRest, false, rest, none2, g0, g1, nothing, publish_gone);
+                if (sm.abort) { aborted = true; break; }
+                one_mP_new = rest * inv_Sp;
+                err_new = 4e-7 * one_mP_new;
+                inv_1mP = 1.0 / one_mP_new;
+            }
+            one_mP = one_mP_new;
+            one_mP_err = err_new;
+            if (!(one_mP > 0.0)) { status |= 16; break; }   // RSD_ST_DRAFT_EXHAUSTED
             c = next;
         }
         if (aborted) break;
@@ -630,7 +703,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
         double s, none;
         float f0, f1;
         if (!residual) { rowp = rowq; ring.forget_node(); }   // (the slots' draft halves are not refreshed by this pass)
-        run_pass(residual ? kPassResidual : kPassTarget, true, s, none, f0, f1, nothing);
+        run_pass(residual ? kPassResidual : kPassTarget, true, s, none, f0, f1, nothing, nothing);
         aborted = sm.abort != 0;
     }
     // the working warps are done: let them go, then finish alone

@@ -559,6 +559,8 @@ def _iid_tree(draft_h, branching, seed):
     B, P, V = draft_h.shape
     rng = np.random.default_rng(seed)
     token = np.full((B, len(parent)), -1, np.int32)
+    if draft_h.dtype == np.uint16:   # bf16 rows come as bit patterns
+        draft_h = (draft_h.astype(np.uint32) << 16).view(np.float32)
     for b in range(B):
         for n in range(1, len(parent)):
             row = draft_h[b, parent[n]].astype(np.float64)
@@ -616,6 +618,66 @@ def test_verify_tree_rule_rrs_is_verify_tree_and_bad_rules_are_refused(rsd):
         rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, rsd.RULE_KSEQ, 0.5, 0, 5, 0)
     with pytest.raises(rsd.RsdError):
         rsd.rsd_verify_tree_rule(draft, target, par_t, tok_t, 2, rsd.RULE_RRS, 1.0, 3, 5, 0)
+
+
+@pytest.mark.parametrize("dtype,V", [("f32", 140000), ("bf16", 262144)])
+def test_verify_tree_longest_rows(rsd, dtype, V):
+    # 4-byte rows of more than 131,072 entries are more than 64 chunks of the copy-engine ring: they take the other walk
+    B, branching = 2, (2, 2)
+    L = len(branching)
+    n_nodes = len(workloads.rsdc_parent_array(branching))
+    base = _rows((B, n_nodes, V), "f32", 2.5, 1500)
+    draft = base[:, :3].to(torch.bfloat16 if dtype == "bf16" else torch.float32).contiguous()
+    target = (base + _rows((B, n_nodes, V), "f32", 1.0, 1501)).to(draft.dtype).contiguous()
+    draft_h = workloads.as_oracle_rows(draft)
+    k, nodes = workloads.rsdc_rows(branching)
+    parent = workloads.rsdc_parent_array(branching)
+    token = workloads.rsdc_tokens_from_rows(branching, oracle.gumbel_topk(draft_h, k, nodes, 3, 1)["token"])
+    g = _np(rsd.rsd_verify_tree(draft, target, torch.from_numpy(parent).cuda(), torch.from_numpy(token).cuda(), L, 3, 1,
+                                want_theta=True))
+    o = oracle.verify_tree(draft_h, workloads.as_oracle_rows(target), parent, token, L, 3, 1)
+    t = Tally()
+    compare_verify(t, g, o, parent)
+    t.check()
+    assert np.array_equal(g["status"], o["status"])
+
+
+@pytest.mark.parametrize("dtype,V,branching", [("f32", 96, (4,)), ("bf16", 1000, (2, 2, 3)), ("f32", 33, (2, 1)),
+                                               ("bf16", 515, (4, 1, 4)), ("bf16", 32000, (3, 2))])
+def test_verify_tree_peaked_draft_flat_target(rsd, dtype, V, branching):
+    # Draft at temperature 0.3 on wide logits, target at temperature 2: the first child often holds all but 1e-6 or
+    # less of the draft mass and is rejected, so the thresholds of its siblings hang on 1 - P, the mass that is left.
+    # Taken as a difference of rounded sums it would be noise; the thresholds must still agree with the oracle's.
+    B = 24 if V <= 5000 else 6
+    L = len(branching)
+    n_nodes = len(workloads.rsdc_parent_array(branching))
+    P = n_nodes - int(np.prod(branching))
+    base = _rows((B, n_nodes, V), "f32", 3.0, 1300 + V)
+    draft = base[:, :P].to(torch.bfloat16 if dtype == "bf16" else torch.float32).contiguous()
+    target = (base + _rows((B, n_nodes, V), "f32", 2.0, 1301 + V)).to(draft.dtype).contiguous()
+    draft_h = workloads.as_oracle_rows(draft)
+    k, nodes = workloads.rsdc_rows(branching)
+    parent = workloads.rsdc_parent_array(branching)
+    t = Tally()
+    small = 0
+    for seed in range(4):
+        token = workloads.rsdc_tokens_from_rows(
+            branching, oracle.gumbel_topk(draft_h, k, nodes, seed, 2, seq_base=7, temperature=0.3)["token"])
+        par_t, tok_t = torch.from_numpy(parent).cuda(), torch.from_numpy(token).cuda()
+        g = _np(rsd.rsd_verify_tree(draft, target, par_t, tok_t, L, seed, 2, seq_base=7, want_theta=True,
+                                    draft_temperature=0.3, target_temperature=2.0))
+        o = oracle.verify_tree(draft_h, workloads.as_oracle_rows(target), parent, token, L, seed, 2, seq_base=7,
+                               draft_temperature=0.3, target_temperature=2.0)
+        compare_verify(t, g, o, parent)
+        assert np.array_equal(g["status"], o["status"])
+        # how peaked: draft mass outside the root's first child
+        row = draft_h[:, 0].astype(np.float64) / 0.3
+        pr = np.exp(row - row.max(axis=1, keepdims=True))
+        pr /= pr.sum(axis=1, keepdims=True)
+        small += int(np.sum(1.0 - pr[np.arange(B), token[:, 1]] < 1e-4))
+    t.check()
+    if V <= 100:
+        assert small > 0          # the regime the test is about does occur
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
