@@ -62,7 +62,8 @@ enum {
     RSD_ST_ZERO_RESIDUAL = 4,   /* sum of [q - p]+ was not positive; the previous residual was kept */
     RSD_ST_ZERO_DRAFT_PROB = 8, /* a child token had draft probability 0 (in fp32: below 2^-126 of the row's largest
                                    weight); accepted iff its residual mass is > 0 */
-    RSD_ST_DRAFT_EXHAUSTED = 16, /* the draft had no mass left after a removal; later siblings were ignored */
+    RSD_ST_DRAFT_EXHAUSTED = 16, /* the draft had no mass left after a removal (in fp32: nothing above 2^-126 of the
+                                    row's largest weight); later siblings were ignored */
     RSD_ST_TIMEOUT = 32         /* an on-chip copy of a row did not complete within about a second (a hardware or
                                    driver fault, never a property of the data): the walk of this sequence was
                                    abandoned, accepted_len counts what was accepted before, last_token is -1 */

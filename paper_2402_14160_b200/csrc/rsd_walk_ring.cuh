@@ -576,8 +576,9 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
         // What the test of child j needs and no pass changes: its token, its probabilities under the node's two rows,
         // whether an earlier sibling with the same token was rejected, and its uniform.
         int j = 0, x = -1;
-        double qx = 0.0, px_row = 0.0, U = 0.0;
-        bool repeated = false;
+        double qx = 0.0, px_row = 0.0, qp = 0.0, U = 0.0;   // q(x), p(x), q(x) / p(x)
+        bool repeated = false, p_none = false;             // p_none: the draft row gives the token no mass (-inf or NaN)
+        const double inv_ratio = st.Sp * inv_Sq;
         auto prepare = [&](int child) {
             float lq, lp;
             if (j < 32) {
@@ -589,10 +590,15 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
                 lq = RowIO<T>::scalar(rowq, x);
                 lp = RowIO<T>::scalar(rowp, x);
             }
-            const float qh = (lq == lq) ? ex2_approx(fmaf(lq, st.kq, -st.mq * st.kq)) : 0.0f;
-            const float ph = (lp == lp) ? ex2_approx(fmaf(lp, st.kp, -st.mp * st.kp)) : 0.0f;
+            const float eq = fmaf(lq, st.kq, -st.mq * st.kq), ep = fmaf(lp, st.kp, -st.mp * st.kp);
+            const float qh = (lq == lq) ? ex2_approx(eq) : 0.0f;
+            const float ph = (lp == lp) ? ex2_approx(ep) : 0.0f;
             qx = (double)qh * inv_Sq;
             px_row = (double)ph * inv_Sp;
+            // The test needs q(x) / p(x) only: taken from the difference of the exponents it survives probabilities
+            // below the fp32 range (children drafted from the far tail of a peaked row), where q(x) and p(x) are both 0.
+            p_none = !(lp == lp) || !(lp > kNegInf);
+            qp = (lq == lq && !p_none) ? (double)ex2_approx(eq - ep) * inv_ratio : 0.0;
             bool mine = false;
 #pragma unroll
             for (int i = 0; i < 4; ++i) mine |= rem_x[i] == x;
@@ -624,13 +630,21 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
         while (c >= 0) {
             // Eq. 3 in closed form: accept iff U < min(1, r (1 - P) / (Z p(x))), r = (q(x) - A p(x))+, tested without
             // the division; a child the draft cannot produce any more is taken iff it has residual mass
-            const double px = repeated ? 0.0 : px_row;
-            const double r = fmax(qx - st.A * px_row, 0.0);
+            const bool no_draft = repeated || p_none;
+            const double px = no_draft ? 0.0 : px_row;
             bool take;
-            if (px > 0.0) take = U * st.Z * px < r * one_mP;
-            else { status |= 8; take = r > 0.0; }   // RSD_ST_ZERO_DRAFT_PROB
-            if (a.dbg_theta && lane == 0)
-                a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)(px > 0.0 ? fmin(1.0, r * one_mP / (st.Z * px)) : (r > 0.0 ? 1.0 : 0.0));
+            double theta;
+            if (!no_draft) {   // U < min(1, (q/p - A)+ (1 - P) / Z)
+                const double g = fmax(qp - st.A, 0.0) * one_mP;
+                take = U * st.Z < g;
+                theta = fmin(1.0, g / st.Z);
+            } else {           // RSD_ST_ZERO_DRAFT_PROB
+                const double r = fmax(qx - st.A * px_row, 0.0);
+                status |= 8;
+                take = r > 0.0;
+                theta = r > 0.0 ? 1.0 : 0.0;
+            }
+            if (a.dbg_theta && lane == 0) a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)theta;
             if (take) { accepted = c; break; }
             // rejected.  Eqs. 1-2 in closed form: A_{j+1} = A_j + Z_j / (1 - P_j), Z_{j+1} = sum (q - A_{j+1} p)+
             ++j;
