@@ -374,12 +374,13 @@ def test_verify_tree_wide_and_large_trees(rsd, dtype, V, branching, aligned):
     assert tested.max() >= branching[0] // 2                       # some walk went through many children of a node
 
 
-def test_verify_tree_repeated_sibling_tokens(rsd):
+@pytest.mark.parametrize("V", [128, 127])      # rows on and off 16-byte boundaries: the two walks
+def test_verify_tree_repeated_sibling_tokens(rsd, V):
     # Two children of a node carry the same token (a caller's tree; Gumbel-Top-k never drafts one): once the first is
     # rejected its draft mass is gone (Eq. 1), so the second is a child the draft could not have produced: threshold 0
     # (its residual mass is 0 too) and RSD_ST_ZERO_DRAFT_PROB, exactly as the oracle reports it.
     rng = np.random.default_rng(8)
-    B, V = 16, 128
+    B = 16
     parent = np.array([-1, 0, 0, 0, 0], np.int32)
     draft_h = rng.normal(0, 1, (B, 1, V)).astype(np.float32)
     target_h = rng.normal(0, 1, (B, 5, V)).astype(np.float32)
