@@ -44,6 +44,7 @@ struct PassCmd {
     int kind;            // kPassEnd, or a pass kind below
     int clean;           // 1: NaN inputs are turned into -inf (a NaN was seen in the node's rows)
     int store_tiles;     // 1: the pass leaves the sum of every 512-element tile in tile_sum
+    int rest;            // kPassTarget only, 1: the row summed is the draft row (kq, cq are its), without sm.gone_tok
     float kq, kp;        // log2(e) / temperature of the target and draft rows
     float cq, cp;        // reference * k: exponentials are 2^(value * k - c)
     float a_hi, a_lo;    // coefficient of the residual pass, as a two-float sum
@@ -109,7 +110,7 @@ __device__ __forceinline__ void values16(const Packed<T>& pk, float (&v)[16]) {
     }
 }
 
-enum { kPassEnd = -1, kPassFirst = 0, kPassTarget = 1, kPassResidual = 2, kPassRest = 3 };
+enum { kPassEnd = -1, kPassFirst = 0, kPassTarget = 1, kPassResidual = 2 };
 
 // State of the walk at one node (control warp only): the closed-form chain of rsd_verify.cuh.
 struct NodeState {
@@ -281,7 +282,8 @@ struct Ring {
     //   kPassFirst     both rows: sums of exp(lt k_q - c_q) and exp(ld k_p - c_p)
     //   kPassTarget    target row only: sum of the weights exp(lt k_q - c_q)
     //   kPassResidual  both rows: sum of the weights (qh - a ph)+
-    //   kPassRest      draft row: sum of exp(ld k_p - c_p) without the tokens listed in sm.gone_tok
+    //                  (cmd.rest: of the draft row instead, without the tokens listed in sm.gone_tok: the same code,
+    //                  so that this rare pass adds nothing to the kernel's size)
     // CLEAN passes turn NaN into -inf (reported through sm.nan_seen) and also return the rows' maxima; the plain ones
     // carry no code for either.  STORE_TILES: the sum of every tile goes to sm.tile_sum.
     template <int KIND, bool CLEAN, bool STORE_TILES>
@@ -289,18 +291,20 @@ struct Ring {
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
         float s0 = 0.0f, s1 = 0.0f, m0 = kNegInf, m1 = kNegInf;
         bool saw_nan = false;
-        // bit c: this warp's tile of chunk c holds one of the listed tokens
+        // cmd.rest, bit c: this warp's tile of chunk c holds one of the listed tokens
+        const bool rest = KIND == kPassTarget && cmd.rest != 0;
         const unsigned long long gone_tiles_of_warp =
-            KIND == kPassRest ? ((unsigned long long)sm.gone_chunks[warp][1] << 32) | sm.gone_chunks[warp][0] : 0ull;
+            rest ? ((unsigned long long)sm.gone_chunks[warp][1] << 32) | sm.gone_chunks[warp][0] : 0ull;
         consume(cmd, [&](int tile, const unsigned char* qt, const unsigned char* pt) {
-            if (KIND == kPassRest) {
-                Packed<T> pp;
-                load_pieces(pp, pt, lane);
-                float p[16];
-                if (CLEAN) m1 = fmaxf(m1, clean<T>(pp, p, saw_nan));
-                else pp.unpack(p);
-                exp16(p, cmd.kp, cmd.cp, p);
-                if ((gone_tiles_of_warp >> (tile / kTPC)) & 1ull) {
+            Packed<T> pq;
+            load_pieces(pq, rest ? pt : qt, lane);
+            float q[16];
+            if (CLEAN) m0 = fmaxf(m0, clean<T>(pq, q, saw_nan));
+            else pq.unpack(q);
+            exp16(q, cmd.kq, cmd.cq, q);
+            float s;
+            if (KIND == kPassTarget) {
+                if (rest && ((gone_tiles_of_warp >> (tile / kTPC)) & 1ull)) {
                     for (int i = 0; i < sm.n_gone_tok; ++i) {
                         const int o = sm.gone_tok[i] - tile * kTileElems;
                         if (o < 0 || o >= kTileElems) continue;
@@ -309,21 +313,10 @@ struct Ring {
                         if (l_ == lane) {
 #pragma unroll
                             for (int jj = 0; jj < 16; ++jj)
-                                if (jj == j_) p[jj] = 0.0f;
+                                if (jj == j_) q[jj] = 0.0f;
                         }
                     }
                 }
-                s0 += tree_sum16(p);
-                return;
-            }
-            Packed<T> pq;
-            load_pieces(pq, qt, lane);
-            float q[16];
-            if (CLEAN) m0 = fmaxf(m0, clean<T>(pq, q, saw_nan));
-            else pq.unpack(q);
-            exp16(q, cmd.kq, cmd.cq, q);
-            float s;
-            if (KIND == kPassTarget) {
                 s = tree_sum16(q);
                 s0 += s;
             } else {
@@ -422,9 +415,6 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             } else if (cmd.kind == kPassTarget) {
                 if (cmd.clean) ring.template work<kPassTarget, true, true>(cmd);
                 else ring.template work<kPassTarget, false, true>(cmd);
-            } else if (cmd.kind == kPassRest) {
-                if (cmd.clean) ring.template work<kPassRest, true, false>(cmd);
-                else ring.template work<kPassRest, false, false>(cmd);
             } else {
                 if (cmd.clean) {
                     if (cmd.store_tiles) ring.template work<kPassResidual, true, true>(cmd);
@@ -465,15 +455,16 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
     // results.  The first kSlots steps are taken before the command is published: what they wait for, if anything, are
     // slot uses of earlier passes, which every working warp finished before it reported its sums; so the copies travel
     // while the working warps wake up.  `meanwhile` runs on the control warp while the pass is under way.
-    auto run_pass = [&](int kind, bool store_tiles, double& S0, double& S1, float& M0, float& M1, auto&& meanwhile, auto&& early) {
-        const bool with_draft = kind != kPassTarget;
+    auto run_pass = [&](int kind, bool store_tiles, double& S0, double& S1, float& M0, float& M1, auto&& meanwhile, auto&& early, bool rest = false) {
+        const bool with_draft = kind != kPassTarget || rest;   // (the rest pass moves both rows like a residual pass: the ring stays as it is)
         int dir;
         unsigned long long parity, missing;
         ring.plan(dir, parity, missing);
         if (lane == 0) {
             PassCmd cmd;
             cmd.kind = kind; cmd.clean = st.has_nan ? 1 : 0; cmd.store_tiles = store_tiles ? 1 : 0;
-            cmd.kq = st.kq; cmd.kp = st.kp; cmd.cq = st.mq * st.kq; cmd.cp = st.mp * st.kp;
+            cmd.rest = rest ? 1 : 0;
+            cmd.kq = rest ? st.kp : st.kq; cmd.kp = st.kp; cmd.cq = rest ? st.mp * st.kp : st.mq * st.kq; cmd.cp = st.mp * st.kp;
             cmd.a_hi = st.a_hi; cmd.a_lo = st.a_lo;
             cmd.backward = dir; cmd.parity = parity;
             sm.cmd = cmd;
@@ -576,9 +567,11 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
         // What the test of child j needs and no pass changes: its token, its probabilities under the node's two rows,
         // whether an earlier sibling with the same token was rejected, and its uniform.
         int j = 0, x = -1;
-        double qx = 0.0, px_row = 0.0, qp = 0.0, U = 0.0;   // q(x), p(x), q(x) / p(x)
+        float qh_x = 0.0f, ph_x = 0.0f, qp = 0.0f;          // weights of x under the two rows; q(x) / p(x)
+        uint32_t U24 = 0u;                                 // the uniform, as 24 bits
         bool repeated = false, p_none = false;             // p_none: the draft row gives the token no mass (-inf or NaN)
-        const double inv_ratio = st.Sp * inv_Sq;
+        // log2(S_p / S_q) for the exponent of q(x)/p(x), by the fast logarithm (absolute error 2^-22)
+        const float lg_inv_ratio = lg2_approx((float)fmin(fmax(st.Sp * inv_Sq, 1e-37), 1e37));
         auto prepare = [&](int child) {
             float lq, lp;
             if (j < 32) {
@@ -591,20 +584,18 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
                 lp = RowIO<T>::scalar(rowp, x);
             }
             const float eq = fmaf(lq, st.kq, -st.mq * st.kq), ep = fmaf(lp, st.kp, -st.mp * st.kp);
-            const float qh = (lq == lq) ? ex2_approx(eq) : 0.0f;
-            const float ph = (lp == lp) ? ex2_approx(ep) : 0.0f;
-            qx = (double)qh * inv_Sq;
-            px_row = (double)ph * inv_Sp;
+            qh_x = (lq == lq) ? ex2_approx(eq) : 0.0f;
+            ph_x = (lp == lp) ? ex2_approx(ep) : 0.0f;
             // The test needs q(x) / p(x) only: taken from the difference of the exponents it survives probabilities
             // below the fp32 range (children drafted from the far tail of a peaked row), where q(x) and p(x) are both 0.
             p_none = !(lp == lp) || !(lp > kNegInf);
-            qp = (lq == lq && !p_none) ? (double)ex2_approx(eq - ep) * inv_ratio : 0.0;
+            qp = (lq == lq && !p_none) ? ex2_approx((eq - ep) + lg_inv_ratio) : 0.0f;
             bool mine = false;
 #pragma unroll
             for (int i = 0; i < 4; ++i) mine |= rem_x[i] == x;
             repeated = __any_sync(0xFFFFFFFFu, mine);   // its draft mass is gone (Eq. 1)
             const uint4 rw = rng_draw(key, (uint32_t)cur, kTagAccept, (uint32_t)j);
-            U = (double)(rw.x >> 8) * (1.0 / 16777216.0);
+            U24 = rw.x >> 8;
         };
         prepare(c);
         // 1 - P of the closed form, the draft mass still in play.  It is carried by subtraction while that is accurate:
@@ -631,20 +622,20 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             // Eq. 3 in closed form: accept iff U < min(1, r (1 - P) / (Z p(x))), r = (q(x) - A p(x))+, tested without
             // the division; a child the draft cannot produce any more is taken iff it has residual mass
             const bool no_draft = repeated || p_none;
+            const double px_row = (double)ph_x * inv_Sp, U = (double)U24 * (1.0 / 16777216.0);
             const double px = no_draft ? 0.0 : px_row;
             bool take;
-            double theta;
+            double g;   // the threshold times Z; with no draft mass: 1 or 0 times Z
             if (!no_draft) {   // U < min(1, (q/p - A)+ (1 - P) / Z)
-                const double g = fmax(qp - st.A, 0.0) * one_mP;
+                g = fmax((double)qp - st.A, 0.0) * one_mP;
                 take = U * st.Z < g;
-                theta = fmin(1.0, g / st.Z);
             } else {           // RSD_ST_ZERO_DRAFT_PROB
-                const double r = fmax(qx - st.A * px_row, 0.0);
+                const double r = fmax((double)qh_x * inv_Sq - st.A * px_row, 0.0);
                 status |= 8;
                 take = r > 0.0;
-                theta = r > 0.0 ? 1.0 : 0.0;
+                g = take ? st.Z : 0.0;
             }
-            if (a.dbg_theta && lane == 0) a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)theta;
+            if (a.dbg_theta && lane == 0) a.dbg_theta[(int64_t)b * a.num_nodes + c] = (float)fmin(1.0, g / st.Z);
             if (take) { accepted = c; break; }
             // rejected.  Eqs. 1-2 in closed form: A_{j+1} = A_j + Z_j / (1 - P_j), Z_{j+1} = sum (q - A_{j+1} p)+
             ++j;
@@ -688,7 +679,7 @@ __global__ void __launch_bounds__(kThreads, 3) verify_tree_ring_kernel(const Ver
             if (next >= 0 && err_new > 2e-6 * one_mP_new && n_removed < kMaxRemovedRing) {   // (every rejected token is listed)
                 double rest, none2;
                 float g0, g1;
-                run_pass(kPassRest, false, rest, none2, g0, g1, nothing, publish_gone);
+                run_pass(kPassTarget, true, rest, none2, g0, g1, nothing, publish_gone, true);
                 if (sm.abort) { aborted = true; break; }
                 one_mP_new = rest * inv_Sp;
                 err_new = 4e-7 * one_mP_new;
