@@ -127,7 +127,7 @@ int rsd_profile_next_scan(void* before, void* after);
  *   out_rows    [B][R][V] dense, the rows' element type; may not overlap the input
  *   out_kept    optional [B][R] int32: entries kept in each row;   status [B]
  * Values that compare equal (+0 and -0 among them) are one value: the smaller token goes first.
- * A row must fit in shared memory with the call's other data (up to about 99,000 2-byte or 49,000 4-byte entries);
+ * A row must fit in shared memory with the call's other data (up to about 101,000 2-byte or 50,700 4-byte entries);
  * longer rows are refused with RSD_ERR_UNSUPPORTED.  A row whose copy into shared memory does not arrive within about a
  * second sets RSD_ST_TIMEOUT for its sequence, and nothing is written for it.
  */

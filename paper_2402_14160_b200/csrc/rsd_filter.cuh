@@ -27,7 +27,8 @@ constexpr int kFineThreads = 256;                // threads that keep private bi
 constexpr int kBins = 16;                        // sub-intervals per search pass over the list
 constexpr int kCoarseBins = 2048;                // bins of the sweep over the row
 constexpr int kCountShift = 47;                  // a histogram entry: count << 47 | weight as fixed point, kept as two 32-bit halves
-constexpr int kListCap = 4096;                   // tokens gathered into a list (indices as 16 bits: rows up to 65,536)
+constexpr int kListCap = 2048;                   // tokens gathered into a list (indices as 16 bits: rows up to 65,536); sized so
+                                                 // that a 4-byte row of 50,272 entries still fits beside this kernel's other data
 constexpr float kValueRange = 24.0f;             // value-linear bins cover this many nats of value / T below the interval's top
 
 struct FilterArgs {

@@ -103,7 +103,7 @@ def test_filter_rows_degenerate_rows(rsd, dtype):
     # (equal entries put cumulative masses exactly on round fractions: rows whose cut the oracle calls borderline may differ)
     for top_k, top_p, T in ((0, 0.9, 1.0), (0, 0.5, 1.0), (100, 1.0, 1.0), (3000, 0.7, 1.0), (0, 0.99, 0.3), (0, 0.999999, 1.0)):
         _check_filter(rsd, rows, top_k, top_p, T, max_borderline=3)
-    big = _rows((1, 2, 70000), dtype, 2.0, 78) if dtype == "bf16" else _rows((1, 2, 40000), dtype, 2.0, 78)
+    big = _rows((1, 2, 70000), dtype, 2.0, 78) if dtype == "bf16" else _rows((1, 2, 50272), dtype, 2.0, 78)   # (fp32: OPT's vocabulary)
     _check_filter(rsd, big, 0, 0.9, 1.0)
     _check_filter(rsd, big, 500, 0.95, 1.0)
 
