@@ -278,3 +278,49 @@ def test_random_beam_search_trees_with_temperature():
     total.failures = []
     total.check()
     assert total.decisions > 1000 and total.final_mismatch <= max(1, 0.01 * total.final_draws)
+
+
+def test_random_residual_draws():
+    """rsd_resample_residual on random rows with random lists of rejected tokens (repeats allowed, the draft's mode
+    among them in a fifth of the rows), temperatures and offsets.  Rows stay within logits of standard deviation 2: with
+    both rows all but one-hot the residual is made of differences below fp32 resolution, which only the oracle's double
+    precision resolves."""
+    import paper_2402_14160_b200 as rsd
+    from tests.test_gpu_parity import _rows
+    rng = random.Random(61)
+    n_rows = mismatches = 0
+    for it in range(150):
+        V = (rng.choice([2, 5, 16, 17, 70, 515, 1000, 4099, 9999, 32000, 50272]) if rng.random() < 0.8 else rng.randint(2, 7000))
+        dtype = rng.choice(["f32", "bf16"])
+        sigma = rng.choice([0.05, 1.0, 2.0])
+        off = rng.choice([0, 0, 1, 3, 8])
+        Bq = rng.randint(1, 8)
+        d = _rows((Bq, V + 9), "f32", sigma, rng.randint(0, 1 << 30))
+        tg = d + _rows((Bq, V + 9), "f32", rng.choice([0.3, 1.0, 3.0]), rng.randint(0, 1 << 30))
+        dd = d.to(torch.bfloat16 if dtype == "bf16" else torch.float32)[:, off:off + V]
+        tt = tg.to(dd.dtype)[:, off:off + V]
+        nodes = torch.tensor([rng.randint(0, 3000) for _ in range(Bq)], dtype=torch.int32, device="cuda")
+        mk = rng.randint(1, 6)
+        rej = np.full((Bq, mk), -1, np.int32)
+        for b in range(Bq):
+            n = rng.randint(0, min(mk, V - 1))
+            vals = [rng.randrange(V) for _ in range(n)]
+            if rng.random() < 0.2 and n:
+                vals[0] = int(torch.argmax(dd[b].float()))
+            rej[b, :n] = vals
+        Td, Tt = rng.choice([1.0, 0.5, 2.0]), rng.choice([1.0, 0.5, 2.0])
+        seed, step, sb = rng.randint(0, 1 << 50), rng.randint(0, 1 << 20), rng.randint(0, 1 << 20)
+        g = _np(rsd.rsd_resample_residual(dd, tt, torch.from_numpy(rej).cuda(), nodes, seed, step, seq_base=sb, want_residual=True,
+                                          draft_temperature=Td, target_temperature=Tt))
+        o = oracle.resample_residual(workloads.as_oracle_rows(dd.contiguous()), workloads.as_oracle_rows(tt.contiguous()), rej,
+                                     nodes.cpu().numpy(), seed, step, seq_base=sb, draft_temperature=Td, target_temperature=Tt)
+        what = (it, V, dtype, sigma, Td, Tt, off, rej.tolist())
+        peak = o["residual"].max(axis=1, keepdims=True)
+        assert np.all(np.abs(g["residual"] - o["residual"]) <= 1e-5 * peak), what
+        differ = g["token"] != o["token"]
+        assert np.all(o["margin"][differ] <= 1e-5), (what, g["token"].tolist(), o["token"].tolist())
+        assert np.array_equal(g["status"], o["status"]), (what, g["status"].tolist(), o["status"].tolist())
+        n_rows += Bq
+        mismatches += int(differ.sum())
+    print("random residual draws: %d rows, %d borderline" % (n_rows, mismatches))
+    assert n_rows > 400 and mismatches <= max(1, n_rows // 200)
